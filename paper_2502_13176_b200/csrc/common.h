@@ -1,0 +1,24 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+#include "baklava.h"
+
+constexpr int kTile = 64;   // chunk lengths are multiples of this many tokens
+
+// Byte offsets of the regions of the decode workspace.
+struct DecodeWorkspace {
+    size_t control_off;    // 64 int32: launch-wide counters
+    size_t arrive_off;     // int32 [n_units]: chunks of a head that have delivered their partial result
+    size_t appended_off;   // int32 [n_units]: 1 if this step appended a row to the head
+    size_t partial_off;    // fp32 [n_items][g * D + 2 * g]: per-chunk (o, m, l)
+    size_t logit_off;      // fp32 [B * seq_stride_tokens][g]: log2-domain logits of this step
+    size_t total;
+};
+
+int baklava_check_shape(const baklava_shape* s);
+size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_units, int32_t B,
+                               int64_t seq_stride_tokens, DecodeWorkspace* layout);
+
+inline bool baklava_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -1,0 +1,255 @@
+// Bulk eviction (Eq. 5-6 applied to a whole prefilled head): choose which of T dense rows stay
+// under the head's budget and copy them, in position order, into the head's slab.
+//
+// Kernel 1 (one CTA per head) finds the score threshold of the heavy-hitter quota with an
+// 8-bit-per-pass radix select and lists the kept rows in ascending position.  Kernel 2 copies
+// the listed rows.  Ties at the threshold go to the earlier positions, so the kept set is the
+// first R rows of the order (sinks, recent window, then score descending / position ascending).
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "baklava.h"
+#include "common.h"
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kCopyThreads = 256;
+constexpr int kCopyRows = 64;   // rows per CTA of the copy kernel
+
+struct EvictParams {
+    __nv_bfloat16* k_slab;
+    __nv_bfloat16* v_slab;
+    int32_t* pos;
+    float* score;
+    int32_t* len;
+    int32_t* free_slot;
+    const int32_t* cap;
+    const int64_t* slab_off;
+    int64_t seq_stride;
+    uint32_t* status;
+    int32_t B, L, Hkv, n_sink, recent_num, recent_den;
+    int32_t layer_begin;
+    const __nv_bfloat16* k_dense;
+    const __nv_bfloat16* v_dense;
+    const float* score_dense;
+    int32_t T, reserve;
+    int64_t stride_layer, stride_seq, stride_head;
+    int32_t* kept;   // [n_units][T]
+};
+
+struct Where {
+    int head, st;
+    int64_t dense0, slab0;
+};
+
+__device__ __forceinline__ Where locate(const EvictParams& p, int unit) {
+    const int li = unit / (p.B * p.Hkv);
+    const int rem = unit - li * (p.B * p.Hkv);
+    const int b = rem / p.Hkv, h = rem - b * p.Hkv;
+    const int l = p.layer_begin + li;
+    Where w;
+    w.head = l * p.Hkv + h;
+    w.st = (b * p.L + l) * p.Hkv + h;
+    w.dense0 = (int64_t)li * p.stride_layer + (int64_t)b * p.stride_seq + (int64_t)h * p.stride_head;
+    w.slab0 = (int64_t)b * p.seq_stride + p.slab_off[w.head];
+    return w;
+}
+
+// fp32 -> uint32 whose unsigned order is the float order (-0 counted as +0)
+__device__ __forceinline__ uint32_t ordered_bits(float x) {
+    const uint32_t b = __float_as_uint(x + 0.0f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// exclusive prefix sum of one int per thread over the CTA; returns the CTA total in `total`
+__device__ __forceinline__ int block_exclusive_scan(int x, int* warp_sums, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_sums[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += y;
+        }
+        warp_sums[lane] = w;   // inclusive over warps
+    }
+    __syncthreads();
+    const int before = warp > 0 ? warp_sums[warp - 1] : 0;
+    total = warp_sums[31];
+    __syncthreads();
+    return before + incl - x;
+}
+
+__global__ void __launch_bounds__(kSelThreads) evict_select_kernel(const EvictParams p) {
+    __shared__ int hist[256];
+    __shared__ int warp_sums[32];
+    __shared__ uint32_t sh_prefix;
+    __shared__ int sh_want;
+
+    const int unit = blockIdx.x, tid = threadIdx.x;
+    const Where w = locate(p, unit);
+    const int C = p.cap[w.head];
+    const int R = C - p.reserve;
+    int32_t* kept = p.kept + (int64_t)unit * p.T;
+    const int T = p.T;
+    if (R < 1) {
+        if (tid == 0) { atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE); p.len[w.st] = 0; p.free_slot[w.st] = 0; }
+        return;
+    }
+    if (T <= R) {
+        for (int j = tid; j < T; j += kSelThreads) kept[j] = j;
+        if (tid == 0) { p.len[w.st] = T; p.free_slot[w.st] = T; }
+        return;
+    }
+    const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
+    const int lo = min(p.n_sink, T);          // candidates are positions lo .. hi-1
+    const int hi = max(lo, T - W);
+    const int quota = R - lo - (T - hi);      // heavy hitters to pick among the candidates
+    if (quota < 0 || quota > hi - lo) {
+        if (tid == 0) { atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE); p.len[w.st] = 0; p.free_slot[w.st] = 0; }
+        return;
+    }
+    const float* sc = p.score_dense ? p.score_dense + w.dense0 : nullptr;
+
+    // radix select: the `quota`-th largest ordered score among the candidates
+    uint32_t prefix = 0;      // bits decided so far (from the top)
+    int want = quota;         // how many still to take among rows matching the prefix
+    if (quota > 0) {
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
+            __syncthreads();
+            const uint32_t mask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
+            for (int j = lo + tid; j < hi; j += kSelThreads) {
+                const uint32_t key = ordered_bits(sc ? sc[j] : 0.0f);
+                if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int left = want, bin = 255;
+                for (; bin > 0; --bin) {
+                    if (hist[bin] >= left) break;
+                    left -= hist[bin];
+                }
+                sh_prefix = prefix | ((uint32_t)bin << shift);
+                sh_want = left;
+            }
+            __syncthreads();
+            prefix = sh_prefix;
+            want = sh_want;
+            __syncthreads();
+        }
+    }
+    // rows with key > prefix are in; of the rows with key == prefix the first `want` by position
+
+    int base_eq = 0, base_out = 0;
+    for (int j0 = 0; j0 < T; j0 += kSelThreads) {
+        const int j = j0 + tid;
+        const bool in_range = j < T;
+        const bool cand = in_range && j >= lo && j < hi;
+        uint32_t key = 0;
+        if (cand) key = ordered_bits(sc ? sc[j] : 0.0f);
+        const int is_eq = (cand && quota > 0 && key == prefix) ? 1 : 0;
+        int total_eq;
+        const int eq_rank = base_eq + block_exclusive_scan(is_eq, warp_sums, total_eq);
+        bool keep = in_range && !cand;                       // sinks and the recent window
+        if (cand && quota > 0) keep = key > prefix || (is_eq && eq_rank < want);
+        int total_keep;
+        const int rank = base_out + block_exclusive_scan(keep ? 1 : 0, warp_sums, total_keep);
+        if (keep) kept[rank] = j;
+        base_eq += total_eq;
+        base_out += total_keep;
+    }
+    if (tid == 0) { p.len[w.st] = R; p.free_slot[w.st] = R; }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kCopyThreads) evict_copy_kernel(const EvictParams p) {
+    const int unit = blockIdx.x;
+    const Where w = locate(p, unit);
+    const int n = p.len[w.st];
+    const int r0 = blockIdx.y * kCopyRows;
+    if (r0 >= n) return;
+    const int32_t* kept = p.kept + (int64_t)unit * p.T;
+    constexpr int kVec = D / 8;                       // 16-byte pieces per row
+    constexpr int kPerRow = 2 * kVec;                 // K and V
+    constexpr int kRowsPerPass = kCopyThreads / kPerRow;
+    const int sub = threadIdx.x / kPerRow, piece = threadIdx.x % kPerRow;
+    for (int r = r0 + sub; r < min(r0 + kCopyRows, n); r += kRowsPerPass) {
+        const int src = kept[r];
+        const bool is_v = piece >= kVec;
+        const int c = is_v ? piece - kVec : piece;
+        const uint4* from = reinterpret_cast<const uint4*>((is_v ? p.v_dense : p.k_dense) + (w.dense0 + src) * D) + c;
+        uint4* to = reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + (w.slab0 + r) * D) + c;
+        *to = __ldg(from);
+        if (piece == 0) {
+            p.pos[w.slab0 + r] = src;
+            p.score[w.slab0 + r] = p.score_dense ? p.score_dense[w.dense0 + src] + 0.0f : 0.0f;
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) size_t baklava_evict_workspace_size(const baklava_shape* shape, int32_t B, int32_t layers, int32_t T) {
+    if (!shape || B <= 0 || layers <= 0 || T <= 0) return 0;
+    return (size_t)B * layers * shape->Hkv * (size_t)T * sizeof(int32_t);
+}
+
+extern "C" __attribute__((visibility("default"))) int baklava_evict(const baklava_shape* shape, const baklava_cache* cache,
+                             int32_t layer_begin, int32_t layer_end,
+                             const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
+                             int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
+                             void* ws, size_t ws_bytes, void* stream) {
+    int rc = baklava_check_shape(shape);
+    if (rc) return rc;
+    if (!cache || !ws) return BAKLAVA_ERR_INVALID_ARG;
+    if (!k_dense || !v_dense) return BAKLAVA_ERR_UNSUPPORTED;   // in-place compaction of a slab
+    if (!cache->k_slab || !cache->v_slab || !cache->pos || !cache->score || !cache->len || !cache->free_slot ||
+        !cache->cap || !cache->slab_off || !cache->status || cache->B <= 0 || cache->seq_stride_tokens <= 0)
+        return BAKLAVA_ERR_INVALID_ARG;
+    if (layer_begin < 0 || layer_end > shape->L || layer_begin >= layer_end) return BAKLAVA_ERR_INVALID_ARG;
+    if (T <= 0 || reserve < 1 || stride_layer < 0 || stride_seq < 0 || stride_head < T) return BAKLAVA_ERR_INVALID_ARG;
+    const void* ptrs[] = {k_dense, v_dense, cache->k_slab, cache->v_slab, ws};
+    for (const void* ptr : ptrs)
+        if (!baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
+    const int layers = layer_end - layer_begin;
+    if (ws_bytes < baklava_evict_workspace_size(shape, cache->B, layers, T)) return BAKLAVA_ERR_WORKSPACE;
+    const int64_t units = (int64_t)layers * cache->B * shape->Hkv;
+    const int64_t row_blocks = ((int64_t)T + kCopyRows - 1) / kCopyRows;
+    if (units > INT32_MAX || row_blocks > 65535) return BAKLAVA_ERR_UNSUPPORTED;
+
+    EvictParams p;
+    p.k_slab = static_cast<__nv_bfloat16*>(cache->k_slab);
+    p.v_slab = static_cast<__nv_bfloat16*>(cache->v_slab);
+    p.pos = cache->pos; p.score = cache->score; p.len = cache->len; p.free_slot = cache->free_slot;
+    p.cap = cache->cap; p.slab_off = cache->slab_off; p.seq_stride = cache->seq_stride_tokens;
+    p.status = cache->status;
+    p.B = cache->B; p.L = shape->L; p.Hkv = shape->Hkv;
+    p.n_sink = shape->n_sink; p.recent_num = shape->recent_num; p.recent_den = shape->recent_den;
+    p.layer_begin = layer_begin;
+    p.k_dense = static_cast<const __nv_bfloat16*>(k_dense);
+    p.v_dense = static_cast<const __nv_bfloat16*>(v_dense);
+    p.score_dense = score_dense;
+    p.T = T; p.reserve = reserve;
+    p.stride_layer = stride_layer; p.stride_seq = stride_seq; p.stride_head = stride_head;
+    p.kept = static_cast<int32_t*>(ws);
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    evict_select_kernel<<<(unsigned)units, kSelThreads, 0, s>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    const dim3 grid((unsigned)units, (unsigned)row_blocks);
+    if (shape->D == 128) evict_copy_kernel<128><<<grid, kCopyThreads, 0, s>>>(p);
+    else evict_copy_kernel<64><<<grid, kCopyThreads, 0, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
+}
