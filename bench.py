@@ -1,0 +1,283 @@
+#!/usr/bin/env python
+"""Decode-step benchmark: retained-KV GB/s of append + attention + score update + eviction over all
+layers of a synthetic LLaMA-3-8B-shaped cache (32K context, 30 % budget) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama|qwen|tiny] [--impl ours|reference]
+
+Prints one JSON line.  `value` is timed with the cache resident in HBM; `e2e` copies each step's
+q / k_new / v_new from pinned host memory and reads the output back inside the timed region.
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+With N > 1 (under torchrun) every rank runs an independent replica of the workload.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2502_13176_b200 import workloads as wl  # noqa: E402
+
+METRIC = "decode-step retained-KV GB/s"
+WORKLOADS = {"llama": wl.LLAMA3_8B_32K, "qwen": wl.QWEN25_7B_8K_B16, "tiny": wl.TINY}
+# dram bytes (read + write) per launch of the dominant kernel from the committed ncu capture, scaled
+# to this workload; None until a capture of the current kernel exists (see profiles/).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) != 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[2:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w, seconds_target=15.0):
+    """Time the CPU oracle's decode step on sampled heads of the workload.  Returns a cpu_baseline dict."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    import threadpoolctl
+
+    from oracle import allocation as oalloc
+    from oracle.cache import HeadCache
+    from paper_2502_13176_b200 import synth
+
+    imp = wl.importance(w).numpy()
+    cap, _, _ = oalloc.allocate(imp, w.t, w.r_num, w.r_den, w.total_pages, w.min_pages, w.max_pages, w.page)
+    cores = os.cpu_count() or 1
+    n_heads = min(w.L * w.Hkv * w.B, max(cores, 16))
+    rng_heads = [(i * (w.L * w.Hkv) // n_heads) for i in range(n_heads)]
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    twins, feeds = [], []
+    for j, flat in enumerate(rng_heads):
+        l, h = divmod(flat, w.Hkv)
+        C = int(cap[l, h]); n = C - 1
+        K = synth.normal_bf16(w.seed, 40, (n, w.D), gen_dev, None, j * 1 << 24).double().cpu().numpy()
+        V = synth.normal_bf16(w.seed, 41, (n, w.D), gen_dev, None, j * 1 << 24).double().cpu().numpy()
+        sc = synth.uniform_f64(w.seed, 42, j * 1 << 20, n).numpy()
+        hc = HeadCache(C, w.D, w.n_sink, w.recent_num, w.recent_den)
+        hc.load(K, V, np.arange(n), sc)
+        twins.append(hc)
+        feeds.append([synth.normal_bf16(w.seed, 43 + i, (w.g + 2, w.D), "cpu", None, j * 4096).double().numpy()
+                      for i in range(3)])
+
+    def one(args):
+        hc, feed, s = args
+        hc.step(feed[:w.g], feed[w.g], feed[w.g + 1], w.T + s)
+        return hc.C * w.D * 4
+
+    total_bytes, steps_done = 0, 0
+    t0 = time.perf_counter()
+    with threadpoolctl.threadpool_limits(limits=1):
+        with ThreadPoolExecutor(max_workers=cores) as pool:
+            while steps_done < 3:
+                total_bytes += sum(pool.map(one, [(hc, f[steps_done], steps_done) for hc, f in zip(twins, feeds)]))
+                steps_done += 1
+                if time.perf_counter() - t0 > seconds_target:
+                    break
+    dt = time.perf_counter() - t0
+    return {"value": total_bytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+            "sample": "%d of %d heads x %d decode steps (fp64 numpy, one thread per head)" % (
+                n_heads, w.L * w.Hkv * w.B, steps_done), "seconds": dt}
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for _ in range(args.warmup):
+        oracle_sample(w, seconds_target=2.0)
+    t_all = time.perf_counter()
+    for _ in range(args.steps):
+        vals.append(oracle_sample(w, seconds_target=5.0))
+    dt = time.perf_counter() - t_all
+    v = statistics.mean(x["value"] for x in vals)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(1, args.steps) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name},
+        "cpu_baseline": {"value": v, "unit": "GB/s", "cores": vals[-1]["cores"], "kind": "oracle",
+                         "sample": vals[-1]["sample"]},
+        "e2e": {"value": v, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--workload", default="llama", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="only the first LAYERS layers (for profiling a small case)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = WORKLOADS[args.workload]
+    if args.layers:
+        w = wl.scaled(w, L=args.layers)
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    from paper_2502_13176_b200 import binding as bk
+    from paper_2502_13176_b200.engine import DecodeSession
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    bk.lib()                                             # fail now if the library is missing
+    sess = DecodeSession(w, dev)
+    sess.prefill_synthetic()
+    total = args.warmup + args.steps
+    feeds = [wl.decode_inputs(w, i, sess.scales, dev) for i in range(2 * total)]
+    torch.cuda.synchronize(dev)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(dev)
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        sess.step(*feeds[i])
+    rows_per_step = int(sess.cache.len.sum().item()) + sess.plan.info.n_units   # rows attended: retained + new
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    with ClockSampler(local) as clocks:
+        ev[0].record()
+        for i in range(args.steps):
+            sess.step(*feeds[args.warmup + i])
+            ev[i + 1].record()
+        torch.cuda.synchronize(dev)
+    barrier()
+    sess.check_status()
+    per_step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    elapsed_ms = ev[0].elapsed_time(ev[-1])
+
+    # ---- end to end: host buffers in, host buffer out, every step
+    host = [tuple(t.cpu().pin_memory() for t in feeds[total + i]) for i in range(total)]
+    dq, dk, dv = (torch.empty_like(t, device=dev) for t in host[0])
+    out_host = torch.empty(sess.out.shape, dtype=sess.out.dtype).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host[0])
+    d2h = out_host.numel() * out_host.element_size()
+
+    def e2e_step(i):
+        q, k, v = host[i]
+        dq.copy_(q, non_blocking=True); dk.copy_(k, non_blocking=True); dv.copy_(v, non_blocking=True)
+        out_host.copy_(sess.step(dq, dk, dv), non_blocking=True)
+
+    for i in range(args.warmup):
+        e2e_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        e2e_step(args.warmup + i)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    sess.check_status()
+
+    times = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
+    elapsed_ms, e2e_ms = times.tolist()
+
+    if rank == 0:
+        bytes_per_step = rows_per_step * w.D * 2 * 2          # K and V rows, bf16
+        gbs = world * bytes_per_step * args.steps / (elapsed_ms * 1e-3) / 1e9
+        e2e_gbs = world * bytes_per_step * args.steps / (e2e_ms * 1e-3) / 1e9
+        peak, peak_kind = measured_peaks()
+        kernel_ms = statistics.mean(per_step_ms)
+        achieved = bytes_per_step / (kernel_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.L, "batch": w.B, "context": w.T, "budget": w.budget,
+                       "kv_bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (no flush)",
+                       "launch": "one baklava_decode_attn call per step covering all layers",
+                       "replicas": world},
+            "tokens_per_s": world * w.B * args.steps / (elapsed_ms * 1e-3),
+            "pct_of_hbm_peak": 100.0 * gbs / world / peak,
+            "ms_per_step_median": statistics.median(per_step_ms),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                         "peak_kind": peak_kind, "kernel": "decode_chunk_kernel",
+                         "note": "events bracket one call = append kernel + decode kernel"},
+            "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clocks.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            cb = oracle_sample(w)
+            cb.pop("seconds")
+            line["cpu_baseline"] = cb
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

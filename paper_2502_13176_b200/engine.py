@@ -1,0 +1,63 @@
+"""Convenience layer over the binding: owns the device buffers of one budgeted cache and drives
+allocate -> bulk evict -> decode steps.  Memory management and call sequencing only; every
+computation happens inside libbaklava.so."""
+import numpy as np
+import torch
+
+from . import binding as bk
+from . import workloads as wl
+
+
+def shape_of(w):
+    return bk.make_shape(w.L, w.Hq, w.Hkv, w.D, w.page, w.n_sink, w.recent_num, w.recent_den)
+
+
+class DecodeSession:
+    def __init__(self, w, device="cuda", layers=None, chunk_tokens=0, uniform=False):
+        self.w, self.device = w, torch.device(device)
+        self.shape = shape_of(w)
+        self.scales = wl.kv_scales(w)
+        self.importance = wl.importance(w).numpy()
+        self.cap, self.off, self.stride = bk.baklava_allocate(
+            self.shape, self.importance, w.t, 0 if uniform else w.r_num, w.r_den, w.total_pages * w.page,
+            w.min_pages * w.page, w.max_pages * w.page)
+        self.cache = bk.Cache(self.shape, self.cap, self.off, self.stride, w.B, self.device)
+        self.lb, self.le = (0, w.L) if layers is None else layers
+        n_sm = torch.cuda.get_device_properties(self.device).multi_processor_count
+        self.plan = bk.baklava_decode_plan(self.shape, self.cap, w.B, self.lb, self.le, self.stride,
+                                           chunk_tokens=chunk_tokens, n_sm=n_sm).to(self.device)
+        self.ws = bk.decode_workspace(self.plan, self.device)
+        nl = self.le - self.lb
+        self.out = torch.zeros((nl, w.B, w.Hq, w.D), dtype=torch.bfloat16, device=self.device)
+        self.lse = torch.zeros((nl, w.B, w.Hq), dtype=torch.float32, device=self.device)
+        self.t = 0
+
+    def prefill_synthetic(self):
+        """Fill every head from the workload's dense synthetic prompt through baklava_evict, a layer at a time."""
+        w = self.w
+        ews = torch.empty((bk.baklava_evict_workspace_size(self.shape, w.B, 1, w.T),), dtype=torch.uint8,
+                          device=self.device)
+        for l in range(self.lb, self.le):
+            k, v = wl.dense_kv_layer(w, l, self.scales, self.device)
+            sc = wl.prefill_scores(w, l, self.device)
+            bk.baklava_evict(self.shape, self.cache, l, l + 1, k, v, sc, w.T, 0, w.Hkv * w.T, w.T, 1, ews)
+            torch.cuda.synchronize(self.device)
+        self.t = w.T
+
+    def step(self, q, k_new, v_new, flags=0):
+        """One decode step for the session's layer range; returns the output tensor (device, bf16)."""
+        bk.baklava_decode_attn(self.shape, self.cache, q, k_new, v_new, self.t, self.out, self.lse, flags,
+                               self.plan, self.ws)
+        if not (flags & bk.FLAG_NO_APPEND):
+            self.t += 1
+        return self.out
+
+    def retained_kv_bytes(self):
+        """Bytes of K and V in valid rows of the session's layers: what one step must read."""
+        n = int(self.cache.len[:, self.lb:self.le].sum().item())
+        return n * self.w.D * 2 * 2
+
+    def check_status(self):
+        code = int(self.cache.status.item())
+        if code:
+            raise RuntimeError("device status word = %d" % code)
