@@ -40,7 +40,7 @@ def _run_case(L, Hkv, B, D, T, caps, n_sink, num, den, score_mode, reserve=1, se
             for h in range(Hkv):
                 C = int(cap[l, h])
                 s_in = np.zeros(T, np.float32) if scc is None else scc[l, b, h, :T]
-                _, _, pos2, s2, idx = oe.bulk_evict(kc[l, b, h, :T], vc[l, b, h, :T], np.arange(T), s_in,
+                _, _, pos2, s2, idx = oe.bulk_evict(kc[l, b, h, :T].double().numpy(), vc[l, b, h, :T].double().numpy(), np.arange(T), s_in,
                                                     C - reserve, n_sink, num, den)
                 n = len(pos2)
                 assert int(cache.len[b, l, h]) == n and int(cache.free_slot[b, l, h]) == n
