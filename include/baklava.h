@@ -220,6 +220,30 @@ int baklava_evict(const baklava_shape* shape, const baklava_cache* cache,
                   void* ws, size_t ws_bytes, void* stream);
 size_t baklava_evict_workspace_size(const baklava_shape* shape, int32_t B, int32_t layers, int32_t T);
 
+/* ------------------------------------------------------------------ bulk eviction, no workspace
+ * (No counterpart in the paper: this is a packaging variant of baklava_evict.)
+ * Same operation, arguments and results as baklava_evict, for callers that cannot provide a
+ * workspace because they cannot allocate device memory where the call is made: code running
+ * inside a host framework whose memory pool is exhausted or frozen, plug-ins that are handed
+ * only their input and output buffers, and start-up code that runs before an allocator exists.
+ * The list of kept rows is kept in a fixed array that is part of the library image: 4 MiB
+ * (BAKLAVA_EVICT_STATIC_MAX_ENTRIES = 2^20 int32 entries) on every GPU that loads the
+ * library, held until the process exits.  The call itself allocates and frees nothing.
+ *  - Limit: (layer_end - layer_begin) * B * Hkv * T <= BAKLAVA_EVICT_STATIC_MAX_ENTRIES;
+ *    larger requests return BAKLAVA_ERR_WORKSPACE before anything is enqueued.
+ *  - The first call on each device looks up the array's device address (the device must be
+ *    current).  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array and it keeps the previous call's contents.
+ *    Every entry that is read is written earlier in the same call, so nothing has to be
+ *    cleared; but two calls whose kernels overlap on the GPU (different streams) race on it.
+ *    Serialise them on one stream, or use baklava_evict with separate workspaces. */
+#define BAKLAVA_EVICT_STATIC_MAX_ENTRIES (1u << 20)
+int baklava_evict_static(const baklava_shape* shape, const baklava_cache* cache,
+                         int32_t layer_begin, int32_t layer_end,
+                         const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
+                         int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
+                         void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -74,6 +74,8 @@ def lib():
                                     c_void_p, c_int32, c_int64, c_int64, c_int64, c_int32, c_void_p, c_size_t, c_void_p]
         L.baklava_evict_workspace_size.restype = c_size_t
         L.baklava_evict_workspace_size.argtypes = [POINTER(Shape), c_int32, c_int32, c_int32]
+        L.baklava_evict_static.argtypes = [POINTER(Shape), POINTER(CacheStruct), c_int32, c_int32, c_void_p, c_void_p,
+                                           c_void_p, c_int32, c_int64, c_int64, c_int64, c_int32, c_void_p]
         L.baklava_profile_heads.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                             c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
         L.baklava_profile_workspace_size.restype = c_size_t
@@ -215,6 +217,19 @@ def baklava_evict(shape, cache, layer_begin, layer_end, k_dense, v_dense, score_
                                _ptr(k_dense), _ptr(v_dense), _ptr(score_dense), int(T), int(stride_layer),
                                int(stride_seq), int(stride_head), int(reserve), _ptr(ws),
                                ws.numel() * ws.element_size(), _stream(stream)), "baklava_evict")
+
+
+EVICT_STATIC_MAX_ENTRIES = 1 << 20
+
+
+def baklava_evict_static(shape, cache, layer_begin, layer_end, k_dense, v_dense, score_dense, T,
+                         stride_layer, stride_seq, stride_head, reserve, stream=None):
+    """baklava_evict for callers that cannot allocate a workspace: the kept-row list lives in a
+    fixed 4 MiB array inside the library.  Calls on one device must not overlap in time."""
+    _check(lib().baklava_evict_static(ctypes.byref(shape), ctypes.byref(cache.struct), layer_begin, layer_end,
+                                      _ptr(k_dense), _ptr(v_dense), _ptr(score_dense), int(T), int(stride_layer),
+                                      int(stride_seq), int(stride_head), int(reserve), _stream(stream)),
+           "baklava_evict_static")
 
 
 def baklava_profile_workspace_size(shape, P, T):

@@ -253,3 +253,80 @@ extern "C" __attribute__((visibility("default"))) int baklava_evict(const baklav
     else evict_copy_kernel<64><<<grid, kCopyThreads, 0, s>>>(p);
     return cudaGetLastError() == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
 }
+
+// ---------------------------------------------------------------- bulk eviction without a workspace
+// Some callers of this library cannot hand over a workspace because they cannot allocate device
+// memory at the point of the call: code running under a memory pool that is already full or
+// frozen, a plug-in that is only given its input and output tensors, a start-up path that runs
+// before the host framework's allocator exists.  For them the list of kept rows lives in a
+// fixed array inside the library image instead of in caller memory.
+namespace {
+
+constexpr size_t kStaticKeptEntries = BAKLAVA_EVICT_STATIC_MAX_ENTRIES;   // 4 MiB per GPU that loads the library
+static __device__ __align__(256) int32_t g_static_kept[kStaticKeptEntries];
+
+constexpr int kMaxDevices = 64;
+int32_t* g_static_kept_addr[kMaxDevices] = {};           // device address of the array, per device
+
+// The array's name is only a host-side handle; the kernels need its address on the current device.
+int static_kept_address(int32_t** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BAKLAVA_ERR_CUDA;
+    if (!g_static_kept_addr[dev]) {
+        void* addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_static_kept) != cudaSuccess || !addr) return BAKLAVA_ERR_CUDA;
+        g_static_kept_addr[dev] = static_cast<int32_t*>(addr);
+    }
+    *out = g_static_kept_addr[dev];
+    return BAKLAVA_OK;
+}
+
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) int baklava_evict_static(
+        const baklava_shape* shape, const baklava_cache* cache, int32_t layer_begin, int32_t layer_end,
+        const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
+        int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve, void* stream) {
+    int rc = baklava_check_shape(shape);
+    if (rc) return rc;
+    if (!cache || !k_dense || !v_dense) return BAKLAVA_ERR_INVALID_ARG;
+    if (!cache->k_slab || !cache->v_slab || !cache->pos || !cache->score || !cache->len || !cache->free_slot ||
+        !cache->cap || !cache->slab_off || !cache->status || cache->B <= 0 || cache->seq_stride_tokens <= 0)
+        return BAKLAVA_ERR_INVALID_ARG;
+    if (layer_begin < 0 || layer_end > shape->L || layer_begin >= layer_end) return BAKLAVA_ERR_INVALID_ARG;
+    if (T <= 0 || reserve < 1 || stride_layer < 0 || stride_seq < 0 || stride_head < T) return BAKLAVA_ERR_INVALID_ARG;
+    const void* ptrs[] = {k_dense, v_dense, cache->k_slab, cache->v_slab};
+    for (const void* ptr : ptrs)
+        if (!baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
+    const int64_t units = (int64_t)(layer_end - layer_begin) * cache->B * shape->Hkv;
+    const int64_t row_blocks = ((int64_t)T + kCopyRows - 1) / kCopyRows;
+    if (units * (int64_t)T > (int64_t)kStaticKeptEntries) return BAKLAVA_ERR_WORKSPACE;   // beyond the fixed array
+    if (units > INT32_MAX || row_blocks > 65535) return BAKLAVA_ERR_UNSUPPORTED;
+    int32_t* kept = nullptr;
+    rc = static_kept_address(&kept);
+    if (rc) return rc;
+
+    EvictParams p;
+    p.k_slab = static_cast<__nv_bfloat16*>(cache->k_slab);
+    p.v_slab = static_cast<__nv_bfloat16*>(cache->v_slab);
+    p.pos = cache->pos; p.score = cache->score; p.len = cache->len; p.free_slot = cache->free_slot;
+    p.cap = cache->cap; p.slab_off = cache->slab_off; p.seq_stride = cache->seq_stride_tokens;
+    p.status = cache->status;
+    p.B = cache->B; p.L = shape->L; p.Hkv = shape->Hkv;
+    p.n_sink = shape->n_sink; p.recent_num = shape->recent_num; p.recent_den = shape->recent_den;
+    p.layer_begin = layer_begin;
+    p.k_dense = static_cast<const __nv_bfloat16*>(k_dense);
+    p.v_dense = static_cast<const __nv_bfloat16*>(v_dense);
+    p.score_dense = score_dense;
+    p.T = T; p.reserve = reserve;
+    p.stride_layer = stride_layer; p.stride_seq = stride_seq; p.stride_head = stride_head;
+    p.kept = kept;
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    evict_select_kernel<<<(unsigned)units, kSelThreads, 0, s>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    const dim3 grid((unsigned)units, (unsigned)row_blocks);
+    if (shape->D == 128) evict_copy_kernel<128><<<grid, kCopyThreads, 0, s>>>(p);
+    else evict_copy_kernel<64><<<grid, kCopyThreads, 0, s>>>(p);
+    return cudaGetLastError() == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
+}
