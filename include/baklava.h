@@ -47,6 +47,7 @@ extern "C" {
 /* bits of the device status word */
 #define BAKLAVA_STATUS_OVERFLOW    1u   /* a token was offered to a cache with no free slot: not appended */
 #define BAKLAVA_STATUS_BAD_STATE   2u   /* len / free_slot outside [0, cap]: head skipped                  */
+#define BAKLAVA_STATUS_TIMEOUT     4u   /* a bounded wait inside a kernel gave up: that head's step is lost  */
 
 /* flags of baklava_decode_attn */
 #define BAKLAVA_FLAG_NO_APPEND     1u   /* attend over the cache as it is; k_new / v_new ignored      */

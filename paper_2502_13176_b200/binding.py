@@ -15,7 +15,7 @@ import torch
 OK = 0
 FLAG_NO_APPEND, FLAG_NO_SCORE, FLAG_NO_EVICT = 1, 2, 4
 SCOPE_LAYER, SCOPE_MODEL = 0, 1
-STATUS_OVERFLOW, STATUS_BAD_STATE = 1, 2
+STATUS_OVERFLOW, STATUS_BAD_STATE, STATUS_TIMEOUT = 1, 2, 4
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbaklava.so")
 _lib = None

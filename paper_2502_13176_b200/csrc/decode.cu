@@ -6,6 +6,12 @@
 // chunk's logits in the workspace.  The CTA that delivers the last partial of a head merges
 // them in chunk order, writes the output, turns the logits into probabilities with the final
 // normaliser, adds them to the scores and picks the row to evict in the same sweep.
+//
+// Inside a chunk: a producer warp streams 64-token K and V tiles with TMA (128-byte swizzle)
+// into a ring of shared-memory stages guarded by full/empty mbarriers; four consumer warps take
+// 16 tokens of each tile, contract the padded query group against K and the probabilities
+// against V with bf16 mma.sync (fp32 accumulate), and keep an online-softmax state each.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -17,10 +23,15 @@
 
 namespace {
 
-constexpr int kWarps = 4;
-constexpr int kThreads = kWarps * 32;
+constexpr int kConsumerWarps = 4;
+constexpr int kThreads = (kConsumerWarps + 1) * 32;     // + one producer warp
+constexpr int kTileTokens = kTile;                      // 64 tokens per stage
+constexpr int kWarpTokens = kTileTokens / kConsumerWarps;
+constexpr int kStages = 3;
+constexpr uint32_t kWaitLimit = 1u << 22;               // bounded mbarrier waits
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+static_assert(kWarpTokens == 16, "a consumer warp owns one 16-token MMA block of each tile");
 
 struct DecodeParams {
     __nv_bfloat16* k_slab;
@@ -33,7 +44,7 @@ struct DecodeParams {
     const int64_t* slab_off;
     int64_t seq_stride;
     uint32_t* status;
-    int32_t B, L, Hq, Hkv, n_sink, recent_num, recent_den;
+    int32_t B, L, Hq, Hkv, G, n_sink, recent_num, recent_den;
     int32_t layer_begin, layers;
     const __nv_bfloat16* q;
     const __nv_bfloat16* k_new;
@@ -103,45 +114,93 @@ __global__ void append_kernel(const DecodeParams p) {
     if (threadIdx.x == 0) p.appended[unit] = ok;
 }
 
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* ptr) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Waits for the phase with the given parity; gives up after kWaitLimit polls and returns false.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col); rows 8..15 of A are zero here
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    const uint32_t zero = 0u;
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(zero), "r"(a2), "r"(zero), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// Byte offset of 16-byte piece `piece` of row `row` inside a [64 rows][D] bf16 tile that TMA wrote with
+// the 128-byte swizzle: the tile is D/64 boxes of 64 rows x 128 bytes, each 1024-byte aligned, and piece
+// c of a box row sits at piece position c ^ (row % 8).
+__device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
+    return (uint32_t)((piece >> 3) * (kTileTokens * 128) + row * 128 + (((piece & 7) ^ (row & 7)) << 4));
+}
+
 // ---------------------------------------------------------------- steps 2-4
-template <int E>
-__device__ __forceinline__ void load_row(const __nv_bfloat16* row, int lane, float (&x)[E]) {
-    if constexpr (E == 4) {
-        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(row) + lane);
-        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-        x[0] = a.x; x[1] = a.y; x[2] = b.x; x[3] = b.y;
-    } else {
-        const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(row) + lane);
-        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw));
-        x[0] = a.x; x[1] = a.y;
-    }
-}
+template <int D>
+__global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodeParams p,
+                                                                const __grid_constant__ CUtensorMap k_map,
+                                                                const __grid_constant__ CUtensorMap v_map) {
+    constexpr int kKSteps = D / 16;                    // MMA k-steps over the head dimension
+    constexpr int kNTiles = D / 8;                     // 8-wide output column blocks
+    constexpr int kTileBytes = kTileTokens * D * 2;    // one K (or V) tile
+    constexpr int kStageBytes = 2 * kTileBytes;
+    constexpr int kG = BAKLAVA_MAX_GROUP;
 
-__device__ __forceinline__ float warp_sum(float x) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-    return x;
-}
-__device__ __forceinline__ float warp_max(float x) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
-    return x;
-}
-
-template <int D, int G>
-__global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodeParams p) {
-    constexpr int E = D / 32;   // elements of a row held by one lane
-    __shared__ float sm_o[kWarps][G][D];
-    __shared__ float sm_m[kWarps][G];
-    __shared__ float sm_l[kWarps][G];
-    __shared__ float sm_M[G];
-    __shared__ float sm_invL[G];
-    __shared__ unsigned long long sm_key[kWarps];
-    __shared__ int sm_slot[kWarps];
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[kStages];
+    __shared__ __align__(8) uint64_t bar_empty[kStages];
+    __shared__ float sm_m[kConsumerWarps][kG];
+    __shared__ float sm_l[kConsumerWarps][kG];
+    __shared__ float sm_M[kG];
+    __shared__ float sm_invL[kG];
+    __shared__ unsigned long long sm_key[kThreads / 32];
+    __shared__ int sm_slot[kThreads / 32];
     __shared__ int sm_last;
+    __shared__ int sm_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = p.G;
     const int4 item = p.items[blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
@@ -158,100 +217,182 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
     if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
+    const int n_tiles = end > begin ? (end - begin + kTileTokens - 1) / kTileTokens : 0;
     const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
 
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
-    const __nv_bfloat16* Kh = p.k_slab + row0 * D;
-    const __nv_bfloat16* Vh = p.v_slab + row0 * D;
-    float* logit_h = p.logit + row0 * G;
+    float* logit_h = p.logit + row0 * G;                  // [G][C] for this head
 
-    float qf[G][E];
-    {
-        const __nv_bfloat16* qrow = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
-#pragma unroll
-        for (int a = 0; a < G; ++a) {
-            load_row<E>(qrow + a * D, lane, qf[a]);
-#pragma unroll
-            for (int e = 0; e < E; ++e) qf[a][e] *= p.scale_log2;
-        }
-    }
-    float m[G], l[G], o[G][E];
-#pragma unroll
-    for (int a = 0; a < G; ++a) {
-        m[a] = -INFINITY;
-        l[a] = 0.0f;
-#pragma unroll
-        for (int e = 0; e < E; ++e) o[a][e] = 0.0f;
-    }
+    // 1024-byte aligned stage ring inside the dynamic shared memory
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
 
-    for (int tile = begin + warp * 32; tile < end; tile += kWarps * 32) {
-        const int cnt = min(32, end - tile);
-        float s_mine[G];
-#pragma unroll
-        for (int a = 0; a < G; ++a) s_mine[a] = -INFINITY;
-#pragma unroll 4
-        for (int j = 0; j < cnt; ++j) {
-            float kx[E];
-            load_row<E>(Kh + (int64_t)(tile + j) * D, lane, kx);
-#pragma unroll
-            for (int a = 0; a < G; ++a) {
-                float part = 0.0f;
-#pragma unroll
-                for (int e = 0; e < E; ++e) part = fmaf(qf[a][e], kx[e], part);
-                part = warp_sum(part);
-                if (lane == j) s_mine[a] = part;
-            }
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), kConsumerWarps);
         }
-        const bool valid = lane < cnt && (tile + lane) != hole;
-        if (keep_logits && lane < cnt) {
-#pragma unroll
-            for (int a = 0; a < G; ++a) logit_h[(int64_t)(tile + lane) * G + a] = s_mine[a];
-        }
-        float pr[G];
-#pragma unroll
-        for (int a = 0; a < G; ++a) {
-            const float s = valid ? s_mine[a] : -INFINITY;
-            const float m_new = fmaxf(m[a], warp_max(s));
-            const float corr = (m_new == -INFINITY) ? 1.0f : exp2f(m[a] - m_new);
-            pr[a] = valid ? exp2f(s - m_new) : 0.0f;
-            l[a] = l[a] * corr + warp_sum(pr[a]);
-#pragma unroll
-            for (int e = 0; e < E; ++e) o[a][e] *= corr;
-            m[a] = m_new;
-        }
-#pragma unroll 4
-        for (int j = 0; j < cnt; ++j) {
-            if (tile + j == hole) continue;
-            float vx[E];
-            load_row<E>(Vh + (int64_t)(tile + j) * D, lane, vx);
-#pragma unroll
-            for (int a = 0; a < G; ++a) {
-                const float pj = __shfl_sync(0xffffffffu, pr[a], j);
-#pragma unroll
-                for (int e = 0; e < E; ++e) o[a][e] = fmaf(pj, vx[e], o[a][e]);
-            }
-        }
-    }
-
-    // the four warps' states -> one partial for the chunk
-#pragma unroll
-    for (int a = 0; a < G; ++a) {
-#pragma unroll
-        for (int e = 0; e < E; ++e) sm_o[warp][a][lane * E + e] = o[a][e];
-        if (lane == 0) { sm_m[warp][a] = m[a]; sm_l[warp][a] = l[a]; }
+        sm_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    float* part = p.partial + (int64_t)blockIdx.x * (G * D + 2 * G);
+
+    // per-warp online-softmax state; row q of the group lives in the quad of lanes with lane / 4 == q
+    const int qrow = lane >> 2, qcol = (lane & 3) * 2;
+    float m_run = -INFINITY, l_run = 0.0f;
+    float o[kNTiles][4];
+#pragma unroll
+    for (int j = 0; j < kNTiles; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f; }
+
+    if (warp == kConsumerWarps) {
+        // ---------------- producer: one lane issues the TMA loads
+        if (lane == 0) {
+            for (int it = 0; it < n_tiles; ++it) {
+                const int s = it % kStages;
+                if (it >= kStages) {
+                    if (!mbar_wait(smem_u32(&bar_empty[s]), ((it / kStages) - 1) & 1)) {
+                        atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
+                        sm_abort = 1;
+                        break;
+                    }
+                }
+                const uint32_t full = smem_u32(&bar_full[s]);
+                const uint32_t dst = ring + s * kStageBytes;
+                const int y = (int)(row0 + begin + it * kTileTokens);
+                mbar_arrive_expect_tx(full, kStageBytes);
+#pragma unroll
+                for (int bx = 0; bx < D / 64; ++bx) {
+                    tma_load_2d(dst + bx * (kTileTokens * 128), &k_map, bx * 64, y, full);
+                    tma_load_2d(dst + kTileBytes + bx * (kTileTokens * 128), &v_map, bx * 64, y, full);
+                }
+            }
+        }
+    } else {
+        // ---------------- consumers
+        // query fragments (A operand): rows >= G are zero; a0 covers k 0..7 of a k-step, a2 k 8..15
+        uint32_t qa0[kKSteps], qa2[kKSteps];
+        {
+            const __nv_bfloat16* qrow_ptr = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + qrow) * D;
+#pragma unroll
+            for (int ks = 0; ks < kKSteps; ++ks) {
+                qa0[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + qcol) : 0u;
+                qa2[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + 8 + qcol) : 0u;
+            }
+        }
+        const int r0 = warp * kWarpTokens;                 // this warp's rows inside a tile
+        const int lm = lane >> 3, li8 = lane & 7;          // ldmatrix: matrix index and row inside it
+        bool alive = true;
+        for (int it = 0; it < n_tiles && alive; ++it) {
+            const int s = it % kStages;
+            if (!mbar_wait(smem_u32(&bar_full[s]), (it / kStages) & 1)) {
+                if (lane == 0) atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
+                alive = false;
+                break;
+            }
+            const uint32_t k_tile = ring + s * kStageBytes;
+            const uint32_t v_tile = k_tile + kTileBytes;
+            const int tok0 = begin + it * kTileTokens + r0;          // first token of this warp's block
+            const int valid = min(kWarpTokens, end - tok0);          // rows of the block inside the chunk
+            if (valid > 0) {
+                // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
+                if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
+                    uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
+                    for (int i = lane; i < kWarpTokens * (D / 8); i += 32) {
+                        const int r = i / (D / 8), c = i % (D / 8);
+                        if (r >= valid || tok0 + r == hole)
+                            *reinterpret_cast<uint4*>(v_ptr + tile_offset(r0 + r, c)) = make_uint4(0, 0, 0, 0);
+                    }
+                    __syncwarp();
+                }
+                // S = Q K^T for 16 tokens: two 8-token column blocks
+                float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+                for (int ks = 0; ks < kKSteps; ++ks) {
+                    uint32_t kb[4];
+                    ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kb);
+                    mma_bf16(sacc[0], qa0[ks], qa2[ks], kb[0], kb[1]);
+                    mma_bf16(sacc[1], qa0[ks], qa2[ks], kb[2], kb[3]);
+                }
+                // this thread: row qrow, tokens tok0 + 8 t + qcol + {0, 1}
+                float sv[4];
+                bool ok[4];
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int tok = tok0 + 8 * t + qcol + e;
+                        sv[2 * t + e] = sacc[t][e] * p.scale_log2;
+                        ok[2 * t + e] = tok < end && tok != hole;
+                    }
+                if (keep_logits && qrow < G) {
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        const int tok = tok0 + 8 * t + qcol;
+                        float* dst = logit_h + (int64_t)qrow * C + tok;
+                        if (tok + 1 < end) *reinterpret_cast<float2*>(dst) = make_float2(sv[2 * t], sv[2 * t + 1]);
+                        else if (tok < end) dst[0] = sv[2 * t];
+                    }
+                }
+                float mx = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) mx = fmaxf(mx, ok[i] ? sv[i] : -INFINITY);
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run, mx);
+                const float corr = (m_new == -INFINITY) ? 1.0f : exp2f(m_run - m_new);
+                float pv[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) pv[i] = ok[i] ? exp2f(sv[i] - m_new) : 0.0f;
+                l_run = l_run * corr + (pv[0] + pv[1]) + (pv[2] + pv[3]);
+                m_run = m_new;
+                if (__any_sync(0xffffffffu, corr != 1.0f)) {
+#pragma unroll
+                    for (int j = 0; j < kNTiles; ++j) { o[j][0] *= corr; o[j][1] *= corr; }
+                }
+                const uint32_t pa0 = pack_bf16(pv[0], pv[1]), pa2 = pack_bf16(pv[2], pv[3]);
+                // O += P V: V^T fragments through ldmatrix.trans, two 8-wide column blocks per load
+#pragma unroll
+                for (int j2 = 0; j2 < kNTiles / 2; ++j2) {
+                    uint32_t vb[4];
+                    ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * j2 + (lm >> 1)), vb);
+                    mma_bf16(o[2 * j2], pa0, pa2, vb[0], vb[1]);
+                    mma_bf16(o[2 * j2 + 1], pa0, pa2, vb[2], vb[3]);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
+        }
+        if (!alive && lane == 0) sm_abort = 1;
+    }
+    __syncthreads();
+    if (sm_abort) return;                                   // a bounded wait gave up: status word says so
+
+    // ---- the four warps' states -> one partial for the chunk (the ring is idle now: reuse it)
+    float* sm_o = reinterpret_cast<float*>(ring_ptr);       // [kConsumerWarps][G][D]
+    if (warp < kConsumerWarps) {
+        float lq = l_run;
+        lq += __shfl_xor_sync(0xffffffffu, lq, 1);
+        lq += __shfl_xor_sync(0xffffffffu, lq, 2);
+        if (qrow < G) {
+#pragma unroll
+            for (int j = 0; j < kNTiles; ++j)
+                *reinterpret_cast<float2*>(sm_o + ((warp * G + qrow) * D + 8 * j + qcol)) = make_float2(o[j][0], o[j][1]);
+            if ((lane & 3) == 0) { sm_m[warp][qrow] = m_run; sm_l[warp][qrow] = lq; }
+        }
+    }
+    __syncthreads();
+    const int psz = G * D + 2 * G;
+    float* part = p.partial + (int64_t)blockIdx.x * psz;
     for (int i = tid; i < G * D; i += kThreads) {
         const int a = i / D, d = i - a * D;
         float mm = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) mm = fmaxf(mm, sm_m[w][a]);
+        for (int w = 0; w < kConsumerWarps; ++w) mm = fmaxf(mm, sm_m[w][a]);
         float acc = 0.0f, lsum = 0.0f;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
+        for (int w = 0; w < kConsumerWarps; ++w) {
             const float c = (sm_m[w][a] == -INFINITY) ? 0.0f : exp2f(sm_m[w][a] - mm);
-            acc = fmaf(sm_o[w][a][d], c, acc);
+            acc = fmaf(sm_o[(w * G + a) * D + d], c, acc);
             lsum = fmaf(sm_l[w][a], c, lsum);
         }
         part[i] = acc;
@@ -268,19 +409,20 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     __threadfence();
 
     // ---- this CTA delivered the head's last partial: merge in chunk order and finish the step
-    const float* part0 = p.partial + (int64_t)(blockIdx.x - piece) * (G * D + 2 * G);
+    const float* part0 = p.partial + (int64_t)(blockIdx.x - piece) * psz;
     if (tid < G) {
         float mm = -INFINITY;
-        for (int c = 0; c < active; ++c) mm = fmaxf(mm, __ldcg(part0 + (int64_t)c * (G * D + 2 * G) + G * D + tid));
+        for (int c = 0; c < active; ++c) mm = fmaxf(mm, __ldcg(part0 + (int64_t)c * psz + G * D + tid));
         float ll = 0.0f;
         for (int c = 0; c < active; ++c) {
-            const float* pc = part0 + (int64_t)c * (G * D + 2 * G);
+            const float* pc = part0 + (int64_t)c * psz;
             const float mc = __ldcg(pc + G * D + tid);
             if (mc != -INFINITY) ll = fmaf(__ldcg(pc + G * D + G + tid), exp2f(mc - mm), ll);
         }
         sm_M[tid] = mm;
         sm_invL[tid] = ll > 0.0f ? 1.0f / ll : 0.0f;
-        if (p.lse) p.lse[(int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + tid] = ll > 0.0f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
+        if (p.lse)
+            p.lse[(int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + tid] = ll > 0.0f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
     }
     __syncthreads();
     __nv_bfloat16* orow = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
@@ -288,7 +430,7 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
         const int a = i / D;
         float acc = 0.0f;
         for (int c = 0; c < active; ++c) {
-            const float* pc = part0 + (int64_t)c * (G * D + 2 * G);
+            const float* pc = part0 + (int64_t)c * psz;
             const float mc = __ldcg(pc + G * D + a);
             if (mc != -INFINITY) acc = fmaf(__ldcg(pc + i), exp2f(mc - sm_M[a]), acc);
         }
@@ -302,14 +444,10 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     int best_slot = -1;
     if (keep_logits) {
         const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
-        float Mq[G], iL[G];
-#pragma unroll
-        for (int a = 0; a < G; ++a) { Mq[a] = sm_M[a]; iL[a] = sm_invL[a]; }
         for (int j = tid; j < n_hi; j += kThreads) {
             if (j == hole) continue;
             float inc = 0.0f;
-#pragma unroll
-            for (int a = 0; a < G; ++a) inc += exp2f(__ldcg(logit_h + (int64_t)j * G + a) - Mq[a]) * iL[a];
+            for (int a = 0; a < G; ++a) inc += exp2f(__ldcg(logit_h + (int64_t)a * C + j) - sm_M[a]) * sm_invL[a];
             const float sc = p.score[row0 + j] + inc;
             p.score[row0 + j] = sc;
             if (evict) {
@@ -336,7 +474,7 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     if (tid == 0) {
         if (appended) {
             if (evict) {
-                for (int w = 0; w < kWarps; ++w)
+                for (int w = 0; w < kThreads / 32; ++w)
                     if (sm_key[w] < best) { best = sm_key[w]; best_slot = sm_slot[w]; }
                 if (best_slot >= 0) {
                     p.free_slot[u.st] = best_slot;
@@ -354,33 +492,54 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     }
 }
 
-template <int D, int G>
-cudaError_t launch_chunks(const DecodeParams& p, cudaStream_t s) {
-    decode_chunk_kernel<D, G><<<p.n_items, kThreads, 0, s>>>(p);
-    return cudaGetLastError();
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// bf16 [rows, D] row-major, boxes of 64 rows x 64 elements (128 bytes), 128-byte swizzle, zero fill
+bool make_slab_map(CUtensorMap* map, void* base, int64_t rows, int D) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTileTokens};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int D>
-cudaError_t launch_for_group(int g, const DecodeParams& p, cudaStream_t s) {
-    switch (g) {
-        case 1: return launch_chunks<D, 1>(p, s);
-        case 2: return launch_chunks<D, 2>(p, s);
-        case 3: return launch_chunks<D, 3>(p, s);
-        case 4: return launch_chunks<D, 4>(p, s);
-        case 5: return launch_chunks<D, 5>(p, s);
-        case 6: return launch_chunks<D, 6>(p, s);
-        case 7: return launch_chunks<D, 7>(p, s);
-        default: return launch_chunks<D, 8>(p, s);
-    }
+cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
+    constexpr int kSmem = kStages * 2 * kTileTokens * D * 2 + 1024;
+    cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    decode_chunk_kernel<D><<<p.n_items, kThreads, kSmem, s>>>(p, km, vm);
+    return cudaGetLastError();
 }
 
 }  // namespace
 
-extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(const baklava_shape* shape, const baklava_cache* cache,
-                                   const void* q, const void* k_new, const void* v_new, int32_t t_pos,
-                                   void* out, float* lse, uint32_t flags,
-                                   const int32_t* items, const baklava_plan_info* info,
-                                   void* ws, size_t ws_bytes, void* stream) {
+extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
+        const baklava_shape* shape, const baklava_cache* cache,
+        const void* q, const void* k_new, const void* v_new, int32_t t_pos,
+        void* out, float* lse, uint32_t flags,
+        const int32_t* items, const baklava_plan_info* info,
+        void* ws, size_t ws_bytes, void* stream) {
     int rc = baklava_check_shape(shape);
     if (rc) return rc;
     if (!cache || !q || !out || !items || !info || !ws) return BAKLAVA_ERR_INVALID_ARG;
@@ -397,10 +556,16 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(const 
         info->B != cache->B || info->n_items <= 0 ||
         info->n_units != (info->layer_end - info->layer_begin) * cache->B * shape->Hkv)
         return BAKLAVA_ERR_INVALID_ARG;
+    const int64_t rows = (int64_t)cache->B * cache->seq_stride_tokens;
+    if (rows > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     DecodeWorkspace lay;
     const size_t need = baklava_decode_ws_bytes(shape, info->n_items, info->n_units, cache->B,
                                                 cache->seq_stride_tokens, &lay);
     if (ws_bytes < need) return BAKLAVA_ERR_WORKSPACE;
+
+    CUtensorMap k_map, v_map;
+    if (!make_slab_map(&k_map, cache->k_slab, rows, shape->D) || !make_slab_map(&v_map, cache->v_slab, rows, shape->D))
+        return BAKLAVA_ERR_CUDA;
 
     DecodeParams p;
     p.k_slab = static_cast<__nv_bfloat16*>(cache->k_slab);
@@ -414,7 +579,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(const 
     p.seq_stride = cache->seq_stride_tokens;
     p.status = cache->status;
     p.B = cache->B;
-    p.L = shape->L; p.Hq = shape->Hq; p.Hkv = shape->Hkv;
+    p.L = shape->L; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.G = shape->Hq / shape->Hkv;
     p.n_sink = shape->n_sink; p.recent_num = shape->recent_num; p.recent_den = shape->recent_den;
     p.layer_begin = info->layer_begin;
     p.layers = info->layer_end - info->layer_begin;
@@ -435,7 +600,6 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(const 
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int g = shape->Hq / shape->Hkv;
     cudaError_t err = cudaSuccess;
     if (!no_append) {
         if (shape->D == 128) append_kernel<128><<<info->n_units, 32, 0, s>>>(p);
@@ -443,6 +607,6 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(const 
         err = cudaGetLastError();
         if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     }
-    err = shape->D == 128 ? launch_for_group<128>(g, p, s) : launch_for_group<64>(g, p, s);
+    err = shape->D == 128 ? launch_chunks<128>(p, k_map, v_map, s) : launch_chunks<64>(p, k_map, v_map, s);
     return err == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
 }
