@@ -59,6 +59,9 @@ struct DecodeParams {
     int32_t* appended;
     float* partial;
     float* logit;
+    float* stats;                  // [n_units][2 * kG]
+    unsigned long long* best_key;  // [n_items]
+    int32_t* best_slot;            // [n_items]
     float scale_log2;   // log2(e) / sqrt(D)
 };
 
@@ -194,8 +197,6 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     __shared__ float sm_l[kConsumerWarps][kG];
     __shared__ float sm_M[kG];
     __shared__ float sm_invL[kG];
-    __shared__ unsigned long long sm_key[kThreads / 32];
-    __shared__ int sm_slot[kThreads / 32];
     __shared__ int sm_last;
     __shared__ int sm_abort;
 
@@ -408,7 +409,8 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     if (!sm_last) return;
     __threadfence();
 
-    // ---- this CTA delivered the head's last partial: merge in chunk order and finish the step
+    // ---- this CTA delivered the head's last partial: merge them in chunk order, write the output
+    // and leave the final (max, 1 / sum) of every query head for the score kernel
     const float* part0 = p.partial + (int64_t)(blockIdx.x - piece) * psz;
     if (tid < G) {
         float mm = -INFINITY;
@@ -419,8 +421,11 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
             const float mc = __ldcg(pc + G * D + tid);
             if (mc != -INFINITY) ll = fmaf(__ldcg(pc + G * D + G + tid), exp2f(mc - mm), ll);
         }
+        const float inv = ll > 0.0f ? 1.0f / ll : 0.0f;
         sm_M[tid] = mm;
-        sm_invL[tid] = ll > 0.0f ? 1.0f / ll : 0.0f;
+        sm_invL[tid] = inv;
+        p.stats[(int64_t)unit * 2 * kG + tid] = mm;
+        p.stats[(int64_t)unit * 2 * kG + kG + tid] = inv;
         if (p.lse)
             p.lse[(int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + tid] = ll > 0.0f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
     }
@@ -428,34 +433,132 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     __nv_bfloat16* orow = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
     for (int i = tid; i < G * D; i += kThreads) {
         const int a = i / D;
+        const float Ma = sm_M[a];
         float acc = 0.0f;
-        for (int c = 0; c < active; ++c) {
+        int c = 0;
+        for (; c + 4 <= active; c += 4) {                   // four chunks' loads in flight, summed in order
+            float mc[4], oc[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float* pc = part0 + (int64_t)(c + k) * psz;
+                mc[k] = __ldcg(pc + G * D + a);
+                oc[k] = __ldcg(pc + i);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (mc[k] != -INFINITY) acc = fmaf(oc[k], exp2f(mc[k] - Ma), acc);
+        }
+        for (; c < active; ++c) {
             const float* pc = part0 + (int64_t)c * psz;
             const float mc = __ldcg(pc + G * D + a);
-            if (mc != -INFINITY) acc = fmaf(__ldcg(pc + i), exp2f(mc - sm_M[a]), acc);
+            if (mc != -INFINITY) acc = fmaf(__ldcg(pc + i), exp2f(mc - Ma), acc);
         }
         orow[i] = __float2bfloat16_rn(acc * sm_invL[a]);
     }
+    if (tid == 0) {
+        p.arrive[unit] = 0;                                 // the score kernel counts arrivals again
+        if (!keep_logits) {                                 // no score pass follows: finish the bookkeeping here
+            if (!no_append && p.appended[unit] != 0) p.free_slot[u.st] = n;
+            p.appended[unit] = 0;
+        }
+    }
+}
 
+// ---------------------------------------------------------------- steps 3-4: scores and eviction
+// One CTA per chunk again.  Every row's logits become probabilities with the head's final
+// normaliser and are added to its score; rows that may be evicted compete on the 64-bit key
+// (score bits, inverted position): the smallest key is the lowest score and, among equal scores,
+// the latest token.  The CTA that finishes a head last picks the head's victim among the chunks'
+// candidates and updates len / free_slot.
+constexpr int kScoreThreads = 128;
+
+__global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const DecodeParams p) {
+    constexpr int kG = BAKLAVA_MAX_GROUP;
+    __shared__ unsigned long long sm_key[kScoreThreads / 32];
+    __shared__ int sm_slot[kScoreThreads / 32];
+    __shared__ int sm_last;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = p.G;
+    const int4 item = p.items[blockIdx.x];
+    const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
+    const Unit u = decode_unit(p, unit);
+    const int C = p.cap[u.head];
+    const int n = p.len[u.st];
+    const int f = p.free_slot[u.st];
+    if (n < 0 || n > C || f < 0 || f > C) return;         // reported by the attention kernel
+    const bool no_append = (p.flags & BAKLAVA_FLAG_NO_APPEND) != 0;
+    const int hole = (no_append && f < n) ? f : -1;
+    const int n_hi = n + (hole >= 0 ? 1 : 0);
+    const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
+    if (piece >= active) return;
+    const int end = min(begin + chunk_len, n_hi);
+
+    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    const float* logit_h = p.logit + row0 * G;
+    float Mq[kG], iL[kG];
+#pragma unroll
+    for (int a = 0; a < kG; ++a) {
+        Mq[a] = a < G ? p.stats[(int64_t)unit * 2 * kG + a] : 0.0f;
+        iL[a] = a < G ? p.stats[(int64_t)unit * 2 * kG + kG + a] : 0.0f;
+    }
     const bool appended = !no_append && p.appended[unit] != 0;
     const int R = C - 1;
-    const bool evict = appended && keep_logits && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n > R;
+    const bool evict = appended && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n > R;
+    const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
+    const int newest_candidate = p.t_pos - W;              // rows with pos > this are in the recent window
+
     unsigned long long best = ~0ull;
     int best_slot = -1;
-    if (keep_logits) {
-        const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
-        for (int j = tid; j < n_hi; j += kThreads) {
-            if (j == hole) continue;
-            float inc = 0.0f;
-            for (int a = 0; a < G; ++a) inc += exp2f(__ldcg(logit_h + (int64_t)a * C + j) - sm_M[a]) * sm_invL[a];
-            const float sc = p.score[row0 + j] + inc;
-            p.score[row0 + j] = sc;
+    for (int j0 = begin + 4 * tid; j0 < end; j0 += 4 * kScoreThreads) {
+        float inc[4] = {0.f, 0.f, 0.f, 0.f};
+        float sc[4];
+        int ps[4] = {0, 0, 0, 0};
+        if (j0 + 4 <= end) {
+            float4 lg[kG];
+#pragma unroll
+            for (int a = 0; a < kG; ++a)
+                if (a < G) lg[a] = __ldcg(reinterpret_cast<const float4*>(logit_h + (int64_t)a * C + j0));
+            const float4 s4 = *reinterpret_cast<const float4*>(p.score + row0 + j0);
             if (evict) {
-                const int ps = p.pos[row0 + j];
-                if (ps >= p.n_sink && ps <= p.t_pos - W) {
-                    // lowest score goes; among equal scores the latest position goes
+                const int4 p4 = *reinterpret_cast<const int4*>(p.pos + row0 + j0);
+                ps[0] = p4.x; ps[1] = p4.y; ps[2] = p4.z; ps[3] = p4.w;
+            }
+#pragma unroll
+            for (int a = 0; a < kG; ++a)
+                if (a < G) {
+                    inc[0] += exp2f(lg[a].x - Mq[a]) * iL[a];
+                    inc[1] += exp2f(lg[a].y - Mq[a]) * iL[a];
+                    inc[2] += exp2f(lg[a].z - Mq[a]) * iL[a];
+                    inc[3] += exp2f(lg[a].w - Mq[a]) * iL[a];
+                }
+            sc[0] = s4.x + inc[0]; sc[1] = s4.y + inc[1]; sc[2] = s4.z + inc[2]; sc[3] = s4.w + inc[3];
+            const float old[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (j0 + e == hole) sc[e] = old[e];         // the freed slot is not a row
+            *reinterpret_cast<float4*>(p.score + row0 + j0) = make_float4(sc[0], sc[1], sc[2], sc[3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = j0 + e;
+                sc[e] = 0.0f;
+                if (j < end && j != hole) {
+                    for (int a = 0; a < G; ++a)
+                        inc[e] += exp2f(__ldcg(logit_h + (int64_t)a * C + j) - Mq[a]) * iL[a];
+                    sc[e] = p.score[row0 + j] + inc[e];
+                    p.score[row0 + j] = sc[e];
+                    if (evict) ps[e] = p.pos[row0 + j];
+                }
+            }
+        }
+        if (evict) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int j = j0 + e;
+                if (j < end && j != hole && ps[e] >= p.n_sink && ps[e] <= newest_candidate) {
                     const unsigned long long key =
-                        ((unsigned long long)__float_as_uint(sc) << 32) | (uint32_t)(~(uint32_t)ps);
+                        ((unsigned long long)__float_as_uint(sc[e]) << 32) | (uint32_t)(~(uint32_t)ps[e]);
                     if (key < best) { best = key; best_slot = j; }
                 }
             }
@@ -469,15 +572,35 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
             if (ok < best) { best = ok; best_slot = os; }
         }
         if (lane == 0) { sm_key[warp] = best; sm_slot[warp] = best_slot; }
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 0; w < kScoreThreads / 32; ++w)
+                if (sm_key[w] < best) { best = sm_key[w]; best_slot = sm_slot[w]; }
+            p.best_key[blockIdx.x] = best;
+            p.best_slot[blockIdx.x] = best_slot;
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int before = atomicAdd(p.arrive + unit, 1);
+        sm_last = (before == active - 1);
     }
     __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
     if (tid == 0) {
         if (appended) {
             if (evict) {
-                for (int w = 0; w < kThreads / 32; ++w)
-                    if (sm_key[w] < best) { best = sm_key[w]; best_slot = sm_slot[w]; }
-                if (best_slot >= 0) {
-                    p.free_slot[u.st] = best_slot;
+                const int64_t first = (int64_t)blockIdx.x - piece;
+                unsigned long long bk = ~0ull;
+                int bs = -1;
+                for (int c = 0; c < active; ++c) {
+                    const unsigned long long kc = __ldcg(p.best_key + first + c);
+                    if (kc < bk) { bk = kc; bs = __ldcg(p.best_slot + first + c); }
+                }
+                if (bs >= 0) {
+                    p.free_slot[u.st] = bs;
                     p.len[u.st] = n - 1;
                 } else {
                     atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);   // capacity too small for sinks + window
@@ -597,6 +720,9 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     p.appended = reinterpret_cast<int32_t*>(base + lay.appended_off);
     p.partial = reinterpret_cast<float*>(base + lay.partial_off);
     p.logit = reinterpret_cast<float*>(base + lay.logit_off);
+    p.stats = reinterpret_cast<float*>(base + lay.stats_off);
+    p.best_key = reinterpret_cast<unsigned long long*>(base + lay.best_off);
+    p.best_slot = reinterpret_cast<int32_t*>(base + lay.best_off + 8 * (size_t)info->n_items);
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -608,5 +734,10 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
         if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     }
     err = shape->D == 128 ? launch_chunks<128>(p, k_map, v_map, s) : launch_chunks<64>(p, k_map, v_map, s);
-    return err == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
+    if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    if (!(p.flags & BAKLAVA_FLAG_NO_SCORE)) {
+        score_evict_kernel<<<p.n_items, kScoreThreads, 0, s>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    }
+    return BAKLAVA_OK;
 }
