@@ -169,6 +169,7 @@ def main():
     ap.add_argument("--workload", default="llama", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="only the first LAYERS layers (for profiling a small case)")
+    ap.add_argument("--chunk", type=int, default=0, help="force the plan's chunk length (tokens); 0 = automatic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
@@ -190,7 +191,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     bk.lib()                                             # fail now if the library is missing
-    sess = DecodeSession(w, dev)
+    sess = DecodeSession(w, dev, chunk_tokens=args.chunk)
     sess.prefill_synthetic()
     total = args.warmup + args.steps
     feeds = [wl.decode_inputs(w, i, sess.scales, dev) for i in range(2 * total)]
