@@ -272,9 +272,9 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
                          "peak_kind": peak_kind, "kernel": "decode_chunk_kernel",
-                         "note": "events bracket one call = append + attention + score/evict kernels"},
+                         "note": "events bracket one call = attention kernel + score/evict kernel"},
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": 3 * args.steps,
+            "gpu_launches": 2 * args.steps,
             "clocks": clocks.summary(t_open, t_close),
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -11,7 +11,6 @@ constexpr int kTile = 64;   // chunk lengths are multiples of this many tokens
 struct DecodeWorkspace {
     size_t control_off;    // 64 int32: launch-wide counters
     size_t arrive_off;     // int32 [n_units]: chunks of a head that have delivered their partial result
-    size_t appended_off;   // int32 [n_units]: 1 if this step appended a row to the head
     size_t stats_off;      // fp32 [n_units][2 * 8]: final (max, 1 / sum) of each query head, log2 domain
     size_t best_off;       // uint64 + int32 pairs [n_items]: each chunk's eviction candidate
     size_t partial_off;    // fp32 [n_items][g * D + 2 * g]: per-chunk (o, m, l)

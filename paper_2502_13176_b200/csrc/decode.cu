@@ -56,7 +56,6 @@ struct DecodeParams {
     const int4* items;
     int32_t n_items;
     int32_t* arrive;
-    int32_t* appended;
     float* partial;
     float* logit;
     float* stats;                  // [n_units][2 * kG]
@@ -81,40 +80,28 @@ __device__ __forceinline__ Unit decode_unit(const DecodeParams& p, int unit) {
     return u;
 }
 
-// ---------------------------------------------------------------- step 1: append (Eq. 4)
-template <int D>
-__global__ void append_kernel(const DecodeParams p) {
-    const int unit = blockIdx.x;
-    const Unit u = decode_unit(p, unit);
-    const int C = p.cap[u.head];
-    const int n = p.len[u.st];
-    const int f = p.free_slot[u.st];
-    int ok = 1;
-    if (n < 0 || n > C || f < 0 || f > n) {
-        if (threadIdx.x == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
-        ok = 0;
-    } else if (n >= C) {
-        if (threadIdx.x == 0) atomicOr(p.status, BAKLAVA_STATUS_OVERFLOW);
-        ok = 0;
-    }
-    if (ok) {
-        const int64_t row = (int64_t)u.b * p.seq_stride + p.slab_off[u.head] + f;
-        const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
-        constexpr int kVec = D / 8;   // 16-byte pieces per row
-        for (int i = threadIdx.x; i < 2 * kVec; i += blockDim.x) {
-            const bool is_v = i >= kVec;
-            const int c = is_v ? i - kVec : i;
-            const uint4* from = reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c;
-            uint4* to = reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c;
-            *to = *from;
-        }
-        if (threadIdx.x == 0) {
-            p.pos[row] = p.t_pos;
-            p.score[row] = 0.0f;
-            p.len[u.st] = n + 1;
-        }
-    }
-    if (threadIdx.x == 0) p.appended[unit] = ok;
+// What a step does to one head, derived identically by every CTA that touches it.
+struct HeadState {
+    int C, n, f;        // capacity, valid rows and free slot before the step
+    int n_att;          // rows 0 .. n_att-1 are scanned by attention
+    int hole;           // a scanned slot that is not a row (-1: none)
+    bool bad;           // inconsistent state: the head is skipped
+    bool overflow;      // a row was offered but the cache has no free slot
+    bool do_append;     // this step writes the new row at slot f (Eq. 4)
+};
+
+__device__ __forceinline__ HeadState head_state(const DecodeParams& p, const Unit& u) {
+    HeadState h;
+    h.C = p.cap[u.head];
+    h.n = p.len[u.st];
+    h.f = p.free_slot[u.st];
+    const bool no_append = (p.flags & BAKLAVA_FLAG_NO_APPEND) != 0;
+    h.bad = h.n < 0 || h.n > h.C || h.f < 0 || h.f > h.C || (!no_append && h.f > h.n);
+    h.overflow = !no_append && h.n >= h.C;
+    h.do_append = !no_append && !h.overflow && !h.bad;
+    h.hole = (no_append && h.f < h.n) ? h.f : -1;
+    h.n_att = h.n + ((h.do_append || h.hole >= 0) ? 1 : 0);
+    return h;
 }
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -205,16 +192,13 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     const int4 item = p.items[blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
-    const int C = p.cap[u.head];
-    const int n = p.len[u.st];
-    const int f = p.free_slot[u.st];
-    if (n < 0 || n > C || f < 0 || f > C) {
+    const HeadState hs = head_state(p, u);
+    if (hs.bad) {
         if (tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
         return;
     }
-    const bool no_append = (p.flags & BAKLAVA_FLAG_NO_APPEND) != 0;
-    const int hole = (no_append && f < n) ? f : -1;       // a freed slot in the middle of the rows
-    const int n_hi = n + (hole >= 0 ? 1 : 0);             // rows 0 .. n_hi-1 are scanned
+    if (hs.overflow && tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_OVERFLOW);
+    const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
     if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
@@ -295,6 +279,23 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
             const int tok0 = begin + it * kTileTokens + r0;          // first token of this warp's block
             const int valid = min(kWarpTokens, end - tok0);          // rows of the block inside the chunk
             if (valid > 0) {
+                if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + kWarpTokens) {
+                    // step 1 (Eq. 4): the new token's row replaces whatever the tile holds at the free slot,
+                    // in shared memory for this pass and in the slab for the steps to come
+                    constexpr int kVec = D / 8;
+                    const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
+                    const int64_t row = row0 + hs.f;
+                    uint8_t* k_ptr = ring_ptr + s * kStageBytes;
+                    for (int i = lane; i < 2 * kVec; i += 32) {
+                        const bool is_v = i >= kVec;
+                        const int c = is_v ? i - kVec : i;
+                        const uint4 val = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
+                        *reinterpret_cast<uint4*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c)) = val;
+                        *(reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c) = val;
+                    }
+                    if (lane == 0) { p.pos[row] = p.t_pos; p.score[row] = 0.0f; }
+                    __syncwarp();
+                }
                 // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
                 if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
                     uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
@@ -457,9 +458,9 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     }
     if (tid == 0) {
         p.arrive[unit] = 0;                                 // the score kernel counts arrivals again
-        if (!keep_logits) {                                 // no score pass follows: finish the bookkeeping here
-            if (!no_append && p.appended[unit] != 0) p.free_slot[u.st] = n;
-            p.appended[unit] = 0;
+        if (!keep_logits && hs.do_append) {                 // no score pass follows: finish the bookkeeping here
+            p.len[u.st] = n + 1;
+            p.free_slot[u.st] = n + 1;
         }
     }
 }
@@ -483,13 +484,9 @@ __global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const Decode
     const int4 item = p.items[blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
-    const int C = p.cap[u.head];
-    const int n = p.len[u.st];
-    const int f = p.free_slot[u.st];
-    if (n < 0 || n > C || f < 0 || f > C) return;         // reported by the attention kernel
-    const bool no_append = (p.flags & BAKLAVA_FLAG_NO_APPEND) != 0;
-    const int hole = (no_append && f < n) ? f : -1;
-    const int n_hi = n + (hole >= 0 ? 1 : 0);
+    const HeadState hs = head_state(p, u);
+    if (hs.bad) return;                                    // reported by the attention kernel
+    const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
     if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
@@ -502,9 +499,9 @@ __global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const Decode
         Mq[a] = a < G ? p.stats[(int64_t)unit * 2 * kG + a] : 0.0f;
         iL[a] = a < G ? p.stats[(int64_t)unit * 2 * kG + kG + a] : 0.0f;
     }
-    const bool appended = !no_append && p.appended[unit] != 0;
+    const bool appended = hs.do_append;
     const int R = C - 1;
-    const bool evict = appended && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n > R;
+    const bool evict = appended && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n_hi > R;
     const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
     const int newest_candidate = p.t_pos - W;              // rows with pos > this are in the recent window
 
@@ -600,18 +597,18 @@ __global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const Decode
                     if (kc < bk) { bk = kc; bs = __ldcg(p.best_slot + first + c); }
                 }
                 if (bs >= 0) {
-                    p.free_slot[u.st] = bs;
-                    p.len[u.st] = n - 1;
+                    p.free_slot[u.st] = bs;                 // len stays n: one row in, one row out
                 } else {
                     atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);   // capacity too small for sinks + window
-                    p.free_slot[u.st] = n;
+                    p.len[u.st] = n + 1;
+                    p.free_slot[u.st] = n + 1;
                 }
             } else {
-                p.free_slot[u.st] = n;
+                p.len[u.st] = n + 1;
+                p.free_slot[u.st] = n + 1;
             }
         }
         p.arrive[unit] = 0;
-        p.appended[unit] = 0;
     }
 }
 
@@ -717,7 +714,6 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     p.n_items = info->n_items;
     char* base = static_cast<char*>(ws);
     p.arrive = reinterpret_cast<int32_t*>(base + lay.arrive_off);
-    p.appended = reinterpret_cast<int32_t*>(base + lay.appended_off);
     p.partial = reinterpret_cast<float*>(base + lay.partial_off);
     p.logit = reinterpret_cast<float*>(base + lay.logit_off);
     p.stats = reinterpret_cast<float*>(base + lay.stats_off);
@@ -727,12 +723,6 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
-    if (!no_append) {
-        if (shape->D == 128) append_kernel<128><<<info->n_units, 32, 0, s>>>(p);
-        else append_kernel<64><<<info->n_units, 32, 0, s>>>(p);
-        err = cudaGetLastError();
-        if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
-    }
     err = shape->D == 128 ? launch_chunks<128>(p, k_map, v_map, s) : launch_chunks<64>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     if (!(p.flags & BAKLAVA_FLAG_NO_SCORE)) {
