@@ -111,7 +111,9 @@ typedef struct baklava_alloc_params {
 
 /* What baklava_decode_plan decided; passed back to baklava_decode_attn unchanged. */
 typedef struct baklava_plan_info {
-    int32_t n_items;        /* work items (one chunk of one head of one sequence each)              */
+    int32_t n_items;        /* attention work items (one chunk of one head of one sequence each)    */
+    int32_t n_score_items;  /* coarser pieces of the same heads for the score / eviction pass,      */
+                            /*   listed after the attention items                                   */
     int32_t n_units;        /* (layer, sequence, KV head) triples in the layer range                */
     int32_t chunk_tokens;   /* target chunk length the plan used                                    */
     int32_t layer_begin, layer_end, B;
@@ -170,7 +172,7 @@ int baklava_allocate(const baklava_shape* shape, const double* kv_importance,
  *   chunk_tokens  target chunk length, 0 = choose from the total work and n_sm
  *   n_sm          streaming multiprocessors of the device (used when chunk_tokens = 0)
  *   items_out     host int32 [4 * items_capacity] or NULL to only fill `info`
- * The caller copies items_out (info->n_items * 16 bytes) to the device and hands it
+ * The caller copies items_out ((info->n_items + info->n_score_items) * 16 bytes) to the device and hands it
  * to baklava_decode_attn together with `info`. */
 int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t B,
                         int32_t layer_begin, int32_t layer_end, int32_t chunk_tokens, int32_t n_sm,

@@ -13,6 +13,7 @@
 // against V with bf16 mma.sync (fp32 accumulate), and keep an online-softmax state each.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cmath>
@@ -53,14 +54,15 @@ struct DecodeParams {
     float* lse;
     int32_t t_pos;
     uint32_t flags;
-    const int4* items;
+    const int4* items;             // attention items, then score items
     int32_t n_items;
+    int32_t n_score_items;
     int32_t* arrive;
     float* partial;
     float* logit;
     float* stats;                  // [n_units][2 * kG]
-    unsigned long long* best_key;  // [n_items]
-    int32_t* best_slot;            // [n_items]
+    unsigned long long* best_key;  // [n_score_items]
+    int32_t* best_slot;            // [n_score_items]
     float scale_log2;   // log2(e) / sqrt(D)
 };
 
@@ -132,10 +134,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+// K and V are read once per step and never fit in L2: ask L2 to drop them first, so that the
+// step's logits, scores and positions (which the score pass re-reads) stay resident.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                            uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -206,7 +217,10 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
 
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
-    float* logit_h = p.logit + row0 * G;                  // [G][C] for this head
+    // this head's share of the scratch: unnormalised probabilities [G][C] in fp16, each relative to the
+    // running maximum its 16-token block was computed under, and those maxima [G][C / 16] in fp32
+    __half* prob_h = reinterpret_cast<__half*>(p.logit + row0 * G);
+    float* mref_h = reinterpret_cast<float*>(prob_h + (int64_t)G * C);
 
     // 1024-byte aligned stage ring inside the dynamic shared memory
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -232,6 +246,7 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     if (warp == kConsumerWarps) {
         // ---------------- producer: one lane issues the TMA loads
         if (lane == 0) {
+            const uint64_t stream_policy = l2_evict_first_policy();
             for (int it = 0; it < n_tiles; ++it) {
                 const int s = it % kStages;
                 if (it >= kStages) {
@@ -247,8 +262,8 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
                 mbar_arrive_expect_tx(full, kStageBytes);
 #pragma unroll
                 for (int bx = 0; bx < D / 64; ++bx) {
-                    tma_load_2d(dst + bx * (kTileTokens * 128), &k_map, bx * 64, y, full);
-                    tma_load_2d(dst + kTileBytes + bx * (kTileTokens * 128), &v_map, bx * 64, y, full);
+                    tma_load_2d(dst + bx * (kTileTokens * 128), &k_map, bx * 64, y, full, stream_policy);
+                    tma_load_2d(dst + kTileBytes + bx * (kTileTokens * 128), &v_map, bx * 64, y, full, stream_policy);
                 }
             }
         }
@@ -326,15 +341,6 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
                         sv[2 * t + e] = sacc[t][e] * p.scale_log2;
                         ok[2 * t + e] = tok < end && tok != hole;
                     }
-                if (keep_logits && qrow < G) {
-#pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        const int tok = tok0 + 8 * t + qcol;
-                        float* dst = logit_h + (int64_t)qrow * C + tok;
-                        if (tok + 1 < end) *reinterpret_cast<float2*>(dst) = make_float2(sv[2 * t], sv[2 * t + 1]);
-                        else if (tok < end) dst[0] = sv[2 * t];
-                    }
-                }
                 float mx = -INFINITY;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) mx = fmaxf(mx, ok[i] ? sv[i] : -INFINITY);
@@ -347,6 +353,16 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
                 for (int i = 0; i < 4; ++i) pv[i] = ok[i] ? exp2f(sv[i] - m_new) : 0.0f;
                 l_run = l_run * corr + (pv[0] + pv[1]) + (pv[2] + pv[3]);
                 m_run = m_new;
+                if (keep_logits && qrow < G) {
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        const int tok = tok0 + 8 * t + qcol;
+                        __half* dst = prob_h + (int64_t)qrow * C + tok;
+                        if (tok + 1 < end) *reinterpret_cast<__half2*>(dst) = __floats2half2_rn(pv[2 * t], pv[2 * t + 1]);
+                        else if (tok < end) dst[0] = __float2half_rn(pv[2 * t]);
+                    }
+                    if ((lane & 3) == 0) mref_h[qrow * (C >> 4) + (tok0 >> 4)] = m_new;
+                }
                 if (__any_sync(0xffffffffu, corr != 1.0f)) {
 #pragma unroll
                     for (int j = 0; j < kNTiles; ++j) { o[j][0] *= corr; o[j][1] *= corr; }
@@ -471,17 +487,17 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
 // (score bits, inverted position): the smallest key is the lowest score and, among equal scores,
 // the latest token.  The CTA that finishes a head last picks the head's victim among the chunks'
 // candidates and updates len / free_slot.
-constexpr int kScoreThreads = 128;
+constexpr int kScoreThreads = 128;                       // eight rows per thread and sweep
 
-__global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const DecodeParams p) {
+template <int G>
+__global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const DecodeParams p) {
     constexpr int kG = BAKLAVA_MAX_GROUP;
     __shared__ unsigned long long sm_key[kScoreThreads / 32];
     __shared__ int sm_slot[kScoreThreads / 32];
     __shared__ int sm_last;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = p.G;
-    const int4 item = p.items[blockIdx.x];
+    const int4 item = p.items[p.n_items + blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
     const HeadState hs = head_state(p, u);
@@ -492,12 +508,13 @@ __global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const Decode
     const int end = min(begin + chunk_len, n_hi);
 
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
-    const float* logit_h = p.logit + row0 * G;
-    float Mq[kG], iL[kG];
+    const __half* prob_h = reinterpret_cast<const __half*>(p.logit + row0 * G);
+    const float* mref_h = reinterpret_cast<const float*>(prob_h + (int64_t)G * C);
+    float Mq[G], iL[G];
 #pragma unroll
-    for (int a = 0; a < kG; ++a) {
-        Mq[a] = a < G ? p.stats[(int64_t)unit * 2 * kG + a] : 0.0f;
-        iL[a] = a < G ? p.stats[(int64_t)unit * 2 * kG + kG + a] : 0.0f;
+    for (int a = 0; a < G; ++a) {
+        Mq[a] = p.stats[(int64_t)unit * 2 * kG + a];
+        iL[a] = p.stats[(int64_t)unit * 2 * kG + kG + a];
     }
     const bool appended = hs.do_append;
     const int R = C - 1;
@@ -507,42 +524,55 @@ __global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const Decode
 
     unsigned long long best = ~0ull;
     int best_slot = -1;
-    for (int j0 = begin + 4 * tid; j0 < end; j0 += 4 * kScoreThreads) {
-        float inc[4] = {0.f, 0.f, 0.f, 0.f};
-        float sc[4];
-        int ps[4] = {0, 0, 0, 0};
-        if (j0 + 4 <= end) {
-            float4 lg[kG];
+    // eight consecutive rows per thread: they share one 16-row block, hence one reference maximum per head
+    for (int j0 = begin + 8 * tid; j0 < end; j0 += 8 * kScoreThreads) {
+        float fac[G];
 #pragma unroll
-            for (int a = 0; a < kG; ++a)
-                if (a < G) lg[a] = __ldcg(reinterpret_cast<const float4*>(logit_h + (int64_t)a * C + j0));
-            const float4 s4 = *reinterpret_cast<const float4*>(p.score + row0 + j0);
+        for (int a = 0; a < G; ++a) {
+            const float mr = __ldcg(mref_h + a * (C >> 4) + (j0 >> 4));
+            fac[a] = (mr == -INFINITY) ? 0.0f : exp2f(mr - Mq[a]) * iL[a];
+        }
+        float inc[8], sc[8];
+        int ps[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { inc[e] = 0.0f; ps[e] = 0; }
+        if (j0 + 8 <= end) {
+            uint4 pr[G];
+#pragma unroll
+            for (int a = 0; a < G; ++a)
+                pr[a] = __ldcg(reinterpret_cast<const uint4*>(prob_h + (int64_t)a * C + j0));
+            const float4 s0 = *reinterpret_cast<const float4*>(p.score + row0 + j0);
+            const float4 s1 = *reinterpret_cast<const float4*>(p.score + row0 + j0 + 4);
             if (evict) {
-                const int4 p4 = *reinterpret_cast<const int4*>(p.pos + row0 + j0);
-                ps[0] = p4.x; ps[1] = p4.y; ps[2] = p4.z; ps[3] = p4.w;
+                const int4 p0 = *reinterpret_cast<const int4*>(p.pos + row0 + j0);
+                const int4 p1 = *reinterpret_cast<const int4*>(p.pos + row0 + j0 + 4);
+                ps[0] = p0.x; ps[1] = p0.y; ps[2] = p0.z; ps[3] = p0.w;
+                ps[4] = p1.x; ps[5] = p1.y; ps[6] = p1.z; ps[7] = p1.w;
             }
 #pragma unroll
-            for (int a = 0; a < kG; ++a)
-                if (a < G) {
-                    inc[0] += exp2f(lg[a].x - Mq[a]) * iL[a];
-                    inc[1] += exp2f(lg[a].y - Mq[a]) * iL[a];
-                    inc[2] += exp2f(lg[a].z - Mq[a]) * iL[a];
-                    inc[3] += exp2f(lg[a].w - Mq[a]) * iL[a];
-                }
-            sc[0] = s4.x + inc[0]; sc[1] = s4.y + inc[1]; sc[2] = s4.z + inc[2]; sc[3] = s4.w + inc[3];
-            const float old[4] = {s4.x, s4.y, s4.z, s4.w};
+            for (int a = 0; a < G; ++a) {
+                const uint32_t w[4] = {pr[a].x, pr[a].y, pr[a].z, pr[a].w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (j0 + e == hole) sc[e] = old[e];         // the freed slot is not a row
+                for (int k = 0; k < 4; ++k) {
+                    const float2 pe = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
+                    inc[2 * k] = fmaf(pe.x, fac[a], inc[2 * k]);
+                    inc[2 * k + 1] = fmaf(pe.y, fac[a], inc[2 * k + 1]);
+                }
+            }
+            const float old[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sc[e] = (j0 + e == hole) ? old[e] : old[e] + inc[e];   // the freed slot is not a row
             *reinterpret_cast<float4*>(p.score + row0 + j0) = make_float4(sc[0], sc[1], sc[2], sc[3]);
+            *reinterpret_cast<float4*>(p.score + row0 + j0 + 4) = make_float4(sc[4], sc[5], sc[6], sc[7]);
         } else {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
+            for (int e = 0; e < 8; ++e) {
                 const int j = j0 + e;
                 sc[e] = 0.0f;
                 if (j < end && j != hole) {
+#pragma unroll
                     for (int a = 0; a < G; ++a)
-                        inc[e] += exp2f(__ldcg(logit_h + (int64_t)a * C + j) - Mq[a]) * iL[a];
+                        inc[e] = fmaf(__half2float(__ldcg(prob_h + (int64_t)a * C + j)), fac[a], inc[e]);
                     sc[e] = p.score[row0 + j] + inc[e];
                     p.score[row0 + j] = sc[e];
                     if (evict) ps[e] = p.pos[row0 + j];
@@ -551,7 +581,7 @@ __global__ void __launch_bounds__(kScoreThreads) score_evict_kernel(const Decode
         }
         if (evict) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
+            for (int e = 0; e < 8; ++e) {
                 const int j = j0 + e;
                 if (j < end && j != hole && ps[e] >= p.n_sink && ps[e] <= newest_candidate) {
                     const unsigned long long key =
@@ -673,13 +703,13 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     for (const void* ptr : ptrs)
         if (ptr && !baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
     if (info->layer_begin < 0 || info->layer_end > shape->L || info->layer_begin >= info->layer_end ||
-        info->B != cache->B || info->n_items <= 0 ||
+        info->B != cache->B || info->n_items <= 0 || info->n_score_items <= 0 ||
         info->n_units != (info->layer_end - info->layer_begin) * cache->B * shape->Hkv)
         return BAKLAVA_ERR_INVALID_ARG;
     const int64_t rows = (int64_t)cache->B * cache->seq_stride_tokens;
     if (rows > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     DecodeWorkspace lay;
-    const size_t need = baklava_decode_ws_bytes(shape, info->n_items, info->n_units, cache->B,
+    const size_t need = baklava_decode_ws_bytes(shape, info->n_items, info->n_score_items, info->n_units, cache->B,
                                                 cache->seq_stride_tokens, &lay);
     if (ws_bytes < need) return BAKLAVA_ERR_WORKSPACE;
 
@@ -712,13 +742,14 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     p.flags = (flags & BAKLAVA_FLAG_NO_SCORE) ? (flags | BAKLAVA_FLAG_NO_EVICT) : flags;
     p.items = reinterpret_cast<const int4*>(items);
     p.n_items = info->n_items;
+    p.n_score_items = info->n_score_items;
     char* base = static_cast<char*>(ws);
     p.arrive = reinterpret_cast<int32_t*>(base + lay.arrive_off);
     p.partial = reinterpret_cast<float*>(base + lay.partial_off);
     p.logit = reinterpret_cast<float*>(base + lay.logit_off);
     p.stats = reinterpret_cast<float*>(base + lay.stats_off);
     p.best_key = reinterpret_cast<unsigned long long*>(base + lay.best_off);
-    p.best_slot = reinterpret_cast<int32_t*>(base + lay.best_off + 8 * (size_t)info->n_items);
+    p.best_slot = reinterpret_cast<int32_t*>(base + lay.best_off + 8 * (size_t)info->n_score_items);
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -726,7 +757,16 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     err = shape->D == 128 ? launch_chunks<128>(p, k_map, v_map, s) : launch_chunks<64>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     if (!(p.flags & BAKLAVA_FLAG_NO_SCORE)) {
-        score_evict_kernel<<<p.n_items, kScoreThreads, 0, s>>>(p);
+        switch (p.G) {
+            case 1: score_evict_kernel<1><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            case 2: score_evict_kernel<2><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            case 3: score_evict_kernel<3><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            case 4: score_evict_kernel<4><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            case 5: score_evict_kernel<5><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            case 6: score_evict_kernel<6><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            case 7: score_evict_kernel<7><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            default: score_evict_kernel<8><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+        }
         if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
     }
     return BAKLAVA_OK;

@@ -160,7 +160,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_allocate(const bak
 }
 
 // ---------------------------------------------------------------- decode work plan
-size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_units, int32_t B,
+size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_score_items, int64_t n_units, int32_t B,
                                int64_t seq_stride_tokens, DecodeWorkspace* lay) {
     const int g = s->Hq / s->Hkv;
     DecodeWorkspace w;
@@ -169,7 +169,7 @@ size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t 
     w.control_off = take(sizeof(int32_t) * 64);
     w.arrive_off = take(sizeof(int32_t) * (size_t)n_units);
     w.stats_off = take(sizeof(float) * (size_t)n_units * 2 * BAKLAVA_MAX_GROUP);
-    w.best_off = take(16 * (size_t)n_items);
+    w.best_off = take(16 * (size_t)n_score_items);
     w.partial_off = take(sizeof(float) * (size_t)n_items * g * (s->D + 2));
     w.logit_off = take(sizeof(float) * (size_t)B * (size_t)seq_stride_tokens * g);
     w.total = off;
@@ -209,34 +209,46 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
     }
     target = std::max<int64_t>(kTile, (target + kTile - 1) / kTile * kTile);
 
-    int64_t n_items = 0;
-    for (int i : heads) {
-        const int64_t c = cap[(size_t)layer_begin * Hkv + i];
-        int64_t pieces = (c + target - 1) / target;
-        const int64_t len = ((c + pieces - 1) / pieces + kTile - 1) / kTile * kTile;
-        pieces = (c + len - 1) / len;
-        if (pieces > 32767) return BAKLAVA_ERR_UNSUPPORTED;
-        const int li = i / Hkv, h = i % Hkv;
-        for (int b = 0; b < B; ++b) {
-            const int64_t unit = ((int64_t)li * B + b) * Hkv + h;
-            for (int64_t pc = 0; pc < pieces; ++pc, ++n_items) {
-                if (!items_out) continue;
-                if (n_items >= items_capacity) return BAKLAVA_ERR_WORKSPACE;
-                int32_t* it = items_out + 4 * n_items;
-                it[0] = (int32_t)unit;
-                it[1] = (int32_t)(pc * len);
-                it[2] = (int32_t)len;
-                it[3] = (int32_t)(pc | (pieces << 16));
+    // cut every head into equal pieces of about `want` tokens and list them, head after head
+    int64_t n_written = 0;
+    auto emit = [&](int64_t want, int64_t* count) -> int {
+        *count = 0;
+        for (int i : heads) {
+            const int64_t c = cap[(size_t)layer_begin * Hkv + i];
+            int64_t pieces = (c + want - 1) / want;
+            const int64_t len = ((c + pieces - 1) / pieces + kTile - 1) / kTile * kTile;
+            pieces = (c + len - 1) / len;
+            if (pieces > 32767) return BAKLAVA_ERR_UNSUPPORTED;
+            const int li = i / Hkv, h = i % Hkv;
+            for (int b = 0; b < B; ++b) {
+                const int64_t unit = ((int64_t)li * B + b) * Hkv + h;
+                for (int64_t pc = 0; pc < pieces; ++pc, ++*count, ++n_written) {
+                    if (!items_out) continue;
+                    if (n_written >= items_capacity) return BAKLAVA_ERR_WORKSPACE;
+                    int32_t* it = items_out + 4 * n_written;
+                    it[0] = (int32_t)unit;
+                    it[1] = (int32_t)(pc * len);
+                    it[2] = (int32_t)len;
+                    it[3] = (int32_t)(pc | (pieces << 16));
+                }
             }
         }
-    }
+        return BAKLAVA_OK;
+    };
+    int64_t n_items = 0, n_score = 0;
+    rc = emit(target, &n_items);                 // attention chunks
+    if (rc) return rc;
+    rc = emit(kScoreChunk, &n_score);            // coarser pieces for the score / eviction pass
+    if (rc) return rc;
+    if (n_score > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     if (n_items > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     info->n_items = (int32_t)n_items;
+    info->n_score_items = (int32_t)n_score;
     info->n_units = layers * B * Hkv;
     info->chunk_tokens = (int32_t)target;
     info->layer_begin = layer_begin;
     info->layer_end = layer_end;
     info->B = B;
-    info->ws_bytes = (int64_t)baklava_decode_ws_bytes(shape, n_items, info->n_units, B, seq_stride_tokens, nullptr);
+    info->ws_bytes = (int64_t)baklava_decode_ws_bytes(shape, n_items, n_score, info->n_units, B, seq_stride_tokens, nullptr);
     return BAKLAVA_OK;
 }

@@ -92,24 +92,30 @@ def test_decode_plan_covers_every_head_once():
         chunk = int(rng.choice([0, 64, 100, 512, 4096]))
         plan = bk.baklava_decode_plan(shape, cap, B, lb, le, int(cap.sum()), chunk_tokens=chunk, n_sm=148)
         it, info = plan.items, plan.info
-        assert info.n_units == (le - lb) * B * Hkv and info.n_items == len(it) and info.ws_bytes > 0
-        seen = {}
-        prev_cap = None
-        for row, (unit, begin, clen, packed) in enumerate(it):
-            piece, pieces = packed & 0xffff, packed >> 16
-            li, rem = divmod(unit, B * Hkv); b, h = divmod(rem, Hkv)
-            c = int(cap[lb + li, h])
-            assert clen % 64 == 0 and begin == piece * clen and begin < c and pieces * clen >= c
-            assert (pieces - 1) * clen < c
-            seen.setdefault(unit, []).append(piece)
-            if piece == 0:
-                assert prev_cap is None or c <= prev_cap       # largest heads first
-                prev_cap = c
-            else:
-                assert it[row - 1][0] == unit and (it[row - 1][3] & 0xffff) == piece - 1   # a head's chunks are adjacent
-        assert sorted(seen) == list(range(info.n_units))
-        for unit, pcs in seen.items():
-            assert pcs == list(range(len(pcs)))
+        assert info.n_units == (le - lb) * B * Hkv and info.ws_bytes > 0
+        assert info.n_items + info.n_score_items == len(it) and info.n_score_items >= info.n_units
+        _check_cover(it[:info.n_items], info, cap, lb, B, Hkv)
+        _check_cover(it[info.n_items:], info, cap, lb, B, Hkv)
+
+
+def _check_cover(it, info, cap, lb, B, Hkv):
+    seen = {}
+    prev_cap = None
+    for row, (unit, begin, clen, packed) in enumerate(it):
+        piece, pieces = packed & 0xffff, packed >> 16
+        li, rem = divmod(unit, B * Hkv); b, h = divmod(rem, Hkv)
+        c = int(cap[lb + li, h])
+        assert clen % 64 == 0 and begin == piece * clen and begin < c and pieces * clen >= c
+        assert (pieces - 1) * clen < c
+        seen.setdefault(unit, []).append(piece)
+        if piece == 0:
+            assert prev_cap is None or c <= prev_cap       # largest heads first
+            prev_cap = c
+        else:
+            assert it[row - 1][0] == unit and (it[row - 1][3] & 0xffff) == piece - 1   # a head's chunks are adjacent
+    assert sorted(seen) == list(range(info.n_units))
+    for unit, pcs in seen.items():
+        assert pcs == list(range(len(pcs)))
 
 
 def test_argument_errors_are_codes_not_crashes():
