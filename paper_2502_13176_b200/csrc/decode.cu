@@ -107,6 +107,12 @@ __device__ __forceinline__ HeadState head_state(const DecodeParams& p, const Uni
 }
 
 // ---------------------------------------------------------------- PTX wrappers
+// Programmatic dependent launch: both kernels of a step are launched with the stream-serialisation
+// attribute.  launch_dependents lets the next kernel's CTAs become resident while this grid drains;
+// grid_dependency_wait returns once the previous grid has completed and its writes are visible.
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* ptr) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
 }
@@ -203,6 +209,8 @@ __global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodePara
     const int4 item = p.items[blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
+    launch_dependents();
+    grid_dependency_wait();                               // len / free_slot / slab rows come from earlier kernels
     const HeadState hs = head_state(p, u);
     if (hs.bad) {
         if (tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
@@ -500,6 +508,8 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
     const int4 item = p.items[p.n_items + blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
+    launch_dependents();
+    grid_dependency_wait();                               // the attention kernel's scratch and statistics
     const HeadState hs = head_state(p, u);
     if (hs.bad) return;                                    // reported by the attention kernel
     const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
@@ -678,8 +688,17 @@ cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CU
     constexpr int kSmem = kStages * 2 * kTileTokens * D * 2 + 1024;
     cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    decode_chunk_kernel<D><<<p.n_items, kThreads, kSmem, s>>>(p, km, vm);
-    return cudaGetLastError();
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.n_items);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_chunk_kernel<D>, p, km, vm);
 }
 
 }  // namespace
@@ -757,16 +776,27 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     err = shape->D == 128 ? launch_chunks<128>(p, k_map, v_map, s) : launch_chunks<64>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     if (!(p.flags & BAKLAVA_FLAG_NO_SCORE)) {
+        void (*score_fn)(const DecodeParams) = nullptr;
         switch (p.G) {
-            case 1: score_evict_kernel<1><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
-            case 2: score_evict_kernel<2><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
-            case 3: score_evict_kernel<3><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
-            case 4: score_evict_kernel<4><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
-            case 5: score_evict_kernel<5><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
-            case 6: score_evict_kernel<6><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
-            case 7: score_evict_kernel<7><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
-            default: score_evict_kernel<8><<<p.n_score_items, kScoreThreads, 0, s>>>(p); break;
+            case 1: score_fn = score_evict_kernel<1>; break;
+            case 2: score_fn = score_evict_kernel<2>; break;
+            case 3: score_fn = score_evict_kernel<3>; break;
+            case 4: score_fn = score_evict_kernel<4>; break;
+            case 5: score_fn = score_evict_kernel<5>; break;
+            case 6: score_fn = score_evict_kernel<6>; break;
+            case 7: score_fn = score_evict_kernel<7>; break;
+            default: score_fn = score_evict_kernel<8>; break;
         }
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)p.n_score_items);
+        cfg.blockDim = dim3(kScoreThreads);
+        cfg.stream = s;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, score_fn, p) != cudaSuccess) return BAKLAVA_ERR_CUDA;
         if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
     }
     return BAKLAVA_OK;
