@@ -90,6 +90,20 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(rows)}
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_rate(world, units_per_rank_step, steps, elapsed_ms):
+    """Aggregate throughput of `world` independent replicas: all units processed / slowest rank's time."""
+    return world * units_per_rank_step * steps / (elapsed_ms * 1e-3)
+
+
 def oracle_sample(w, seconds_target=15.0):
     """Time the CPU oracle's decode step on sampled heads of the workload.  Returns a cpu_baseline dict."""
     from concurrent.futures import ThreadPoolExecutor
@@ -245,15 +259,12 @@ def main():
     e2e_ms = e0.elapsed_time(e1)
     sess.check_status()
 
-    times = torch.tensor([elapsed_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
-    elapsed_ms, e2e_ms = times.tolist()
+    elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e_ms], dev)
 
     if rank == 0:
         bytes_per_step = rows_per_step * w.D * 2 * 2          # K and V rows, bf16
-        gbs = world * bytes_per_step * args.steps / (elapsed_ms * 1e-3) / 1e9
-        e2e_gbs = world * bytes_per_step * args.steps / (e2e_ms * 1e-3) / 1e9
+        gbs = whole_job_rate(world, bytes_per_step, args.steps, elapsed_ms) / 1e9
+        e2e_gbs = whole_job_rate(world, bytes_per_step, args.steps, e2e_ms) / 1e9
         peak, peak_kind = measured_peaks()
         kernel_ms = elapsed_ms / args.steps               # one step = the two kernels of one call, back to back
         achieved = bytes_per_step / (kernel_ms * 1e-3) / 1e9
@@ -265,7 +276,7 @@ def main():
                        "kv_bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (no flush)",
                        "launch": "one baklava_decode_attn call per step covering all layers",
                        "replicas": world},
-            "tokens_per_s": world * w.B * args.steps / (elapsed_ms * 1e-3),
+            "tokens_per_s": whole_job_rate(world, w.B, args.steps, elapsed_ms),
             "pct_of_hbm_peak": 100.0 * gbs / world / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
