@@ -6,6 +6,8 @@
 #include "baklava.h"
 
 constexpr int kTile = 64;          // chunk lengths are multiples of this many tokens
+constexpr int kCtasPerSm = 3;       // resident CTAs of the attention kernel per SM (its launch bounds)
+constexpr int kMinChunk = 256;      // shortest chunk the automatic plan makes
 constexpr int kScoreChunk = 4096;  // target length of a piece of the score / eviction pass
 
 // Byte offsets of the regions of the decode workspace.

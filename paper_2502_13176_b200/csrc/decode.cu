@@ -28,7 +28,7 @@ constexpr int kConsumerWarps = 4;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;     // + one producer warp
 constexpr int kTileTokens = kTile;                      // 64 tokens per stage
 constexpr int kWarpTokens = kTileTokens / kConsumerWarps;
-constexpr int kStages = 3;
+constexpr int kStages = 2;                              // 64 KB per CTA, three CTAs per SM
 constexpr uint32_t kWaitLimit = 1u << 22;               // bounded mbarrier waits
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -185,7 +185,7 @@ __device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
 
 // ---------------------------------------------------------------- steps 2-4
 template <int D>
-__global__ void __launch_bounds__(kThreads) decode_chunk_kernel(const DecodeParams p,
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(const DecodeParams p,
                                                                 const __grid_constant__ CUtensorMap k_map,
                                                                 const __grid_constant__ CUtensorMap v_map) {
     constexpr int kKSteps = D / 16;                    // MMA k-steps over the head dimension

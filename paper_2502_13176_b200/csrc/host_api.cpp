@@ -201,20 +201,33 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
         return cap[(size_t)layer_begin * Hkv + a] > cap[(size_t)layer_begin * Hkv + b];
     });
 
+    // Chunk length.  A fixed request is used as given.  Otherwise the launch is self-balancing: CTAs are
+    // dispatched in item order, so the list starts with long chunks (about half of a CTA slot's share of
+    // the tokens: little per-chunk overhead) and ends with short ones (a short tail).
+    const bool guided = chunk_tokens == 0;
     int64_t target = chunk_tokens;
-    if (target == 0) {
-        // aim at about 16 items per SM so that the tail of the launch is short
-        target = (tokens / ((int64_t)n_sm * 16) + kTile - 1) / kTile * kTile;
-        target = std::max<int64_t>(256, std::min<int64_t>(target, 8192));
+    if (guided) {
+        const int64_t slots = (int64_t)n_sm * kCtasPerSm;
+        target = (tokens / (2 * slots) + kTile - 1) / kTile * kTile;
+        target = std::max<int64_t>(kMinChunk, std::min<int64_t>(target, 4096));
     }
     target = std::max<int64_t>(kTile, (target + kTile - 1) / kTile * kTile);
 
     // cut every head into equal pieces of about `want` tokens and list them, head after head
     int64_t n_written = 0;
-    auto emit = [&](int64_t want, int64_t* count) -> int {
+    auto emit = [&](int64_t base, bool shrink, int64_t* count) -> int {
         *count = 0;
+        int64_t done = 0;                                  // tokens listed so far
         for (int i : heads) {
             const int64_t c = cap[(size_t)layer_begin * Hkv + i];
+            int64_t want = base;
+            if (shrink) {
+                if (done * 20 >= tokens * 19) want = base / 8;          // last 5 % of the tokens
+                else if (done * 5 >= tokens * 4) want = base / 4;       // 80 % .. 95 %
+                else if (done * 2 >= tokens) want = base / 2;           // 50 % .. 80 %
+                want = std::max<int64_t>(kMinChunk, want);
+            }
+            done += c * B;
             int64_t pieces = (c + want - 1) / want;
             const int64_t len = ((c + pieces - 1) / pieces + kTile - 1) / kTile * kTile;
             pieces = (c + len - 1) / len;
@@ -236,9 +249,9 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
         return BAKLAVA_OK;
     };
     int64_t n_items = 0, n_score = 0;
-    rc = emit(target, &n_items);                 // attention chunks
+    rc = emit(target, guided, &n_items);         // attention chunks
     if (rc) return rc;
-    rc = emit(kScoreChunk, &n_score);            // coarser pieces for the score / eviction pass
+    rc = emit(kScoreChunk, false, &n_score);     // coarser pieces for the score / eviction pass
     if (rc) return rc;
     if (n_score > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     if (n_items > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
