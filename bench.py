@@ -175,17 +175,67 @@ def run_reference(args, w):
         "e2e": {"value": v, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def run_profile_pass(args):
+    """The one-time profiling pass (Algorithm 1 step 1) on the LLaMA-3-8B attention shape: one step = one
+    layer's heads for all prompts.  Reported against the tensor roofline; not the headline benchmark."""
+    from paper_2502_13176_b200 import binding as bk
+    from paper_2502_13176_b200.engine import shape_of
+
+    w = wl.LLAMA3_8B_32K
+    P, T = args.prompts, args.prompt_tokens
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    shape = shape_of(w)
+    parts = [wl.profile_inputs(w, p, 0, T, dev) for p in range(P)]
+    q = torch.stack([x[0] for x in parts]); k = torch.stack([x[1] for x in parts]); v = torch.stack([x[2] for x in parts])
+    del parts
+    head_cos = torch.empty((P, w.Hq), dtype=torch.float32, device=dev)
+    ws = torch.empty((bk.baklava_profile_workspace_size(shape, P, T),), dtype=torch.uint8, device=dev)
+    for _ in range(args.warmup):
+        bk.baklava_profile_heads(shape, q, k, v, None, P, T, head_cos, None, ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    with ClockSampler(dev.index) as clocks:
+        t_open = time.perf_counter()
+        e0.record()
+        for _ in range(args.steps):
+            bk.baklava_profile_heads(shape, q, k, v, None, P, T, head_cos, None, ws)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        t_close = time.perf_counter()
+    ms = e0.elapsed_time(e1) / args.steps
+    flop = P * w.Hq * 2.0 * T * T * w.D          # QK^T and PV under the causal mask: 2 * (T^2 / 2) * D * 2 each
+    peak = 1653.9
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            peak = float(json.load(f)["bf16_tflops"])
+    tf = flop / (ms * 1e-3) / 1e12
+    print(json.dumps({"metric": "profiling-pass TFLOP/s (causal attention + cosine, one layer)", "value": tf,
+                      "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "profile-llama3-8b", "prompts": P, "prompt_tokens": T, "heads": w.Hq,
+                                 "kv_heads": w.Hkv, "head_dim": w.D},
+                      "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s",
+                                   "frac": tf / peak, "traffic": None, "kernel": "profile_kernel (mma.sync path)"},
+                      "gpu_launches": 2 * args.steps, "clocks": clocks.summary(t_open, t_close)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=8)
-    ap.add_argument("--workload", default="llama", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="llama", choices=sorted(WORKLOADS) + ["profile"])
+    ap.add_argument("--prompts", type=int, default=64, help="profile workload: prompts per step")
+    ap.add_argument("--prompt-tokens", type=int, default=4096, help="profile workload: tokens per prompt")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="only the first LAYERS layers (for profiling a small case)")
     ap.add_argument("--chunk", type=int, default=0, help="force the plan's chunk length (tokens); 0 = automatic")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.workload == "profile":
+        return run_profile_pass(args)
     w = WORKLOADS[args.workload]
     if args.layers:
         w = wl.scaled(w, L=args.layers)
