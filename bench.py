@@ -27,9 +27,9 @@ from paper_2502_13176_b200 import workloads as wl  # noqa: E402
 
 METRIC = "decode-step retained-KV GB/s"
 WORKLOADS = {"llama": wl.LLAMA3_8B_32K, "qwen": wl.QWEN25_7B_8K_B16, "tiny": wl.TINY}
-# dram bytes (read + write) per launch of the dominant kernel from the committed ncu capture, scaled
-# to this workload; None until a capture of the current kernel exists (see profiles/).
-NCU_TRAFFIC_BYTES = {"llama3-8b-32k-30pct": 1316800000}   # profiles/decode_chunk_kernel_llama3-8b-32k.md
+# dram bytes (read + write) per launch of the attention kernel from the committed ncu capture under
+# profiles/ (taken on 8 layers and scaled by rows); a workload without a current capture reports null.
+NCU_TRAFFIC_BYTES = {"llama3-8b-32k-30pct": 1316800000}
 
 
 def measured_peaks():
