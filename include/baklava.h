@@ -51,7 +51,10 @@ extern "C" {
 
 /* flags of baklava_decode_attn */
 #define BAKLAVA_FLAG_NO_APPEND     1u   /* attend over the cache as it is; k_new / v_new ignored      */
-#define BAKLAVA_FLAG_NO_SCORE      2u   /* do not accumulate attention into `score` (implies NO_EVICT) */
+#define BAKLAVA_FLAG_NO_SCORE      2u   /* do not accumulate attention into `score`.  Implies NO_EVICT,  */
+                                        /*   except under the pure sinks + window policy (recent_num ==   */
+                                        /*   recent_den), where the oldest row outside both is evicted:  */
+                                        /*   the paper's evaluated policy, with no score traffic at all  */
 #define BAKLAVA_FLAG_NO_EVICT      4u   /* never evict; a cache that fills up stays full              */
 
 #define BAKLAVA_SCOPE_LAYER        0    /* Algorithm 2 inside each layer                              */

@@ -16,7 +16,7 @@ struct DecodeWorkspace {
     size_t arrive_off;     // int32 [n_units]: chunks of a head that have delivered their partial result
     size_t stats_off;      // fp32 [n_units][2 * 8]: final (max, 1 / sum) of each query head, log2 domain
     size_t best_off;       // uint64 [n_score_items] + int32 [n_score_items]: each score piece's eviction candidate
-    size_t partial_off;    // fp32 [n_items][g * D + 2 * g]: per-chunk (o, m, l)
+    size_t partial_off;    // fp32 [n_items][g * D + 2 * g + 2]: per-chunk (o, m, l) and its oldest evictable row (pos, slot)
     size_t logit_off;      // fp32 [B * seq_stride_tokens][g]: log2-domain logits of this step
     size_t total;
 };

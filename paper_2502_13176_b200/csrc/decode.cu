@@ -16,6 +16,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <climits>
 #include <cmath>
 #include <cstdint>
 
@@ -54,6 +55,7 @@ struct DecodeParams {
     float* lse;
     int32_t t_pos;
     uint32_t flags;
+    int32_t window_evict;          // 1: no scores are kept and the policy is sinks + window: evict by position
     const int4* items;             // attention items, then score items
     int32_t n_items;
     int32_t n_score_items;
@@ -203,6 +205,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     __shared__ float sm_invL[kG];
     __shared__ int sm_last;
     __shared__ int sm_abort;
+    __shared__ int sm_old_pos[kConsumerWarps];
+    __shared__ int sm_old_slot[kConsumerWarps];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.G;
@@ -223,6 +227,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const int end = min(begin + chunk_len, n_hi);
     const int n_tiles = end > begin ? (end - begin + kTileTokens - 1) / kTileTokens : 0;
     const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
+    // sinks + window without scores: the one row that is neither a sink nor in the window (the oldest) goes
+    const bool pos_evict = p.window_evict && hs.do_append && n_hi > C - 1;
+    const int window_from = p.t_pos - max(0, (int)(((int64_t)(C - 1 - p.n_sink) * p.recent_num) / p.recent_den));
+    int old_pos = INT32_MAX, old_slot = -1;                // per lane, then per warp: oldest evictable row seen
 
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
     // this head's share of the scratch: unnormalised probabilities [G][C] in fp16, each relative to the
@@ -319,6 +327,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                     if (lane == 0) { p.pos[row] = p.t_pos; p.score[row] = 0.0f; }
                     __syncwarp();
                 }
+                if (pos_evict && lane < valid && tok0 + lane != hs.f) {
+                    const int ps = p.pos[row0 + tok0 + lane];
+                    if (ps >= p.n_sink && ps <= window_from && ps < old_pos) { old_pos = ps; old_slot = tok0 + lane; }
+                }
                 // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
                 if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
                     uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
@@ -396,6 +408,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     // ---- the four warps' states -> one partial for the chunk (the ring is idle now: reuse it)
     float* sm_o = reinterpret_cast<float*>(ring_ptr);       // [kConsumerWarps][G][D]
     if (warp < kConsumerWarps) {
+        if (pos_evict) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const int op = __shfl_xor_sync(0xffffffffu, old_pos, off);
+                const int os = __shfl_xor_sync(0xffffffffu, old_slot, off);
+                if (op < old_pos) { old_pos = op; old_slot = os; }
+            }
+            if (lane == 0) { sm_old_pos[warp] = old_pos; sm_old_slot[warp] = old_slot; }
+        }
         float lq = l_run;
         lq += __shfl_xor_sync(0xffffffffu, lq, 1);
         lq += __shfl_xor_sync(0xffffffffu, lq, 2);
@@ -407,7 +428,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         }
     }
     __syncthreads();
-    const int psz = G * D + 2 * G;
+    const int psz = G * D + 2 * G + 2;                      // o, m, l, and the chunk's oldest evictable row
     float* part = p.partial + (int64_t)blockIdx.x * psz;
     for (int i = tid; i < G * D; i += kThreads) {
         const int a = i / D, d = i - a * D;
@@ -423,6 +444,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         }
         part[i] = acc;
         if (d == 0) { part[G * D + a] = mm; part[G * D + G + a] = lsum; }
+    }
+    if (pos_evict && tid == 0) {
+        int bp = INT32_MAX, bs = -1;
+        for (int w = 0; w < kConsumerWarps; ++w)
+            if (sm_old_pos[w] < bp) { bp = sm_old_pos[w]; bs = sm_old_slot[w]; }
+        part[G * D + 2 * G] = __int_as_float(bp);
+        part[G * D + 2 * G + 1] = __int_as_float(bs);
     }
     __threadfence();
     __syncthreads();
@@ -483,8 +511,22 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     if (tid == 0) {
         p.arrive[unit] = 0;                                 // the score kernel counts arrivals again
         if (!keep_logits && hs.do_append) {                 // no score pass follows: finish the bookkeeping here
-            p.len[u.st] = n + 1;
-            p.free_slot[u.st] = n + 1;
+            int victim = -1;
+            if (pos_evict) {
+                int bp = INT32_MAX;
+                for (int c = 0; c < active; ++c) {
+                    const float* pc = part0 + (int64_t)c * psz + G * D + 2 * G;
+                    const int cp = __float_as_int(__ldcg(pc));
+                    if (cp < bp) { bp = cp; victim = __float_as_int(__ldcg(pc + 1)); }
+                }
+                if (victim < 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);   // nothing outside sinks + window
+            }
+            if (victim >= 0) {
+                p.free_slot[u.st] = victim;                 // len stays n: one row in, one row out (Eq. 5-6)
+            } else {
+                p.len[u.st] = n + 1;
+                p.free_slot[u.st] = n + 1;
+            }
         }
     }
 }
@@ -758,7 +800,10 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lse = lse;
     p.t_pos = t_pos;
-    p.flags = (flags & BAKLAVA_FLAG_NO_SCORE) ? (flags | BAKLAVA_FLAG_NO_EVICT) : flags;
+    // without scores only the pure sinks + window policy can still choose a victim (by position)
+    p.window_evict = (flags & BAKLAVA_FLAG_NO_SCORE) && !(flags & BAKLAVA_FLAG_NO_EVICT) &&
+                     shape->recent_num == shape->recent_den;
+    p.flags = ((flags & BAKLAVA_FLAG_NO_SCORE) && !p.window_evict) ? (flags | BAKLAVA_FLAG_NO_EVICT) : flags;
     p.items = reinterpret_cast<const int4*>(items);
     p.n_items = info->n_items;
     p.n_score_items = info->n_score_items;

@@ -170,7 +170,7 @@ size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t 
     w.arrive_off = take(sizeof(int32_t) * (size_t)n_units);
     w.stats_off = take(sizeof(float) * (size_t)n_units * 2 * BAKLAVA_MAX_GROUP);
     w.best_off = take(16 * (size_t)n_score_items);
-    w.partial_off = take(sizeof(float) * (size_t)n_items * g * (s->D + 2));
+    w.partial_off = take(sizeof(float) * (size_t)n_items * (g * (s->D + 2) + 2));
     w.logit_off = take(sizeof(float) * (size_t)B * (size_t)seq_stride_tokens * g);
     w.total = off;
     if (lay) *lay = w;

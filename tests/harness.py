@@ -138,7 +138,8 @@ class Session:
             li = l - self.lb
             o_ref, lse_ref, ev = tw.step(qh[li, b, h * g:(h + 1) * g], knh[li, b, h], vnh[li, b, h], t_pos,
                                          append=append, update_score=not (flags & bk.FLAG_NO_SCORE),
-                                         evict=not (flags & (bk.FLAG_NO_EVICT | bk.FLAG_NO_SCORE)))
+                                         evict=not (flags & bk.FLAG_NO_EVICT) and
+                                         (not (flags & bk.FLAG_NO_SCORE) or w.recent_num == w.recent_den))
             tag = "step %d head (b%d,l%d,h%d)" % (step_index, b, l, h)
             assert_close(out[li, b, h * g:(h + 1) * g], o_ref, tag + " out")
             assert_close(lse[li, b, h * g:(h + 1) * g], lse_ref, tag + " lse")

@@ -95,6 +95,33 @@ def test_flags():
     assert all(tw.length == tw.C for tw in s.twins.values())
 
 
+def test_window_only_policy_without_scores():
+    """The paper's evaluated policy (sinks + recent window): with NO_SCORE the library keeps no scores and
+    still evicts, by position.  Checked against the oracle and against the closed form of what must remain."""
+    w = wl.scaled(wl.LLAMA3_8B_32K, L=2, T=900, steps=40, recent_num=1, recent_den=1)
+    s = Session(w, chunk_tokens=128)
+    score_before = s.cache.score.clone()
+    for i in range(w.steps):
+        s.step(i, flags=bk.FLAG_NO_SCORE)
+    assert torch.equal(score_before[s.cache.pos.ne(-1) & (s.cache.pos < w.T)],
+                       s.cache.score[s.cache.pos.ne(-1) & (s.cache.pos < w.T)])      # old rows' scores untouched
+    t_last = w.T + w.steps - 1
+    for (b, l, h) in s.heads:
+        st = s.head_state(b, l, h)
+        kept = sorted(st["pos"][s.valid_slots(st)])
+        R = int(s.cap[l, h]) - 1
+        if t_last + 1 <= R:
+            assert kept == list(range(t_last + 1))
+        else:
+            assert kept == list(range(w.n_sink)) + list(range(t_last + 1 - (R - w.n_sink), t_last + 1))
+    # filling an empty cache under the same policy
+    w2 = wl.scaled(wl.TINY, T=64, steps=70, recent_num=1, recent_den=1)
+    s2 = Session(w2, prefill=False, chunk_tokens=64)
+    for i in range(w2.steps):
+        s2.step(i, flags=bk.FLAG_NO_SCORE)
+    assert all(tw.length == tw.C - 1 for tw in s2.twins.values())
+
+
 def test_overflow_sets_status_and_keeps_state():
     w = wl.scaled(wl.TINY, T=200, steps=4)
     s = Session(w, chunk_tokens=64)
