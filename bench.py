@@ -232,6 +232,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="only the first LAYERS layers (for profiling a small case)")
     ap.add_argument("--chunk", type=int, default=0, help="force the plan's chunk length (tokens); 0 = automatic")
+    ap.add_argument("--policy", default="heavy", choices=["heavy", "window"],
+                    help="heavy: sinks + window + accumulated-attention heavy hitters (default); "
+                         "window: the paper's evaluated sinks + window policy, run without scores")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.workload == "profile":
@@ -239,6 +242,8 @@ def main():
     w = WORKLOADS[args.workload]
     if args.layers:
         w = wl.scaled(w, L=args.layers)
+    if args.policy == "window":
+        w = wl.scaled(w, name=w.name + "-window", recent_num=1, recent_den=1)
     if args.impl == "reference":
         return run_reference(args, w)
 
@@ -255,6 +260,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     bk.lib()                                             # fail now if the library is missing
+    step_flags = bk.FLAG_NO_SCORE if args.policy == "window" else 0
     sess = DecodeSession(w, dev, chunk_tokens=args.chunk)
     sess.prefill_synthetic()
     total = args.warmup + args.steps
@@ -270,13 +276,13 @@ def main():
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     with ClockSampler(local) as clocks:
         for i in range(args.warmup):                       # load the GPU before the clock window opens
-            sess.step(*feeds[i])
+            sess.step(*feeds[i], flags=step_flags)
         barrier()
         rows_per_step = int(sess.cache.len.sum().item()) + sess.plan.info.n_units   # rows attended: retained + new
         t_open = time.perf_counter()
         ev[0].record()
         for i in range(args.steps):
-            sess.step(*feeds[args.warmup + i])
+            sess.step(*feeds[args.warmup + i], flags=step_flags)
         ev[1].record()
         torch.cuda.synchronize(dev)
         t_close = time.perf_counter()
@@ -294,7 +300,7 @@ def main():
     def e2e_step(i):
         q, k, v = host[i]
         dq.copy_(q, non_blocking=True); dk.copy_(k, non_blocking=True); dv.copy_(v, non_blocking=True)
-        out_host.copy_(sess.step(dq, dk, dv), non_blocking=True)
+        out_host.copy_(sess.step(dq, dk, dv, flags=step_flags), non_blocking=True)
 
     for i in range(args.warmup):
         e2e_step(i)
@@ -324,7 +330,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "layers": w.L, "batch": w.B, "context": w.T, "budget": w.budget,
                        "kv_bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (no flush)",
-                       "launch": "one baklava_decode_attn call per step covering all layers",
+                       "launch": "one baklava_decode_attn call per step covering all layers", "policy": args.policy,
                        "replicas": world},
             "tokens_per_s": whole_job_rate(world, w.B, args.steps, elapsed_ms),
             "pct_of_hbm_peak": 100.0 * gbs / world / peak,
@@ -333,7 +339,7 @@ def main():
                          "peak_kind": peak_kind, "kernel": "decode_chunk_kernel",
                          "note": "events bracket one call = attention kernel + score/evict kernel"},
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": 2 * args.steps,
+            "gpu_launches": (1 if args.policy == "window" else 2) * args.steps,
             "clocks": clocks.summary(t_open, t_close),
         }
         if world == 1 and not args.no_cpu_baseline:
