@@ -226,6 +226,22 @@ int baklava_evict(const baklava_shape* shape, const baklava_cache* cache,
                   void* ws, size_t ws_bytes, void* stream);
 size_t baklava_evict_workspace_size(const baklava_shape* shape, int32_t B, int32_t layers, int32_t T);
 
+/* ------------------------------------------------------------------ prompt scores (seed of step 3)
+ * The accumulated attention a prompt leaves on its own tokens, for ONE layer: with the causal
+ * attention matrix A_h = softmax(Q_h K^T / sqrt(D)) of Eq. 1,
+ *     score[b, c, j] = sum over the g query heads h of KV head c, sum over rows i >= j of A_h[i, j],
+ * exactly what decoding the prompt one token at a time through baklava_decode_attn would have
+ * accumulated.  It is the score_dense input of baklava_evict (stride_seq = Hkv * T, stride_head = T).
+ *   q           device bf16 [B, Hq, T, D]
+ *   k           device bf16 [B, Hkv, T, D]
+ *   prompt_len  device int32 [B] (rows and keys at or past len count for nothing) or NULL for len = T
+ *   score       device fp32 [B, Hkv, T], overwritten
+ *   ws          device workspace >= baklava_prefill_workspace_size() bytes */
+int baklava_prefill_scores(const baklava_shape* shape, const void* q, const void* k,
+                           const int32_t* prompt_len, int32_t B, int32_t T,
+                           float* score, void* ws, size_t ws_bytes, void* stream);
+size_t baklava_prefill_workspace_size(const baklava_shape* shape, int32_t B, int32_t T);
+
 /* ------------------------------------------------------------------ bulk eviction, no workspace
  * (No counterpart in the paper: this is a packaging variant of baklava_evict.)
  * Same operation, arguments and results as baklava_evict, for callers that cannot provide a

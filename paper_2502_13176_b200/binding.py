@@ -78,6 +78,10 @@ def lib():
                                            c_void_p, c_int32, c_int64, c_int64, c_int64, c_int32, c_void_p]
         L.baklava_profile_heads.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                             c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.baklava_prefill_scores.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_int32, c_int32,
+                                             c_void_p, c_void_p, c_size_t, c_void_p]
+        L.baklava_prefill_workspace_size.restype = c_size_t
+        L.baklava_prefill_workspace_size.argtypes = [POINTER(Shape), c_int32, c_int32]
         L.baklava_profile_workspace_size.restype = c_size_t
         L.baklava_profile_workspace_size.argtypes = [POINTER(Shape), c_int32, c_int32]
         _lib = L
@@ -242,3 +246,13 @@ def baklava_profile_heads(shape, q, k, v, prompt_len, P, T, head_cos, token_cos,
                                        _ptr(head_cos), _ptr(token_cos), _ptr(ws),
                                        0 if ws is None else ws.numel() * ws.element_size(), _stream(stream)),
            "baklava_profile_heads")
+
+
+def baklava_prefill_workspace_size(shape, B, T):
+    return int(lib().baklava_prefill_workspace_size(ctypes.byref(shape), B, T))
+
+
+def baklava_prefill_scores(shape, q, k, prompt_len, B, T, score, ws, stream=None):
+    _check(lib().baklava_prefill_scores(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(prompt_len), B, T, _ptr(score),
+                                        _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "baklava_prefill_scores")
