@@ -221,12 +221,44 @@ def run_profile_pass(args):
                       "gpu_launches": 2 * args.steps, "clocks": clocks.summary(t_open, t_close)}))
 
 
+def run_prefill_scores(args):
+    """Exact seeding of the heavy-hitter scores for one layer of a 32K prompt (two passes over Q K^T)."""
+    from paper_2502_13176_b200 import binding as bk, synth
+    from paper_2502_13176_b200.engine import shape_of
+
+    w = wl.LLAMA3_8B_32K
+    B, T = 1, args.prompt_tokens
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    shape = shape_of(w)
+    q = synth.normal_bf16(w.seed, wl.T_PROFILE_Q, (B, w.Hq, T, w.D), dev)
+    k = synth.normal_bf16(w.seed, wl.T_PROFILE_K, (B, w.Hkv, T, w.D), dev)
+    score = torch.empty((B, w.Hkv, T), dtype=torch.float32, device=dev)
+    ws = torch.empty((bk.baklava_prefill_workspace_size(shape, B, T),), dtype=torch.uint8, device=dev)
+    for _ in range(args.warmup):
+        bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    e0.record()
+    for _ in range(args.steps):
+        bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    ms = e0.elapsed_time(e1) / args.steps
+    flop = 2 * B * w.Hq * 1.0 * T * T * w.D           # Q K^T under the causal mask, twice
+    tf = flop / (ms * 1e-3) / 1e12
+    print(json.dumps({"metric": "prompt-score seeding TFLOP/s (one layer)", "value": tf, "unit": "TFLOP/s",
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "dtype": "bf16",
+                      "config": {"workload": "prefill-scores-llama3-8b", "batch": B, "prompt_tokens": T},
+                      "gpu_launches": 2 * args.steps}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=8)
-    ap.add_argument("--workload", default="llama", choices=sorted(WORKLOADS) + ["profile"])
+    ap.add_argument("--workload", default="llama", choices=sorted(WORKLOADS) + ["profile", "prefill"])
     ap.add_argument("--prompts", type=int, default=64, help="profile workload: prompts per step")
     ap.add_argument("--prompt-tokens", type=int, default=4096, help="profile workload: tokens per prompt")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -239,6 +271,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "profile":
         return run_profile_pass(args)
+    if args.workload == "prefill":
+        return run_prefill_scores(args)
     w = WORKLOADS[args.workload]
     if args.layers:
         w = wl.scaled(w, L=args.layers)
