@@ -186,7 +186,9 @@ __device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
 }
 
 // ---------------------------------------------------------------- steps 2-4
-template <int D>
+// kByPosition: the score-free sinks + window policy (a second instantiation, so that the default
+// path carries none of its registers or branches).
+template <int D, bool kByPosition>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(const DecodeParams p,
                                                                 const __grid_constant__ CUtensorMap k_map,
                                                                 const __grid_constant__ CUtensorMap v_map) {
@@ -228,7 +230,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const int n_tiles = end > begin ? (end - begin + kTileTokens - 1) / kTileTokens : 0;
     const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
     // sinks + window without scores: the one row that is neither a sink nor in the window (the oldest) goes
-    const bool pos_evict = p.window_evict && hs.do_append && n_hi > C - 1;
+    const bool pos_evict = kByPosition && hs.do_append && n_hi > C - 1;
     const int window_from = p.t_pos - max(0, (int)(((int64_t)(C - 1 - p.n_sink) * p.recent_num) / p.recent_den));
     int old_pos = INT32_MAX, old_slot = -1;                // per lane, then per warp: oldest evictable row seen
 
@@ -327,7 +329,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                     if (lane == 0) { p.pos[row] = p.t_pos; p.score[row] = 0.0f; }
                     __syncwarp();
                 }
-                if (pos_evict && lane < valid && tok0 + lane != hs.f) {
+                if (kByPosition && pos_evict && lane < valid && tok0 + lane != hs.f) {
                     const int ps = p.pos[row0 + tok0 + lane];
                     if (ps >= p.n_sink && ps <= window_from && ps < old_pos) { old_pos = ps; old_slot = tok0 + lane; }
                 }
@@ -408,7 +410,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     // ---- the four warps' states -> one partial for the chunk (the ring is idle now: reuse it)
     float* sm_o = reinterpret_cast<float*>(ring_ptr);       // [kConsumerWarps][G][D]
     if (warp < kConsumerWarps) {
-        if (pos_evict) {
+        if (kByPosition && pos_evict) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
                 const int op = __shfl_xor_sync(0xffffffffu, old_pos, off);
@@ -445,7 +447,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         part[i] = acc;
         if (d == 0) { part[G * D + a] = mm; part[G * D + G + a] = lsum; }
     }
-    if (pos_evict && tid == 0) {
+    if (kByPosition && pos_evict && tid == 0) {
         int bp = INT32_MAX, bs = -1;
         for (int w = 0; w < kConsumerWarps; ++w)
             if (sm_old_pos[w] < bp) { bp = sm_old_pos[w]; bs = sm_old_slot[w]; }
@@ -512,7 +514,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         p.arrive[unit] = 0;                                 // the score kernel counts arrivals again
         if (!keep_logits && hs.do_append) {                 // no score pass follows: finish the bookkeeping here
             int victim = -1;
-            if (pos_evict) {
+            if (kByPosition && pos_evict) {
                 int bp = INT32_MAX;
                 for (int c = 0; c < active; ++c) {
                     const float* pc = part0 + (int64_t)c * psz + G * D + 2 * G;
@@ -725,10 +727,10 @@ bool make_slab_map(CUtensorMap* map, void* base, int64_t rows, int D) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D>
+template <int D, bool kByPosition>
 cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
     constexpr int kSmem = kStages * 2 * kTileTokens * D * 2 + 1024;
-    cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D, kByPosition>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -740,7 +742,7 @@ cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CU
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_chunk_kernel<D>, p, km, vm);
+    return cudaLaunchKernelEx(&cfg, decode_chunk_kernel<D, kByPosition>, p, km, vm);
 }
 
 }  // namespace
@@ -818,7 +820,8 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
-    err = shape->D == 128 ? launch_chunks<128>(p, k_map, v_map, s) : launch_chunks<64>(p, k_map, v_map, s);
+    if (p.window_evict) err = shape->D == 128 ? launch_chunks<128, true>(p, k_map, v_map, s) : launch_chunks<64, true>(p, k_map, v_map, s);
+    else err = shape->D == 128 ? launch_chunks<128, false>(p, k_map, v_map, s) : launch_chunks<64, false>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     if (!(p.flags & BAKLAVA_FLAG_NO_SCORE)) {
         void (*score_fn)(const DecodeParams) = nullptr;
