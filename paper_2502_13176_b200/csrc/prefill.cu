@@ -2,10 +2,13 @@
 // processed, i.e. the column sums of the causal attention matrix of Eq. 1, added over the g query heads
 // that share a KV head.
 //
-// Two passes over Q K^T (V is not needed).  Pass 1 gives every query row its log-sum-exp; pass 2 owns
-// key blocks: a CTA keeps 64 keys as the A operand in registers, streams every query tile at or below
-// them through a two-stage TMA ring, turns logits into probabilities with the rows' log-sum-exp and
-// adds them up per key.  Every sum has a fixed order, so the result is reproducible bit for bit.
+// Two passes over Q K^T (V is not needed), both on the 5th-generation tensor cores.  A CTA keeps one
+// 128-row operand tile resident in shared memory and streams the other operand's tiles through a
+// two-stage TMA ring; one thread issues tcgen05.mma into a double-buffered 128 x 128 fp32 accumulator in
+// tensor memory; four epilogue warps read it back with tcgen05.ld, one accumulator row per thread.
+//   pass 1 (rows = queries): every query row's log-sum-exp, a running max / sum kept by its thread;
+//   pass 2 (rows = keys):    exp2(logit - lse[query]) summed along each key's row, again by its thread.
+// No reduction crosses a thread, so every sum has a fixed order and the result is reproducible.
 #include <cmath>
 #include <cstdint>
 
@@ -17,9 +20,12 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kRows = 64;          // query rows / keys per tile
-constexpr int kThreads = 128;
+constexpr int kTileRows = 128;       // rows of an operand tile = accumulator rows = accumulator columns
+constexpr int kThreads = 192;        // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
+constexpr int kEpilogueThreads = 128;
+constexpr uint32_t kTmemColumns = 256;   // two 128-column accumulators
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kPassLse = 0, kPassColumnSums = 1;
 
 struct PrefillParams {
     const int32_t* prompt_len;   // [B] or null
@@ -30,259 +36,219 @@ struct PrefillParams {
     float scale_log2;
 };
 
-// ---------------------------------------------------------------- pass 1: row log-sum-exp
-template <int D>
-__global__ void __launch_bounds__(kThreads) prefill_lse_kernel(const PrefillParams p,
-                                                               const __grid_constant__ CUtensorMap q_map,
-                                                               const __grid_constant__ CUtensorMap k_map) {
-    constexpr int kKSteps = D / 16;
-    constexpr int kTileBytes = kRows * D * 2;
+template <int D, int PASS>
+__global__ void __launch_bounds__(kThreads) qk_pass_kernel(const PrefillParams p,
+                                                           const __grid_constant__ CUtensorMap q_map,
+                                                           const __grid_constant__ CUtensorMap k_map) {
+    constexpr int kKSteps = D / 16;                         // one MMA covers 16 elements of the head dimension
+    constexpr int kBoxBytes = kTileRows * 128;              // one TMA box: 128 rows x 64 elements
+    constexpr int kTileBytes = kTileRows * D * 2;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q;
-    __shared__ __align__(8) uint64_t bar_k[2];
+    __shared__ __align__(8) uint64_t bar_res, bar_full[2], bar_empty[2], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ float sm_lse[2][kTileRows];
     __shared__ int sm_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int qb = p.n_blk - 1 - blockIdx.x;               // long rows of the causal triangle first
-    const int h = blockIdx.y, b = blockIdx.z;
-    const int kvh = h / (p.Hq / p.Hkv);
-    const int len = p.prompt_len ? min(max(p.prompt_len[b], 0), p.T) : p.T;
-    float* lse_row = p.lse2 + ((int64_t)b * p.Hq + h) * p.T;
-    if (qb * kRows >= len) {
-        for (int r = tid; r < kRows; r += kThreads)
-            if (qb * kRows + r < p.T) lse_row[qb * kRows + r] = INFINITY;
-        return;
-    }
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_tile = base;
-    if (tid == 0) {
-        mbar_init(smem_u32(&bar_q), 1);
-        mbar_init(smem_u32(&bar_k[0]), 1);
-        mbar_init(smem_u32(&bar_k[1]), 1);
-        sm_abort = 0;
-        fence_mbar_init();
-    }
-    __syncthreads();
-    auto issue_k = [&](int kb) {
-        const uint32_t bar = smem_u32(&bar_k[kb & 1]);
-        mbar_arrive_expect_tx(bar, kTileBytes);
-#pragma unroll
-        for (int bx = 0; bx < D / 64; ++bx)
-            tma_load_3d(base + (1 + (kb & 1)) * kTileBytes + bx * (kRows * 128), &k_map, bx * 64, kb * kRows,
-                        b * p.Hkv + kvh, bar);
-    };
-    if (tid == 0) {
-        mbar_arrive_expect_tx(smem_u32(&bar_q), kTileBytes);
-#pragma unroll
-        for (int bx = 0; bx < D / 64; ++bx)
-            tma_load_3d(q_tile + bx * (kRows * 128), &q_map, bx * 64, qb * kRows, b * p.Hq + h, smem_u32(&bar_q));
-        issue_k(0);
-    }
-    const int r0 = warp * 16;
-    const int lm = lane >> 3, li8 = lane & 7;
-    const int qrow = lane >> 2, qcol = (lane & 3) * 2;
-    bool alive = mbar_wait(smem_u32(&bar_q), 0);
-    uint32_t qa[kKSteps][4];
-    if (alive) {
-#pragma unroll
-        for (int ks = 0; ks < kKSteps; ++ks)
-            ldmatrix_x4(q_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * ks + (lm >> 1)), qa[ks]);
-    }
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
-    for (int kb = 0; kb <= qb; ++kb) {
-        __syncthreads();
-        if (sm_abort) break;
-        if (tid == 0 && kb + 1 <= qb) issue_k(kb + 1);
-        if (!alive || !mbar_wait(smem_u32(&bar_k[kb & 1]), (kb >> 1) & 1)) {
-            alive = false;
-            sm_abort = 1;
-            continue;
-        }
-        const uint32_t k_tile = base + (1 + (kb & 1)) * kTileBytes;
-        float sacc[8][4];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) { sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.0f; }
-#pragma unroll
-        for (int ks = 0; ks < kKSteps; ++ks)
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                uint32_t kf[4];
-                ldmatrix_x4(k_tile + tile_offset(16 * kk + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kf);
-                mma_bf16(sacc[2 * kk], qa[ks], kf[0], kf[1]);
-                mma_bf16(sacc[2 * kk + 1], qa[ks], kf[2], kf[3]);
-            }
-        const bool diagonal = kb == qb;
-        float mx[2] = {-INFINITY, -INFINITY};
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float v = sacc[nt][e] * p.scale_log2;
-                if (diagonal && 8 * nt + qcol + (e & 1) > r0 + qrow + (e >> 1) * 8) v = -INFINITY;   // causal mask
-                sacc[nt][e] = v;
-                mx[e >> 1] = fmaxf(mx[e >> 1], v);
-            }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-            const float m_new = fmaxf(m_run[r], mx[r]);      // finite: key 0 is never masked
-            l_run[r] *= exp2f(m_run[r] - m_new);
-            m_run[r] = m_new;
-        }
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) l_run[e >> 1] += exp2f(sacc[nt][e] - m_run[e >> 1]);
-    }
-    __syncthreads();
-    if (sm_abort) {
-        if (tid == 0) atomicOr(p.error, 1u);
-        return;
-    }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        float l = l_run[r];
-        l += __shfl_xor_sync(0xffffffffu, l, 1);
-        l += __shfl_xor_sync(0xffffffffu, l, 2);
-        const int t = qb * kRows + r0 + qrow + r * 8;
-        if ((lane & 3) == 0 && t < p.T) lse_row[t] = t < len ? m_run[r] + log2f(l) : INFINITY;
-    }
-}
-
-// ---------------------------------------------------------------- pass 2: column sums per key block
-template <int D>
-__global__ void __launch_bounds__(kThreads) prefill_colsum_kernel(const PrefillParams p,
-                                                                  const __grid_constant__ CUtensorMap q_map,
-                                                                  const __grid_constant__ CUtensorMap k_map) {
-    constexpr int kKSteps = D / 16;
-    constexpr int kTileBytes = kRows * D * 2;
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_k;
-    __shared__ __align__(8) uint64_t bar_q[2];
-    __shared__ float sm_lse[2][kRows];
-    __shared__ int sm_abort;
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int kb = blockIdx.x;                              // early key blocks have the most query tiles: first
-    const int kvh = blockIdx.y, b = blockIdx.z;
     const int g = p.Hq / p.Hkv;
+    const int b = blockIdx.z;
     const int len = p.prompt_len ? min(max(p.prompt_len[b], 0), p.T) : p.T;
-    if (kb * kRows >= len) {                                // keys past the prompt receive nothing
-        for (int r = tid; r < kRows; r += kThreads)
-            if (kb * kRows + r < p.T) p.score[((int64_t)b * p.Hkv + kvh) * p.T + kb * kRows + r] = 0.0f;
-        return;
+    int blk, n_it, nq = 1, head_res, head_first;            // resident block, streamed tiles, heads
+    if (PASS == kPassLse) {
+        blk = p.n_blk - 1 - blockIdx.x;                     // long rows of the causal triangle first
+        const int h = blockIdx.y;
+        head_res = b * p.Hq + h;
+        head_first = b * p.Hkv + h / g;
+        n_it = blk + 1;
+        if (blk * kTileRows >= len) {
+            for (int r = tid; r < kTileRows; r += kThreads)
+                if (blk * kTileRows + r < p.T) p.lse2[(int64_t)head_res * p.T + blk * kTileRows + r] = INFINITY;
+            return;
+        }
+    } else {
+        blk = blockIdx.x;                                   // early key blocks meet the most query tiles: first
+        const int kvh = blockIdx.y;
+        head_res = b * p.Hkv + kvh;
+        head_first = b * p.Hq + kvh * g;
+        if (blk * kTileRows >= len) {                       // keys past the prompt receive nothing
+            for (int r = tid; r < kTileRows; r += kThreads)
+                if (blk * kTileRows + r < p.T) p.score[(int64_t)head_res * p.T + blk * kTileRows + r] = 0.0f;
+            return;
+        }
+        nq = (len + kTileRows - 1) / kTileRows - blk;       // query tiles of the prompt at or below this key block
+        n_it = g * nq;
     }
-    const int nq = (len + kRows - 1) / kRows - kb;          // query tiles of the prompt at or below this key block
-    const int n_it = g * nq;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t k_tile = base;
+    const uint32_t res_tile = base;
     if (tid == 0) {
-        mbar_init(smem_u32(&bar_k), 1);
-        mbar_init(smem_u32(&bar_q[0]), 1);
-        mbar_init(smem_u32(&bar_q[1]), 1);
+        mbar_init(smem_u32(&bar_res), 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+            mbar_init(smem_u32(&bar_acc_full[s]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[s]), kEpilogueThreads / 32);
+        }
         sm_abort = 0;
         fence_mbar_init();
     }
-    __syncthreads();
-    auto issue_q = [&](int it) {
-        const int a = it / nq, qb = kb + it % nq;
-        const uint32_t bar = smem_u32(&bar_q[it & 1]);
-        mbar_arrive_expect_tx(bar, kTileBytes);
-#pragma unroll
-        for (int bx = 0; bx < D / 64; ++bx)
-            tma_load_3d(base + (1 + (it & 1)) * kTileBytes + bx * (kRows * 128), &q_map, bx * 64, qb * kRows,
-                        b * p.Hq + kvh * g + a, bar);
-    };
-    auto fetch_lse = [&](int it) -> float {                  // threads 0..63: one query row of tile `it`
-        const int a = it / nq, qb = kb + it % nq;
-        const int t = qb * kRows + tid;
-        return t < p.T ? p.lse2[((int64_t)b * p.Hq + kvh * g + a) * p.T + t] : INFINITY;
-    };
-    if (tid == 0) {
-        mbar_arrive_expect_tx(smem_u32(&bar_k), kTileBytes);
-#pragma unroll
-        for (int bx = 0; bx < D / 64; ++bx)
-            tma_load_3d(k_tile + bx * (kRows * 128), &k_map, bx * 64, kb * kRows, b * p.Hkv + kvh, smem_u32(&bar_k));
-        issue_q(0);
+    if (warp == 1) {
+        tc::tmem_alloc(smem_u32(&tmem_slot), kTmemColumns);
+        tc::tmem_relinquish();
     }
-    if (tid < kRows) sm_lse[0][tid] = fetch_lse(0);
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
 
-    const int r0 = warp * 16;                               // this warp's keys inside the block
-    const int lm = lane >> 3, li8 = lane & 7;
-    const int qrow = lane >> 2, qcol = (lane & 3) * 2;
-    bool alive = mbar_wait(smem_u32(&bar_k), 0);
-    uint32_t ka[kKSteps][4];                                // the warp's 16 keys as the A operand, kept all along
-    if (alive) {
+    // which streamed tile iteration `it` is: (head of the group, row block)
+    auto stream_head = [&](int it) { return PASS == kPassLse ? head_first : head_first + it / nq; };
+    auto stream_blk = [&](int it) { return PASS == kPassLse ? it : blk + it % nq; };
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            const CUtensorMap* res_map = PASS == kPassLse ? &q_map : &k_map;
+            const CUtensorMap* str_map = PASS == kPassLse ? &k_map : &q_map;
+            mbar_arrive_expect_tx(smem_u32(&bar_res), kTileBytes);
 #pragma unroll
-        for (int ks = 0; ks < kKSteps; ++ks)
-            ldmatrix_x4(k_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * ks + (lm >> 1)), ka[ks]);
-    }
-    float colsum[2] = {0.0f, 0.0f};                          // keys r0 + qrow and r0 + qrow + 8
-    for (int it = 0; it < n_it; ++it) {
-        __syncthreads();                                    // tile it - 1 is consumed; sm_lse[it & 1] is in place
-        if (sm_abort) break;
-        if (it + 1 < n_it) {
-            if (tid == 0) issue_q(it + 1);
-            if (tid < kRows) sm_lse[(it + 1) & 1][tid] = fetch_lse(it + 1);
+            for (int bx = 0; bx < D / 64; ++bx)
+                tma_load_3d(res_tile + bx * kBoxBytes, res_map, bx * 64, blk * kTileRows, head_res, smem_u32(&bar_res));
+            for (int it = 0; it < n_it; ++it) {
+                const int s = it & 1;
+                if (it >= 2 && !mbar_wait(smem_u32(&bar_empty[s]), ((it >> 1) - 1) & 1)) { sm_abort = 1; break; }
+                const uint32_t bar = smem_u32(&bar_full[s]);
+                mbar_arrive_expect_tx(bar, kTileBytes);
+#pragma unroll
+                for (int bx = 0; bx < D / 64; ++bx)
+                    tma_load_3d(base + (1 + s) * kTileBytes + bx * kBoxBytes, str_map, bx * 64,
+                                stream_blk(it) * kTileRows, stream_head(it), bar);
+            }
         }
-        if (!alive || !mbar_wait(smem_u32(&bar_q[it & 1]), (it >> 1) & 1)) {
-            alive = false;
+    } else if (warp == 1) {
+        // ---------------- MMA issuer: D[128 x 128] = resident (A) x streamed^T (B), both K-major
+        if (lane == 0) {
+            constexpr uint32_t idesc = tc::idesc_bf16_f32(kTileRows, kTileRows);
+            bool ok = mbar_wait(smem_u32(&bar_res), 0);
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int s = it & 1;
+                ok = mbar_wait(smem_u32(&bar_full[s]), (it >> 1) & 1);
+                if (ok && it >= 2) ok = mbar_wait(smem_u32(&bar_acc_empty[s]), ((it >> 1) - 1) & 1);
+                if (!ok) break;
+                tc::fence_after_sync();
+                const uint32_t str_tile = base + (1 + s) * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < kKSteps; ++ks) {
+                    const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;    // 64-element span, then 32 B per step
+                    tc::umma_bf16(tmem_base + s * kTileRows, tc::desc_k_major_sw128(res_tile + off),
+                                  tc::desc_k_major_sw128(str_tile + off), idesc, ks > 0);
+                }
+                tc::umma_commit(smem_u32(&bar_empty[s]));        // the stage may be overwritten
+                tc::umma_commit(smem_u32(&bar_acc_full[s]));     // the accumulator may be read
+            }
+            if (!ok) sm_abort = 1;
+        }
+    } else {
+        // ---------------- epilogue: thread = accumulator row (its warp's quarter of the TMEM lanes)
+        const int e = tid - 64;
+        const int row = 32 * (warp & 3) + lane;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+        float m_run = -INFINITY, l_run = 0.0f, colsum = 0.0f;
+        auto fetch_lse = [&](int it) -> float {              // the log-sum-exp of streamed query row e of tile it
+            const int t = stream_blk(it) * kTileRows + e;
+            return t < p.T ? p.lse2[(int64_t)stream_head(it) * p.T + t] : INFINITY;
+        };
+        if (PASS == kPassColumnSums) {
+            sm_lse[0][e] = fetch_lse(0);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        bool ok = true;
+        for (int it = 0; it < n_it; ++it) {
+            const int s = it & 1;
+            float next_lse = 0.0f;
+            if (PASS == kPassColumnSums && it + 1 < n_it) next_lse = fetch_lse(it + 1);
+            if (!mbar_wait(smem_u32(&bar_acc_full[s]), (it >> 1) & 1)) { ok = false; break; }
+            tc::fence_after_sync();
+            const bool diagonal = stream_blk(it) == blk;
+            const uint32_t acc = lane_addr + s * kTileRows;
+            if (PASS == kPassLse) {
+                // row = query, columns = keys: keys above the query are masked on the diagonal tile
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld_32x32(acc + c0, v);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (!(diagonal && c0 + c > row)) mx = fmaxf(mx, __uint_as_float(v[c]));
+                }
+                const float m_new = fmaxf(m_run, mx * p.scale_log2);       // finite: key 0 is never masked
+                float sum = 0.0f;
+#pragma unroll
+                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld_32x32(acc + c0, v);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (!(diagonal && c0 + c > row)) sum += exp2f(__uint_as_float(v[c]) * p.scale_log2 - m_new);
+                }
+                l_run = l_run * exp2f(m_run - m_new) + sum;
+                m_run = m_new;
+            } else {
+                // row = key, columns = queries: queries before the key are masked on the diagonal tile;
+                // queries past the prompt carry lse = +inf and contribute exp2(-inf) = 0
+                const float* lse = sm_lse[s];
+#pragma unroll
+                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld_32x32(acc + c0, v);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float pe = exp2f(__uint_as_float(v[c]) * p.scale_log2 - lse[c0 + c]);
+                        if (!(diagonal && row > c0 + c)) colsum += pe;
+                    }
+                }
+            }
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_acc_empty[s]));
+            if (PASS == kPassColumnSums) {
+                sm_lse[s ^ 1][e] = next_lse;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+        }
+        if (!ok) {
             sm_abort = 1;
-            continue;
+        } else if (PASS == kPassLse) {
+            const int t = blk * kTileRows + row;
+            if (t < p.T) p.lse2[(int64_t)head_res * p.T + t] = t < len ? m_run + log2f(l_run) : INFINITY;
+        } else {
+            const int t = blk * kTileRows + row;
+            if (t < p.T) p.score[(int64_t)head_res * p.T + t] = colsum;
         }
-        const uint32_t q_tile = base + (1 + (it & 1)) * kTileBytes;
-        const bool diagonal = (it % nq) == 0;
-        // S^T = K Q^T: rows are this warp's keys, columns the tile's 64 queries
-        float sacc[8][4];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) { sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.0f; }
-#pragma unroll
-        for (int ks = 0; ks < kKSteps; ++ks)
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                uint32_t qf[4];
-                ldmatrix_x4(q_tile + tile_offset(16 * kk + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), qf);
-                mma_bf16(sacc[2 * kk], ka[ks], qf[0], qf[1]);
-                mma_bf16(sacc[2 * kk + 1], ka[ks], qf[2], qf[3]);
-            }
-        const float* lse = sm_lse[it & 1];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int query = 8 * nt + qcol + (e & 1);          // inside the tile
-                const int key = r0 + qrow + (e >> 1) * 8;
-                float pe = exp2f(sacc[nt][e] * p.scale_log2 - lse[query]);   // lse = +inf past the prompt: 0
-                if (diagonal && key > query) pe = 0.0f;             // causal mask
-                colsum[e >> 1] += pe;
-            }
     }
+    tc::fence_before_sync();
     __syncthreads();
-    if (sm_abort) {
-        if (tid == 0) atomicOr(p.error, 1u);
-        return;
+    if (warp == 1) {
+        tc::fence_after_sync();
+        tc::tmem_dealloc(tmem_base, kTmemColumns);
     }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        float c = colsum[r];
-        c += __shfl_xor_sync(0xffffffffu, c, 1);
-        c += __shfl_xor_sync(0xffffffffu, c, 2);
-        const int t = kb * kRows + r0 + qrow + r * 8;
-        if ((lane & 3) == 0 && t < p.T) p.score[((int64_t)b * p.Hkv + kvh) * p.T + t] = c;
-    }
+    if (tid == 0 && sm_abort) atomicOr(p.error, 1u);
 }
 
 template <int D>
 cudaError_t launch_prefill(const PrefillParams& p, const CUtensorMap& qm, const CUtensorMap& km, cudaStream_t s) {
-    constexpr int kSmem = 3 * kRows * D * 2 + 1024;      // one resident tile + a two-stage ring
-    cudaError_t e = cudaFuncSetAttribute(prefill_lse_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    // at least 100 KB per CTA, so that never more than two CTAs (2 x 256 TMEM columns) share an SM
+    constexpr int kSmem = (3 * kTileRows * D * 2 + 1024) > 100 * 1024 ? (3 * kTileRows * D * 2 + 1024) : 100 * 1024;
+    cudaError_t e = cudaFuncSetAttribute(qk_pass_kernel<D, kPassLse>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_colsum_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    e = cudaFuncSetAttribute(qk_pass_kernel<D, kPassColumnSums>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    prefill_lse_kernel<D><<<dim3(p.n_blk, p.Hq, p.B), kThreads, kSmem, s>>>(p, qm, km);
+    qk_pass_kernel<D, kPassLse><<<dim3(p.n_blk, p.Hq, p.B), kThreads, kSmem, s>>>(p, qm, km);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    prefill_colsum_kernel<D><<<dim3(p.n_blk, p.Hkv, p.B), kThreads, kSmem, s>>>(p, qm, km);
+    qk_pass_kernel<D, kPassColumnSums><<<dim3(p.n_blk, p.Hkv, p.B), kThreads, kSmem, s>>>(p, qm, km);
     return cudaGetLastError();
 }
 
@@ -312,12 +278,12 @@ extern "C" __attribute__((visibility("default"))) int baklava_prefill_scores(
     p.lse2 = reinterpret_cast<float*>(static_cast<char*>(ws) + 256);
     p.score = score;
     p.B = B; p.T = T; p.Hq = shape->Hq; p.Hkv = shape->Hkv;
-    p.n_blk = (T + kRows - 1) / kRows;
+    p.n_blk = (T + kTileRows - 1) / kTileRows;
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
 
     CUtensorMap qm, km;
-    if (!make_head_map(&qm, q, (int64_t)B * shape->Hq, T, shape->D) ||
-        !make_head_map(&km, k, (int64_t)B * shape->Hkv, T, shape->D))
+    if (!make_head_map(&qm, q, (int64_t)B * shape->Hq, T, shape->D, kTileRows) ||
+        !make_head_map(&km, k, (int64_t)B * shape->Hkv, T, shape->D, kTileRows))
         return BAKLAVA_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 256, s) != cudaSuccess) return BAKLAVA_ERR_CUDA;
