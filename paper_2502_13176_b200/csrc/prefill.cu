@@ -5,10 +5,11 @@
 // Two passes over Q K^T (V is not needed), both on the 5th-generation tensor cores.  A CTA keeps one
 // 128-row operand tile resident in shared memory and streams the other operand's tiles through a
 // two-stage TMA ring; one thread issues tcgen05.mma into a double-buffered 128 x 128 fp32 accumulator in
-// tensor memory; four epilogue warps read it back with tcgen05.ld, one accumulator row per thread.
+// tensor memory; eight epilogue warps read it back with tcgen05.ld, one accumulator row per pair of threads.
 //   pass 1 (rows = queries): every query row's log-sum-exp, a running max / sum kept by its thread;
 //   pass 2 (rows = keys):    exp2(logit - lse[query]) summed along each key's row, again by its thread.
-// No reduction crosses a thread, so every sum has a fixed order and the result is reproducible.
+// The only reduction across threads joins the two halves of a row in a fixed order, so the result is
+// reproducible bit for bit.
 #include <cmath>
 #include <cstdint>
 
@@ -21,8 +22,8 @@ namespace {
 using namespace ptx;
 
 constexpr int kTileRows = 128;       // rows of an operand tile = accumulator rows = accumulator columns
-constexpr int kThreads = 192;        // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-5: epilogue
-constexpr int kEpilogueThreads = 128;
+constexpr int kThreads = 320;        // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-9: epilogue
+constexpr int kEpilogueThreads = 256; // two threads per accumulator row, 64 columns each
 constexpr uint32_t kTmemColumns = 256;   // two 128-column accumulators
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kPassLse = 0, kPassColumnSums = 1;
@@ -37,7 +38,7 @@ struct PrefillParams {
 };
 
 template <int D, int PASS>
-__global__ void __launch_bounds__(kThreads) qk_pass_kernel(const PrefillParams p,
+__global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParams p,
                                                            const __grid_constant__ CUtensorMap q_map,
                                                            const __grid_constant__ CUtensorMap k_map) {
     constexpr int kKSteps = D / 16;                         // one MMA covers 16 elements of the head dimension
@@ -148,85 +149,96 @@ __global__ void __launch_bounds__(kThreads) qk_pass_kernel(const PrefillParams p
             if (!ok) sm_abort = 1;
         }
     } else {
-        // ---------------- epilogue: thread = accumulator row (its warp's quarter of the TMEM lanes)
+        // ---------------- epilogue: a warp reads its quarter of the TMEM lanes (thread = accumulator row);
+        // warps 2-5 take columns 0..63 of every tile, warps 6-9 columns 64..127
         const int e = tid - 64;
         const int row = 32 * (warp & 3) + lane;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+        const int half = (warp - 2) >> 2;
+        const int col_base = half * (kTileRows / 2);
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + col_base;
         float m_run = -INFINITY, l_run = 0.0f, colsum = 0.0f;
         auto fetch_lse = [&](int it) -> float {              // the log-sum-exp of streamed query row e of tile it
             const int t = stream_blk(it) * kTileRows + e;
             return t < p.T ? p.lse2[(int64_t)stream_head(it) * p.T + t] : INFINITY;
         };
         if (PASS == kPassColumnSums) {
-            sm_lse[0][e] = fetch_lse(0);
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (e < kTileRows) sm_lse[0][e] = fetch_lse(0);
+            asm volatile("bar.sync 1, 256;" ::: "memory");
         }
         bool ok = true;
         for (int it = 0; it < n_it; ++it) {
             const int s = it & 1;
             float next_lse = 0.0f;
-            if (PASS == kPassColumnSums && it + 1 < n_it) next_lse = fetch_lse(it + 1);
+            if (PASS == kPassColumnSums && e < kTileRows && it + 1 < n_it) next_lse = fetch_lse(it + 1);
             if (!mbar_wait(smem_u32(&bar_acc_full[s]), (it >> 1) & 1)) { ok = false; break; }
             tc::fence_after_sync();
             const bool diagonal = stream_blk(it) == blk;
             const uint32_t acc = lane_addr + s * kTileRows;
             if (PASS == kPassLse) {
-                // row = query, columns = keys: keys above the query are masked on the diagonal tile
-                float mx = -INFINITY;
+                // row = query, columns = keys: keys above the query are masked on the diagonal tile.
+                // Online softmax statistics, 32 columns at a time.
 #pragma unroll
-                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
+                for (int c0 = 0; c0 < kTileRows / 2; c0 += 32) {
                     uint32_t v[32];
                     tc::tmem_ld_32x32(acc + c0, v);
                     tc::tmem_ld_wait();
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int c = 0; c < 32; ++c)
-                        if (!(diagonal && c0 + c > row)) mx = fmaxf(mx, __uint_as_float(v[c]));
-                }
-                const float m_new = fmaxf(m_run, mx * p.scale_log2);       // finite: key 0 is never masked
-                float sum = 0.0f;
+                        if (!(diagonal && col_base + c0 + c > row)) mx[c & 3] = fmaxf(mx[c & 3], __uint_as_float(v[c]));
+                    const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
+                    if (m_new != -INFINITY) {                 // (a diagonal tile's first rows see none of the upper columns)
+                        float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld_32x32(acc + c0, v);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (!(diagonal && c0 + c > row)) sum += exp2f(__uint_as_float(v[c]) * p.scale_log2 - m_new);
+                        for (int c = 0; c < 32; ++c)
+                            if (!(diagonal && col_base + c0 + c > row))
+                                sum[c & 3] += exp2f(__uint_as_float(v[c]) * p.scale_log2 - m_new);
+                        l_run = l_run * exp2f(m_run - m_new) + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
+                        m_run = m_new;
+                    }
                 }
-                l_run = l_run * exp2f(m_run - m_new) + sum;
-                m_run = m_new;
             } else {
                 // row = key, columns = queries: queries before the key are masked on the diagonal tile;
                 // queries past the prompt carry lse = +inf and contribute exp2(-inf) = 0
-                const float* lse = sm_lse[s];
+                const float* lse = sm_lse[s] + col_base;
+                uint32_t v0[32], v1[32];                     // this thread's 64 columns of the tile
+                tc::tmem_ld_32x32(acc, v0);
+                tc::tmem_ld_32x32(acc + 32, v1);
+                tc::tmem_ld_wait();
+                float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld_32x32(acc + c0, v);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float pe = exp2f(__uint_as_float(v[c]) * p.scale_log2 - lse[c0 + c]);
-                        if (!(diagonal && row > c0 + c)) colsum += pe;
-                    }
+                for (int c = 0; c < 32; ++c) {
+                    const float p0 = exp2f(__uint_as_float(v0[c]) * p.scale_log2 - lse[c]);
+                    const float p1 = exp2f(__uint_as_float(v1[c]) * p.scale_log2 - lse[32 + c]);
+                    if (!(diagonal && row > col_base + c)) sum[c & 3] += p0;
+                    if (!(diagonal && row > col_base + 32 + c)) sum[c & 3] += p1;
                 }
+                colsum += (sum[0] + sum[1]) + (sum[2] + sum[3]);
             }
             tc::fence_before_sync();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(smem_u32(&bar_acc_empty[s]));
             if (PASS == kPassColumnSums) {
-                sm_lse[s ^ 1][e] = next_lse;
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (e < kTileRows) sm_lse[s ^ 1][e] = next_lse;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
             }
         }
+        // join the two halves of every row: the upper half hands its state over through shared memory
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (half == 1) { sm_lse[0][row] = PASS == kPassLse ? m_run : colsum; sm_lse[1][row] = l_run; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (!ok) {
             sm_abort = 1;
-        } else if (PASS == kPassLse) {
+        } else if (half == 0) {
             const int t = blk * kTileRows + row;
-            if (t < p.T) p.lse2[(int64_t)head_res * p.T + t] = t < len ? m_run + log2f(l_run) : INFINITY;
-        } else {
-            const int t = blk * kTileRows + row;
-            if (t < p.T) p.score[(int64_t)head_res * p.T + t] = colsum;
+            if (PASS == kPassLse) {
+                const float m_hi = sm_lse[0][row], l_hi = sm_lse[1][row];
+                const float m_all = fmaxf(m_run, m_hi);      // m_run is finite: column 0 belongs to the lower half
+                const float l_all = l_run * exp2f(m_run - m_all) + (m_hi == -INFINITY ? 0.0f : l_hi * exp2f(m_hi - m_all));
+                if (t < p.T) p.lse2[(int64_t)head_res * p.T + t] = t < len ? m_all + log2f(l_all) : INFINITY;
+            } else {
+                if (t < p.T) p.score[(int64_t)head_res * p.T + t] = colsum + sm_lse[0][row];
+            }
         }
     }
     tc::fence_before_sync();
