@@ -28,6 +28,13 @@ constexpr uint32_t kTmemColumns = 256;   // two 128-column accumulators
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kPassLse = 0, kPassColumnSums = 1;
 
+// 2^x on the special-function unit (one instruction; -inf gives 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 struct PrefillParams {
     const int32_t* prompt_len;   // [B] or null
     float* lse2;                 // [B, Hq, T] log2-domain log-sum-exp of every query row (+inf past the prompt)
@@ -182,18 +189,21 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
                     uint32_t v[32];
                     tc::tmem_ld_32x32(acc + c0, v);
                     tc::tmem_ld_wait();
+                    if (diagonal) {                            // keys above the query do not exist for it
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (col_base + c0 + c > row) v[c] = 0xff800000u;    // -inf
+                    }
                     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (!(diagonal && col_base + c0 + c > row)) mx[c & 3] = fmaxf(mx[c & 3], __uint_as_float(v[c]));
+                    for (int c = 0; c < 32; ++c) mx[c & 3] = fmaxf(mx[c & 3], __uint_as_float(v[c]));
                     const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
                     if (m_new != -INFINITY) {                 // (a diagonal tile's first rows see none of the upper columns)
                         float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (!(diagonal && col_base + c0 + c > row))
-                                sum[c & 3] += exp2f(__uint_as_float(v[c]) * p.scale_log2 - m_new);
-                        l_run = l_run * exp2f(m_run - m_new) + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
+                            sum[c & 3] += fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -m_new));
+                        l_run = l_run * fast_exp2(m_run - m_new) + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
                         m_run = m_new;
                     }
                 }
@@ -205,13 +215,18 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
                 tc::tmem_ld_32x32(acc, v0);
                 tc::tmem_ld_32x32(acc + 32, v1);
                 tc::tmem_ld_wait();
+                if (diagonal) {                                // queries before the key do not see it
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        if (row > col_base + c) v0[c] = 0xff800000u;             // -inf
+                        if (row > col_base + 32 + c) v1[c] = 0xff800000u;
+                    }
+                }
                 float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
-                    const float p0 = exp2f(__uint_as_float(v0[c]) * p.scale_log2 - lse[c]);
-                    const float p1 = exp2f(__uint_as_float(v1[c]) * p.scale_log2 - lse[32 + c]);
-                    if (!(diagonal && row > col_base + c)) sum[c & 3] += p0;
-                    if (!(diagonal && row > col_base + 32 + c)) sum[c & 3] += p1;
+                    sum[c & 3] += fast_exp2(fmaf(__uint_as_float(v0[c]), p.scale_log2, -lse[c]));
+                    sum[(c + 2) & 3] += fast_exp2(fmaf(__uint_as_float(v1[c]), p.scale_log2, -lse[32 + c]));
                 }
                 colsum += (sum[0] + sum[1]) + (sum[2] + sum[3]);
             }
