@@ -265,21 +265,44 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
     if (tid == 0 && sm_abort) atomicOr(p.error, 1u);
 }
 
-template <int D>
-cudaError_t launch_prefill(const PrefillParams& p, const CUtensorMap& qm, const CUtensorMap& km, cudaStream_t s) {
+template <int D, int PASS>
+cudaError_t launch_pass(const PrefillParams& p, const CUtensorMap& qm, const CUtensorMap& km, dim3 grid, cudaStream_t s) {
     // at least 100 KB per CTA, so that never more than two CTAs (2 x 256 TMEM columns) share an SM
     constexpr int kSmem = (3 * kTileRows * D * 2 + 1024) > 100 * 1024 ? (3 * kTileRows * D * 2 + 1024) : 100 * 1024;
-    cudaError_t e = cudaFuncSetAttribute(qk_pass_kernel<D, kPassLse>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(qk_pass_kernel<D, PASS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(qk_pass_kernel<D, kPassColumnSums>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-    if (e != cudaSuccess) return e;
-    qk_pass_kernel<D, kPassLse><<<dim3(p.n_blk, p.Hq, p.B), kThreads, kSmem, s>>>(p, qm, km);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    qk_pass_kernel<D, kPassColumnSums><<<dim3(p.n_blk, p.Hkv, p.B), kThreads, kSmem, s>>>(p, qm, km);
+    qk_pass_kernel<D, PASS><<<grid, kThreads, kSmem, s>>>(p, qm, km);
     return cudaGetLastError();
 }
 
+template <int D>
+cudaError_t launch_prefill(const PrefillParams& p, const CUtensorMap& qm, const CUtensorMap& km, cudaStream_t s) {
+    cudaError_t e = launch_pass<D, kPassLse>(p, qm, km, dim3(p.n_blk, p.Hq, p.B), s);
+    if (e != cudaSuccess) return e;
+    return launch_pass<D, kPassColumnSums>(p, qm, km, dim3(p.n_blk, p.Hkv, p.B), s);
+}
+
 }  // namespace
+
+// Pass 1 alone, for the profiling kernel: log2-domain log-sum-exp of every causal query row.
+int baklava_launch_row_lse(const baklava_shape* shape, const void* q, const void* k, const int32_t* prompt_len,
+                           int32_t B, int32_t T, float* lse2, uint32_t* error, cudaStream_t s) {
+    PrefillParams p;
+    p.prompt_len = prompt_len;
+    p.error = error;
+    p.lse2 = lse2;
+    p.score = nullptr;
+    p.B = B; p.T = T; p.Hq = shape->Hq; p.Hkv = shape->Hkv;
+    p.n_blk = (T + kTileRows - 1) / kTileRows;
+    p.scale_log2 = kLog2e / sqrtf((float)shape->D);
+    CUtensorMap qm, km;
+    if (!make_head_map(&qm, q, (int64_t)B * shape->Hq, T, shape->D, kTileRows) ||
+        !make_head_map(&km, k, (int64_t)B * shape->Hkv, T, shape->D, kTileRows))
+        return BAKLAVA_ERR_CUDA;
+    cudaError_t e = shape->D == 128 ? launch_pass<128, kPassLse>(p, qm, km, dim3(p.n_blk, p.Hq, B), s)
+                                    : launch_pass<64, kPassLse>(p, qm, km, dim3(p.n_blk, p.Hq, B), s);
+    return e == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
+}
 
 extern "C" __attribute__((visibility("default"))) size_t baklava_prefill_workspace_size(const baklava_shape* shape,
                                                                                     int32_t B, int32_t T) {

@@ -2,286 +2,276 @@
 // causal softmax attention O = softmax(Q K^T / sqrt(D)) V and the token-wise cosine between the
 // head's input V_t and its output O_t, averaged over the prompt's tokens.
 //
-// One CTA owns 64 query rows of one (prompt, head): four warps of 16 rows each.  K and V tiles of
-// 64 keys are brought in by TMA (128-byte swizzle) into a two-stage ring; logits and P.V run on
-// the tensor cores (bf16 mma.sync, fp32 accumulate) with an online softmax.  O is never written:
-// the last key tile is the diagonal one, whose V rows are exactly the rows the cosine needs, so
-// the epilogue reads them from shared memory.  Per-CTA cosine sums go to the workspace and a
-// second kernel adds them in a fixed order (deterministic mean).
-#include <cuda.h>
-#include <cuda_bf16.h>
-#include <cuda_runtime.h>
-
+// Two launches on the 5th-generation tensor cores.  The first gives every query row its log-sum-exp
+// (the row pass of the prompt-score kernels).  The second owns 128 query rows per CTA: the Q tile stays
+// in shared memory, K and V tiles of 128 keys stream through a two-stage TMA ring; one thread issues
+// S = Q K^T into tensor memory (double-buffered), eight softmax warps read S back, form the already
+// normalised probabilities exp2(s - lse) in bf16 and store them as the next MMA's A operand in shared
+// memory, and the same thread issues O += P V with V as an MN-major B operand; O accumulates in tensor
+// memory over all key tiles and is never written.  The last key tile is the diagonal one, whose V rows
+// are exactly the rows the cosine needs, so the final epilogue reads them from shared memory.
+// Per-CTA cosine sums go to the workspace and a small kernel adds them in a fixed order.
 #include <cmath>
 #include <cstdint>
 
 #include "baklava.h"
 #include "common.h"
+#include "ptx.cuh"
 
 namespace {
 
-constexpr int kRows = 64;          // query rows per CTA = keys per tile
-constexpr int kThreads = 128;
-constexpr uint32_t kWaitLimit = 1u << 22;
+using namespace ptx;
+
+constexpr int kTileRows = 128;        // query rows per CTA = keys per streamed tile
+constexpr int kThreads = 320;         // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-9: softmax / epilogue
+constexpr int kSoftmaxWarps = 8;
+constexpr uint32_t kTmemColumns = 512;    // S: 2 x 128 columns, O: D columns
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kCosEps = 1e-12f;
 
 struct ProfileParams {
     const int32_t* prompt_len;   // [P] or null
+    const float* lse2;           // [P, Hq, T] from the row pass
     float* head_cos;             // [P, Hq]
     float* token_cos;            // [P, Hq, T] or null
-    float* block_sum;            // [P, Hq, n_qb]
-    uint32_t* error;             // one word in the workspace, set when a bounded wait gives up
-    int32_t P, T, Hq, Hkv, n_qb;
+    float* block_sum;            // [P, Hq, n_blk]
+    uint32_t* error;
+    int32_t P, T, Hq, Hkv, n_blk;
     float scale_log2;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* ptr) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-        "{%0, %1, %2, %3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
 }
-// 16-byte piece `piece` of row `row` in a [64][D] bf16 tile written by TMA with the 128-byte swizzle
-__device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
-    return (uint32_t)((piece >> 3) * (kRows * 128) + row * 128 + (((piece & 7) ^ (row & 7)) << 4));
-}
 
 template <int D>
-__global__ void __launch_bounds__(kThreads) profile_kernel(const ProfileParams p,
-                                                           const __grid_constant__ CUtensorMap q_map,
-                                                           const __grid_constant__ CUtensorMap k_map,
-                                                           const __grid_constant__ CUtensorMap v_map) {
-    constexpr int kKSteps = D / 16;
-    constexpr int kNTiles = D / 8;
-    constexpr int kTileBytes = kRows * D * 2;
-
+__global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfileParams p,
+                                                                 const __grid_constant__ CUtensorMap q_map,
+                                                                 const __grid_constant__ CUtensorMap k_map,
+                                                                 const __grid_constant__ CUtensorMap v_map) {
+    constexpr int kKSteps = D / 16;                          // MMA steps over the head dimension (S = Q K^T)
+    constexpr int kPvSteps = kTileRows / 16;                 // MMA steps over the keys (O += P V)
+    constexpr int kBoxBytes = kTileRows * 128;               // one TMA box: 128 rows x 64 elements
+    constexpr int kTileBytes = kTileRows * D * 2;            // a Q, K or V tile
+    constexpr int kPBytes = kTileRows * kTileRows * 2;       // a probability tile: 128 queries x 128 keys, bf16
+    constexpr int kStageBytes = 2 * kTileBytes;              // K then V
+    constexpr uint32_t kOColumn = 2 * kTileRows;             // O sits after the two S buffers in tensor memory
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q;
-    __shared__ __align__(8) uint64_t bar_kv[2];
-    __shared__ float sm_sum[kThreads / 32];
+    __shared__ __align__(8) uint64_t bar_q, bar_full[2], bar_empty[2], bar_s_full[2], bar_s_empty[2], bar_p_full[2],
+        bar_p_empty[2], bar_o_full;
+    __shared__ uint32_t tmem_slot;
+    __shared__ float sm_part[3][kTileRows];                  // upper half's (dot, |V|^2, |O|^2) per row
+    __shared__ float sm_warp_sum[kSoftmaxWarps];
     __shared__ int sm_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int qb = p.n_qb - 1 - blockIdx.x;               // long rows of the causal triangle first
+    const int qb = p.n_blk - 1 - blockIdx.x;                 // long rows of the causal triangle first
     const int h = blockIdx.y, pr = blockIdx.z;
     const int kvh = h / (p.Hq / p.Hkv);
     const int len = p.prompt_len ? min(max(p.prompt_len[pr], 0), p.T) : p.T;
-    float* out_sum = p.block_sum + ((int64_t)pr * p.Hq + h) * p.n_qb + qb;
-    if (qb * kRows >= len) {
+    float* out_sum = p.block_sum + ((int64_t)pr * p.Hq + h) * p.n_blk + qb;
+    if (qb * kTileRows >= len) {
         if (tid == 0) *out_sum = 0.0f;
         return;
     }
+    const int n_it = qb + 1;                                 // key tiles 0 .. qb
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t q_tile = base;
-    auto k_tile = [&](int s) { return base + kTileBytes + s * 2 * kTileBytes; };
-    auto v_tile = [&](int s) { return base + 2 * kTileBytes + s * 2 * kTileBytes; };
+    const uint32_t stage0 = base + kTileBytes;
+    const uint32_t p_tile0 = stage0 + 2 * kStageBytes;
 
     if (tid == 0) {
         mbar_init(smem_u32(&bar_q), 1);
-        mbar_init(smem_u32(&bar_kv[0]), 1);
-        mbar_init(smem_u32(&bar_kv[1]), 1);
+        mbar_init(smem_u32(&bar_o_full), 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+            mbar_init(smem_u32(&bar_s_full[s]), 1);
+            mbar_init(smem_u32(&bar_s_empty[s]), kSoftmaxWarps);
+            mbar_init(smem_u32(&bar_p_full[s]), kSoftmaxWarps);
+            mbar_init(smem_u32(&bar_p_empty[s]), 1);
+        }
         sm_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_mbar_init();
     }
+    if (warp == 1) {
+        tc::tmem_alloc(smem_u32(&tmem_slot), kTmemColumns);
+        tc::tmem_relinquish();
+    }
+    tc::fence_before_sync();
     __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
 
-    auto issue_kv = [&](int kb) {
-        const int s = kb & 1;
-        const uint32_t bar = smem_u32(&bar_kv[s]);
-        mbar_arrive_expect_tx(bar, 2 * kTileBytes);
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            mbar_arrive_expect_tx(smem_u32(&bar_q), kTileBytes);
 #pragma unroll
-        for (int bx = 0; bx < D / 64; ++bx) {
-            tma_load_3d(k_tile(s) + bx * (kRows * 128), &k_map, bx * 64, kb * kRows, pr * p.Hkv + kvh, bar);
-            tma_load_3d(v_tile(s) + bx * (kRows * 128), &v_map, bx * 64, kb * kRows, pr * p.Hkv + kvh, bar);
-        }
-    };
-    if (tid == 0) {
-        mbar_arrive_expect_tx(smem_u32(&bar_q), kTileBytes);
+            for (int bx = 0; bx < D / 64; ++bx)
+                tma_load_3d(q_tile + bx * kBoxBytes, &q_map, bx * 64, qb * kTileRows, pr * p.Hq + h, smem_u32(&bar_q));
+            for (int it = 0; it < n_it; ++it) {
+                const int s = it & 1;
+                if (it >= 2 && !mbar_wait(smem_u32(&bar_empty[s]), ((it >> 1) - 1) & 1)) { sm_abort = 1; break; }
+                const uint32_t bar = smem_u32(&bar_full[s]);
+                mbar_arrive_expect_tx(bar, kStageBytes);
 #pragma unroll
-        for (int bx = 0; bx < D / 64; ++bx)
-            tma_load_3d(q_tile + bx * (kRows * 128), &q_map, bx * 64, qb * kRows, pr * p.Hq + h, smem_u32(&bar_q));
-        issue_kv(0);
-    }
-
-    const int r0 = warp * 16;
-    const int lm = lane >> 3, li8 = lane & 7;
-    const int qrow = lane >> 2, qcol = (lane & 3) * 2;
-    bool alive = mbar_wait(smem_u32(&bar_q), 0);
-    uint32_t qa[kKSteps][4];
-    if (alive) {
-#pragma unroll
-        for (int ks = 0; ks < kKSteps; ++ks)
-            ldmatrix_x4(q_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * ks + (lm >> 1)), qa[ks]);
-    }
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
-    float o[kNTiles][4];
-#pragma unroll
-    for (int j = 0; j < kNTiles; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f; }
-
-    for (int kb = 0; kb <= qb; ++kb) {
-        __syncthreads();                                   // everyone is done with the stage kb + 1 will overwrite
-        if (sm_abort) break;
-        if (tid == 0 && kb + 1 <= qb) issue_kv(kb + 1);
-        const int s = kb & 1;
-        if (!alive || !mbar_wait(smem_u32(&bar_kv[s]), (kb >> 1) & 1)) {
-            alive = false;
-            sm_abort = 1;
-            continue;
-        }
-        float sacc[8][4];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) { sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.0f; }
-#pragma unroll
-        for (int ks = 0; ks < kKSteps; ++ks) {
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                uint32_t kf[4];
-                ldmatrix_x4(k_tile(s) + tile_offset(16 * kk + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kf);
-                mma_bf16(sacc[2 * kk], qa[ks], kf[0], kf[1]);
-                mma_bf16(sacc[2 * kk + 1], qa[ks], kf[2], kf[3]);
+                for (int bx = 0; bx < D / 64; ++bx) {
+                    tma_load_3d(stage0 + s * kStageBytes + bx * kBoxBytes, &k_map, bx * 64, it * kTileRows,
+                                pr * p.Hkv + kvh, bar);
+                    tma_load_3d(stage0 + s * kStageBytes + kTileBytes + bx * kBoxBytes, &v_map, bx * 64, it * kTileRows,
+                                pr * p.Hkv + kvh, bar);
+                }
             }
         }
-        const bool diagonal = kb == qb;
-        float mx[2] = {-INFINITY, -INFINITY};
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = tc::idesc_bf16_f32(kTileRows, kTileRows);      // S[128 q x 128 keys]
+            constexpr uint32_t idesc_o = tc::idesc_bf16_f32_b_mn(kTileRows, D);         // O[128 q x D]
+            bool ok = mbar_wait(smem_u32(&bar_q), 0);
+            auto issue_s = [&](int it) {                     // S_it = Q K_it^T into S buffer it & 1
+                const int s = it & 1;
+                if (!mbar_wait(smem_u32(&bar_full[s]), (it >> 1) & 1)) return false;
+                if (it >= 2 && !mbar_wait(smem_u32(&bar_s_empty[s]), ((it >> 1) - 1) & 1)) return false;
+                tc::fence_after_sync();
+                const uint32_t k_tile = stage0 + s * kStageBytes;
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
+                for (int ks = 0; ks < kKSteps; ++ks) {
+                    const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+                    tc::umma_bf16(tmem_base + s * kTileRows, tc::desc_k_major_sw128(q_tile + off),
+                                  tc::desc_k_major_sw128(k_tile + off), idesc_s, ks > 0);
+                }
+                tc::umma_commit(smem_u32(&bar_s_full[s]));
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int s = it & 1;
+                if (it + 1 < n_it) ok = issue_s(it + 1);     // the next tile's logits while this tile's softmax runs
+                if (ok) ok = mbar_wait(smem_u32(&bar_p_full[s]), (it >> 1) & 1);
+                if (!ok) break;
+                tc::fence_after_sync();
+                const uint32_t v_tile = stage0 + s * kStageBytes + kTileBytes;
+                const uint32_t p_tile = p_tile0 + s * kPBytes;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int key = 8 * nt + qcol + (e & 1);            // inside the tile
-                const int row = r0 + qrow + (e >> 1) * 8;
-                float v = sacc[nt][e] * p.scale_log2;
-                if (diagonal && key > row) v = -INFINITY;           // causal mask
-                sacc[nt][e] = v;
-                mx[e >> 1] = fmaxf(mx[e >> 1], v);
+                for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step
+                    const uint32_t p_off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+                    tc::umma_bf16(tmem_base + kOColumn, tc::desc_k_major_sw128(p_tile + p_off),
+                                  tc::desc_mn_major_sw128(v_tile + ks * 2048, kBoxBytes), idesc_o, (it > 0) || (ks > 0));
+                }
+                tc::umma_commit(smem_u32(&bar_empty[s]));    // K and V of this stage are consumed
+                tc::umma_commit(smem_u32(&bar_p_empty[s]));  // so is the probability tile
             }
-        float corr[2];
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-            const float m_new = fmaxf(m_run[r], mx[r]);             // finite: key 0 is never masked
-            corr[r] = exp2f(m_run[r] - m_new);
-            m_run[r] = m_new;
+            if (ok) tc::umma_commit(smem_u32(&bar_o_full));
+            else sm_abort = 1;
         }
-        float rs[2] = {0.0f, 0.0f};
+    } else {
+        // ---------------- softmax warps: thread = query row; warps 2-5 take keys 0..63 of a tile, 6-9 keys 64..127
+        const int row = 32 * (warp & 3) + lane;
+        const int half = (warp - 2) >> 2;
+        const int col_base = half * (kTileRows / 2);
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+        const int t = qb * kTileRows + row;
+        const float lse = t < p.T ? p.lse2[((int64_t)pr * p.Hq + h) * p.T + t] : INFINITY;   // +inf past the prompt
+        bool ok = true;
+        for (int it = 0; it < n_it; ++it) {
+            const int s = it & 1;
+            if (!mbar_wait(smem_u32(&bar_s_full[s]), (it >> 1) & 1)) { ok = false; break; }
+            if (it >= 2 && !mbar_wait(smem_u32(&bar_p_empty[s]), ((it >> 1) - 1) & 1)) { ok = false; break; }
+            tc::fence_after_sync();
+            uint32_t v0[32], v1[32];
+            tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base, v0);
+            tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base + 32, v1);
+            tc::tmem_ld_wait();
+            if (it == qb) {                                   // diagonal tile: keys above the query do not exist
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float pe = exp2f(sacc[nt][e] - m_run[e >> 1]);
-                sacc[nt][e] = pe;
-                rs[e >> 1] += pe;
+                for (int c = 0; c < 32; ++c) {
+                    if (col_base + c > row) v0[c] = 0xff800000u;
+                    if (col_base + 32 + c > row) v1[c] = 0xff800000u;
+                }
             }
-        l_run[0] = l_run[0] * corr[0] + rs[0];
-        l_run[1] = l_run[1] * corr[1] + rs[1];
+            // probabilities of this thread's 64 keys -> bf16 -> the K-major, 128-byte-swizzled A tile
+            uint8_t* p_row = base_ptr + (p_tile0 - base) + s * kPBytes + half * kBoxBytes + row * 128;
 #pragma unroll
-        for (int j = 0; j < kNTiles; ++j) {
-            o[j][0] *= corr[0]; o[j][1] *= corr[0];
-            o[j][2] *= corr[1]; o[j][3] *= corr[1];
-        }
+            for (int cc = 0; cc < 8; ++cc) {                  // 16-byte pieces of 8 keys
+                uint32_t w[4];
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-            uint32_t pa[4];
-            pa[0] = pack_bf16(sacc[2 * kk][0], sacc[2 * kk][1]);
-            pa[1] = pack_bf16(sacc[2 * kk][2], sacc[2 * kk][3]);
-            pa[2] = pack_bf16(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1]);
-            pa[3] = pack_bf16(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3]);
-#pragma unroll
-            for (int j2 = 0; j2 < kNTiles / 2; ++j2) {
-                uint32_t vf[4];
-                ldmatrix_x4_trans(v_tile(s) + tile_offset(16 * kk + (lm & 1) * 8 + li8, 2 * j2 + (lm >> 1)), vf);
-                mma_bf16(o[2 * j2], pa, vf[0], vf[1]);
-                mma_bf16(o[2 * j2 + 1], pa, vf[2], vf[3]);
+                for (int k2 = 0; k2 < 4; ++k2) {
+                    const int c = cc * 8 + k2 * 2;
+                    const uint32_t a = c < 32 ? v0[c] : v1[c - 32], bq = c + 1 < 32 ? v0[c + 1] : v1[c + 1 - 32];
+                    w[k2] = pack_bf16(fast_exp2(fmaf(__uint_as_float(a), p.scale_log2, -lse)),
+                                      fast_exp2(fmaf(__uint_as_float(bq), p.scale_log2, -lse)));
+                }
+                *reinterpret_cast<uint4*>(p_row + ((cc ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            tc::fence_proxy_async_smem();
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                tc::mbar_arrive(smem_u32(&bar_p_full[s]));
+                tc::mbar_arrive(smem_u32(&bar_s_empty[s]));
             }
         }
-    }
-    __syncthreads();
-    if (sm_abort) {
-        if (tid == 0) { atomicOr(p.error, 1u); *out_sum = 0.0f; }
-        return;
-    }
-
-    // ---- cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile (stage qb & 1)
-    const uint8_t* v_rows = base_ptr + 2 * kTileBytes + (qb & 1) * 2 * kTileBytes;
-    float my_sum = 0.0f;
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        const int row = r0 + qrow + r * 8;
+        // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile
+        if (ok) ok = mbar_wait(smem_u32(&bar_o_full), 0);
         float dot = 0.0f, vv = 0.0f, oo = 0.0f;
+        if (ok) {
+            tc::fence_after_sync();
+            constexpr int kCols = D / 2;                      // this thread's share of the head dimension
+            const uint8_t* v_row = base_ptr + (stage0 - base) + (qb & 1) * kStageBytes + kTileBytes + row * 128;
 #pragma unroll
-        for (int j = 0; j < kNTiles; ++j) {
-            const uint32_t raw = *reinterpret_cast<const uint32_t*>(v_rows + tile_offset(row, j) + qcol * 2);
-            const float2 vx = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw));
-            const float o0 = o[j][2 * r], o1 = o[j][2 * r + 1];
-            dot = fmaf(vx.x, o0, fmaf(vx.y, o1, dot));
-            vv = fmaf(vx.x, vx.x, fmaf(vx.y, vx.y, vv));
-            oo = fmaf(o0, o0, fmaf(o1, o1, oo));
-        }
+            for (int c0 = 0; c0 < kCols; c0 += 32) {
+                uint32_t o[32];
+                tc::tmem_ld_32x32(lane_addr + kOColumn + half * kCols + c0, o);
+                tc::tmem_ld_wait();
 #pragma unroll
-        for (int off = 1; off <= 2; off <<= 1) {
-            dot += __shfl_xor_sync(0xffffffffu, dot, off);
-            vv += __shfl_xor_sync(0xffffffffu, vv, off);
-            oo += __shfl_xor_sync(0xffffffffu, oo, off);
+                for (int cc = 0; cc < 4; ++cc) {              // 16-byte pieces of 8 elements
+                    const int piece = (half * kCols + c0) / 8 + cc;             // within the row: 0 .. D/8 - 1
+                    const uint4 raw = *reinterpret_cast<const uint4*>(v_row + (piece >> 3) * kBoxBytes +
+                                                                      (((piece & 7) ^ (row & 7)) << 4));
+                    const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int k2 = 0; k2 < 4; ++k2) {
+                        const float2 vx = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[k2]));
+                        const float o0 = __uint_as_float(o[cc * 8 + k2 * 2]), o1 = __uint_as_float(o[cc * 8 + k2 * 2 + 1]);
+                        dot = fmaf(vx.x, o0, fmaf(vx.y, o1, dot));
+                        vv = fmaf(vx.x, vx.x, fmaf(vx.y, vx.y, vv));
+                        oo = fmaf(o0, o0, fmaf(o1, o1, oo));
+                    }
+                }
+            }
         }
-        // O here is unnormalised (missing 1 / l): the cosine does not depend on a positive scale,
-        // except through the floor on the denominator, so apply 1 / l to the norm product
-        float lr = l_run[r];
-        lr += __shfl_xor_sync(0xffffffffu, lr, 1);
-        lr += __shfl_xor_sync(0xffffffffu, lr, 2);
-        const float inv_l = 1.0f / lr;
-        const float c = (dot * inv_l) / fmaxf(sqrtf(vv) * sqrtf(oo) * inv_l, kCosEps);
-        const int t = qb * kRows + row;
-        if (t < len && (lane & 3) == 0) {
-            my_sum += c;
+        if (half == 1) { sm_part[0][row] = dot; sm_part[1][row] = vv; sm_part[2][row] = oo; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        float c = 0.0f;
+        if (half == 0 && ok && t < len) {
+            dot += sm_part[0][row]; vv += sm_part[1][row]; oo += sm_part[2][row];
+            c = dot / fmaxf(sqrtf(vv) * sqrtf(oo), kCosEps);
             if (p.token_cos) p.token_cos[((int64_t)pr * p.Hq + h) * p.T + t] = c;
         }
-    }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) my_sum += __shfl_xor_sync(0xffffffffu, my_sum, off);
-    if (lane == 0) sm_sum[warp] = my_sum;
+        for (int off = 16; off > 0; off >>= 1) c += __shfl_xor_sync(0xffffffffu, c, off);
+        if (lane == 0) sm_warp_sum[warp - 2] = c;
+        if (!ok) sm_abort = 1;
+    }
+    tc::fence_before_sync();
     __syncthreads();
-    if (tid == 0) *out_sum = (sm_sum[0] + sm_sum[1]) + (sm_sum[2] + sm_sum[3]);
+    if (warp == 1) {
+        tc::fence_after_sync();
+        tc::tmem_dealloc(tmem_base, kTmemColumns);
+    }
+    if (tid == 0) {
+        if (sm_abort) atomicOr(p.error, 1u);
+        *out_sum = sm_abort ? 0.0f : (sm_warp_sum[0] + sm_warp_sum[1]) + (sm_warp_sum[2] + sm_warp_sum[3]);
+    }
 }
 
 __global__ void profile_mean_kernel(const ProfileParams p) {
@@ -290,42 +280,19 @@ __global__ void profile_mean_kernel(const ProfileParams p) {
     const int pr = i / p.Hq;
     const int len = p.prompt_len ? min(max(p.prompt_len[pr], 0), p.T) : p.T;
     float acc = 0.0f;
-    for (int b = 0; b < p.n_qb; ++b) acc += p.block_sum[(int64_t)i * p.n_qb + b];
+    for (int b = 0; b < p.n_blk; ++b) acc += p.block_sum[(int64_t)i * p.n_blk + b];
     p.head_cos[i] = len > 0 ? acc / (float)len : 0.0f;
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// bf16 [heads, T, D]: boxes of 64 tokens x 64 elements of one head, 128-byte swizzle, zero fill past T
-bool make_map(CUtensorMap* map, const void* base, int64_t heads, int T, int D) {
-    static EncodeTiledFn enc = nullptr;
-    if (!enc) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult res;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
-            res != cudaDriverEntryPointSuccess)
-            return false;
-        enc = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)heads};
-    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
-    const cuuint32_t box[3] = {64, (cuuint32_t)kRows, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int D>
 cudaError_t launch_profile(const ProfileParams& p, const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
                            cudaStream_t s) {
-    constexpr int kSmem = 5 * kRows * D * 2 + 1024;      // Q tile + two (K, V) stages
-    cudaError_t e = cudaFuncSetAttribute(profile_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    // Q tile, two (K, V) stages, two probability tiles
+    constexpr int kSmem = kTileRows * D * 2 * 5 + 2 * kTileRows * kTileRows * 2 + 1024;
+    cudaError_t e = cudaFuncSetAttribute(profile_pv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    const dim3 grid(p.n_qb, p.Hq, p.P);
-    profile_kernel<D><<<grid, kThreads, kSmem, s>>>(p, qm, km, vm);
+    const dim3 grid(p.n_blk, p.Hq, p.P);
+    profile_pv_kernel<D><<<grid, kThreads, kSmem, s>>>(p, qm, km, vm);
     return cudaGetLastError();
 }
 
@@ -334,8 +301,8 @@ cudaError_t launch_profile(const ProfileParams& p, const CUtensorMap& qm, const 
 extern "C" __attribute__((visibility("default"))) size_t baklava_profile_workspace_size(const baklava_shape* shape,
                                                                                     int32_t P, int32_t T) {
     if (!shape || P <= 0 || T <= 0) return 0;
-    const size_t n_qb = ((size_t)T + kRows - 1) / kRows;
-    return 256 + sizeof(float) * (size_t)P * shape->Hq * n_qb;
+    const size_t n_blk = ((size_t)T + kTileRows - 1) / kTileRows;
+    return 256 + sizeof(float) * (size_t)P * shape->Hq * ((size_t)T + n_blk);
 }
 
 extern "C" __attribute__((visibility("default"))) int baklava_profile_heads(
@@ -356,19 +323,23 @@ extern "C" __attribute__((visibility("default"))) int baklava_profile_heads(
     p.head_cos = head_cos;
     p.token_cos = token_cos;
     p.error = static_cast<uint32_t*>(ws);
-    p.block_sum = reinterpret_cast<float*>(static_cast<char*>(ws) + 256);
+    float* lse2 = reinterpret_cast<float*>(static_cast<char*>(ws) + 256);
+    p.lse2 = lse2;
+    p.block_sum = lse2 + (size_t)P * shape->Hq * (size_t)T;
     p.P = P; p.T = T; p.Hq = shape->Hq; p.Hkv = shape->Hkv;
-    p.n_qb = (T + kRows - 1) / kRows;
+    p.n_blk = (T + kTileRows - 1) / kTileRows;
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
 
     CUtensorMap qm, km, vm;
-    if (!make_map(&qm, q, (int64_t)P * shape->Hq, T, shape->D) ||
-        !make_map(&km, k, (int64_t)P * shape->Hkv, T, shape->D) ||
-        !make_map(&vm, v, (int64_t)P * shape->Hkv, T, shape->D))
+    if (!make_head_map(&qm, q, (int64_t)P * shape->Hq, T, shape->D, kTileRows) ||
+        !make_head_map(&km, k, (int64_t)P * shape->Hkv, T, shape->D, kTileRows) ||
+        !make_head_map(&vm, v, (int64_t)P * shape->Hkv, T, shape->D, kTileRows))
         return BAKLAVA_ERR_CUDA;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 256, s) != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    rc = baklava_launch_row_lse(shape, q, k, prompt_len, P, T, lse2, p.error, s);
+    if (rc) return rc;
     cudaError_t err = shape->D == 128 ? launch_profile<128>(p, qm, km, vm, s) : launch_profile<64>(p, qm, km, vm, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     const int n = P * shape->Hq;

@@ -149,3 +149,25 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 
 }  // namespace tc
+
+namespace tc {
+
+// Descriptor of an MN-major bf16 operand (rows of the tile are the K index, 64 contiguous elements of
+// the M/N index per 128-byte row, 128-byte swizzle): 8-row groups along K are 1024 bytes apart, the
+// next 64 elements of M/N start `mn_group_bytes` further on.
+__device__ __forceinline__ uint64_t desc_mn_major_sw128(uint32_t smem_addr, uint32_t mn_group_bytes) {
+    uint64_t d = (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((mn_group_bytes >> 4) & 0x3FFFu) << 16;   // leading byte offset: between 64-element M/N groups
+    d |= (uint64_t)(1024 >> 4) << 32;                         // stride byte offset: between 8-row K groups
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// bf16 x bf16 -> fp32 with A K-major and B MN-major
+__host__ __device__ constexpr uint32_t idesc_bf16_f32_b_mn(int M, int N) {
+    return idesc_bf16_f32(M, N) | (1u << 16);
+}
+// makes this thread's shared-memory writes visible to the tensor core / TMA (async proxy)
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+}  // namespace tc
