@@ -217,7 +217,7 @@ def run_profile_pass(args):
                       "config": {"workload": "profile-llama3-8b", "prompts": P, "prompt_tokens": T, "heads": w.Hq,
                                  "kv_heads": w.Hkv, "head_dim": w.D},
                       "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s",
-                                   "frac": tf / peak, "traffic": None, "kernel": "profile_kernel (mma.sync path)"},
+                                   "frac": tf / peak, "traffic": None, "kernel": "qk_pass_kernel + profile_pv_kernel (tcgen05)"},
                       "gpu_launches": 2 * args.steps, "clocks": clocks.summary(t_open, t_close)}))
 
 

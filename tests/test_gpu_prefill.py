@@ -46,6 +46,11 @@ def test_llama_head_shape_with_prompt_lengths_and_peaked_attention():
     _run(B=3, Hq=8, Hkv=2, T=300, D=128, lens=[300, 129, 1], q_scale=3.0)
 
 
+def test_many_tiles_wrap_the_rings():
+    _run(B=1, Hq=2, Hkv=1, T=1200, D=128, lens=[1170])
+    _run(B=1, Hq=2, Hkv=2, T=900, D=64)
+
+
 def test_group_of_seven():
     _run(B=1, Hq=7, Hkv=1, T=150, D=128)
 

@@ -48,6 +48,12 @@ def test_llama_head_shape_and_prompt_lengths():
     _run(P=3, Hq=8, Hkv=2, T=300, D=128, lens=[300, 129, 1])
 
 
+def test_many_key_tiles_wrap_the_rings():
+    # ten 128-key tiles per row block: every stage, accumulator and probability buffer is reused several times
+    _run(P=1, Hq=2, Hkv=1, T=1200, D=128, want_tokens=True, lens=[1170])
+    _run(P=1, Hq=2, Hkv=2, T=900, D=64, want_tokens=False)
+
+
 def test_group_of_seven():
     _run(P=1, Hq=7, Hkv=1, T=150, D=128, want_tokens=False)
 
