@@ -5,7 +5,7 @@
 // Two launches on the 5th-generation tensor cores.  The first gives every query row its log-sum-exp
 // (the row pass of the prompt-score kernels).  The second owns 128 query rows per CTA: the Q tile stays
 // in shared memory, K and V tiles of 128 keys stream through a two-stage TMA ring; one thread issues
-// S = Q K^T into tensor memory (double-buffered), eight softmax warps read S back, form the already
+// S = Q K^T into tensor memory (double-buffered), sixteen softmax warps read S back, form the already
 // normalised probabilities exp2(s - lse) in bf16 and store them as the next MMA's A operand in shared
 // memory, and the same thread issues O += P V with V as an MN-major B operand; O accumulates in tensor
 // memory over all key tiles and is never written.  The last key tile is the diagonal one, whose V rows
@@ -23,8 +23,8 @@ namespace {
 using namespace ptx;
 
 constexpr int kTileRows = 128;        // query rows per CTA = keys per streamed tile
-constexpr int kThreads = 320;         // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-9: softmax / epilogue
-constexpr int kSoftmaxWarps = 8;
+constexpr int kSoftmaxWarps = 16;     // four threads per query row, 32 keys of a tile each
+constexpr int kThreads = (2 + kSoftmaxWarps) * 32;   // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, then softmax
 constexpr uint32_t kTmemColumns = 512;    // S: 2 x 128 columns, O: D columns
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kCosEps = 1e-12f;
@@ -66,7 +66,6 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     __shared__ __align__(8) uint64_t bar_q, bar_full[2], bar_empty[2], bar_s_full[2], bar_s_empty[2], bar_p_full[2],
         bar_p_empty[2], bar_o_full;
     __shared__ uint32_t tmem_slot;
-    __shared__ float sm_part[3][kTileRows];                  // upper half's (dot, |V|^2, |O|^2) per row
     __shared__ float sm_warp_sum[kSoftmaxWarps];
     __shared__ int sm_abort;
 
@@ -174,10 +173,11 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
             else sm_abort = 1;
         }
     } else {
-        // ---------------- softmax warps: thread = query row; warps 2-5 take keys 0..63 of a tile, 6-9 keys 64..127
+        // ---------------- softmax warps: a warp reads its quarter of the TMEM lanes (thread = query row);
+        // warps 2-5 take keys 0..31 of every tile, warps 6-9 keys 32..63, and so on
         const int row = 32 * (warp & 3) + lane;
-        const int half = (warp - 2) >> 2;
-        const int col_base = half * (kTileRows / 2);
+        const int part = (warp - 2) >> 2;                     // 0 .. 3
+        const int col_base = part * 32;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
         const int t = qb * kTileRows + row;
         const float lse = t < p.T ? p.lse2[((int64_t)pr * p.Hq + h) * p.T + t] : INFINITY;   // +inf past the prompt
@@ -187,30 +187,27 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
             if (!mbar_wait(smem_u32(&bar_s_full[s]), (it >> 1) & 1)) { ok = false; break; }
             if (it >= 2 && !mbar_wait(smem_u32(&bar_p_empty[s]), ((it >> 1) - 1) & 1)) { ok = false; break; }
             tc::fence_after_sync();
-            uint32_t v0[32], v1[32];
-            tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base, v0);
-            tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base + 32, v1);
+            uint32_t v[32];
+            tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base, v);
             tc::tmem_ld_wait();
             if (it == qb) {                                   // diagonal tile: keys above the query do not exist
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    if (col_base + c > row) v0[c] = 0xff800000u;
-                    if (col_base + 32 + c > row) v1[c] = 0xff800000u;
-                }
+                for (int c = 0; c < 32; ++c)
+                    if (col_base + c > row) v[c] = 0xff800000u;
             }
-            // probabilities of this thread's 64 keys -> bf16 -> the K-major, 128-byte-swizzled A tile
-            uint8_t* p_row = base_ptr + (p_tile0 - base) + s * kPBytes + half * kBoxBytes + row * 128;
+            // probabilities of this thread's 32 keys -> bf16 -> the K-major, 128-byte-swizzled A tile
+            uint8_t* p_row = base_ptr + (p_tile0 - base) + s * kPBytes + (part >> 1) * kBoxBytes + row * 128;
 #pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {                  // 16-byte pieces of 8 keys
+            for (int cc = 0; cc < 4; ++cc) {                  // 16-byte pieces of 8 keys
                 uint32_t w[4];
 #pragma unroll
                 for (int k2 = 0; k2 < 4; ++k2) {
                     const int c = cc * 8 + k2 * 2;
-                    const uint32_t a = c < 32 ? v0[c] : v1[c - 32], bq = c + 1 < 32 ? v0[c + 1] : v1[c + 1 - 32];
-                    w[k2] = pack_bf16(fast_exp2(fmaf(__uint_as_float(a), p.scale_log2, -lse)),
-                                      fast_exp2(fmaf(__uint_as_float(bq), p.scale_log2, -lse)));
+                    w[k2] = pack_bf16(fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -lse)),
+                                      fast_exp2(fmaf(__uint_as_float(v[c + 1]), p.scale_log2, -lse)));
                 }
-                *reinterpret_cast<uint4*>(p_row + ((cc ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                const int piece = (part & 1) * 4 + cc;        // inside the 64-key box
+                *reinterpret_cast<uint4*>(p_row + ((piece ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
             tc::fence_proxy_async_smem();
             tc::fence_before_sync();
@@ -220,41 +217,48 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                 tc::mbar_arrive(smem_u32(&bar_s_empty[s]));
             }
         }
-        // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile
+        // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile.
+        // Four threads per row take 32 columns of the head dimension each (two of them when D = 64).
         if (ok) ok = mbar_wait(smem_u32(&bar_o_full), 0);
         float dot = 0.0f, vv = 0.0f, oo = 0.0f;
-        if (ok) {
+        if (ok && part * 32 < D) {
             tc::fence_after_sync();
-            constexpr int kCols = D / 2;                      // this thread's share of the head dimension
             const uint8_t* v_row = base_ptr + (stage0 - base) + (qb & 1) * kStageBytes + kTileBytes + row * 128;
+            uint32_t o[32];
+            tc::tmem_ld_32x32(lane_addr + kOColumn + part * 32, o);
+            tc::tmem_ld_wait();
 #pragma unroll
-            for (int c0 = 0; c0 < kCols; c0 += 32) {
-                uint32_t o[32];
-                tc::tmem_ld_32x32(lane_addr + kOColumn + half * kCols + c0, o);
-                tc::tmem_ld_wait();
+            for (int cc = 0; cc < 4; ++cc) {                  // 16-byte pieces of 8 elements
+                const int piece = part * 4 + cc;              // within the row: 0 .. D/8 - 1
+                const uint4 raw = *reinterpret_cast<const uint4*>(v_row + (piece >> 3) * kBoxBytes +
+                                                                  (((piece & 7) ^ (row & 7)) << 4));
+                const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {              // 16-byte pieces of 8 elements
-                    const int piece = (half * kCols + c0) / 8 + cc;             // within the row: 0 .. D/8 - 1
-                    const uint4 raw = *reinterpret_cast<const uint4*>(v_row + (piece >> 3) * kBoxBytes +
-                                                                      (((piece & 7) ^ (row & 7)) << 4));
-                    const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                    for (int k2 = 0; k2 < 4; ++k2) {
-                        const float2 vx = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[k2]));
-                        const float o0 = __uint_as_float(o[cc * 8 + k2 * 2]), o1 = __uint_as_float(o[cc * 8 + k2 * 2 + 1]);
-                        dot = fmaf(vx.x, o0, fmaf(vx.y, o1, dot));
-                        vv = fmaf(vx.x, vx.x, fmaf(vx.y, vx.y, vv));
-                        oo = fmaf(o0, o0, fmaf(o1, o1, oo));
-                    }
+                for (int k2 = 0; k2 < 4; ++k2) {
+                    const float2 vx = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[k2]));
+                    const float o0 = __uint_as_float(o[cc * 8 + k2 * 2]), o1 = __uint_as_float(o[cc * 8 + k2 * 2 + 1]);
+                    dot = fmaf(vx.x, o0, fmaf(vx.y, o1, dot));
+                    vv = fmaf(vx.x, vx.x, fmaf(vx.y, vx.y, vv));
+                    oo = fmaf(o0, o0, fmaf(o1, o1, oo));
                 }
             }
         }
-        if (half == 1) { sm_part[0][row] = dot; sm_part[1][row] = vv; sm_part[2][row] = oo; }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // join the four parts of every row through shared memory (the probability tiles are idle now)
+        float* sm_part = reinterpret_cast<float*>(base_ptr + (p_tile0 - base));      // [3][4][128]
+        sm_part[(0 * 4 + part) * kTileRows + row] = dot;
+        sm_part[(1 * 4 + part) * kTileRows + row] = vv;
+        sm_part[(2 * 4 + part) * kTileRows + row] = oo;
+        asm volatile("bar.sync 1, 512;" ::: "memory");
         float c = 0.0f;
-        if (half == 0 && ok && t < len) {
-            dot += sm_part[0][row]; vv += sm_part[1][row]; oo += sm_part[2][row];
-            c = dot / fmaxf(sqrtf(vv) * sqrtf(oo), kCosEps);
+        if (part == 0 && ok && t < len) {
+            float d4 = 0.0f, v4 = 0.0f, o4 = 0.0f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                d4 += sm_part[(0 * 4 + k) * kTileRows + row];
+                v4 += sm_part[(1 * 4 + k) * kTileRows + row];
+                o4 += sm_part[(2 * 4 + k) * kTileRows + row];
+            }
+            c = d4 / fmaxf(sqrtf(v4) * sqrtf(o4), kCosEps);
             if (p.token_cos) p.token_cos[((int64_t)pr * p.Hq + h) * p.T + t] = c;
         }
 #pragma unroll
