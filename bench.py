@@ -104,74 +104,95 @@ def whole_job_rate(world, units_per_rank_step, steps, elapsed_ms):
     return world * units_per_rank_step * steps / (elapsed_ms * 1e-3)
 
 
-def oracle_sample(w, seconds_target=15.0):
+class OracleSample:
+    """A bounded sample of the workload for the CPU oracle: a few heads with their full retained caches, built
+    once from the seeded generator; `step()` runs one oracle decode step (append, attention, score update,
+    eviction) over all of them, one thread per head, and returns the K+V bytes it attended."""
+
+    def __init__(self, w):
+        import threadpoolctl
+
+        from oracle import allocation as oalloc
+        from oracle.cache import HeadCache
+        from paper_2502_13176_b200 import synth
+
+        self.w = w
+        imp = wl.importance(w).numpy()
+        cap, _, _ = oalloc.allocate(imp, w.t, w.r_num, w.r_den, w.total_pages, w.min_pages, w.max_pages, w.page)
+        self.cores = os.cpu_count() or 1
+        self.n_heads = min(w.L * w.Hkv * w.B, max(self.cores, 16))
+        picks = [(i * (w.L * w.Hkv) // self.n_heads) for i in range(self.n_heads)]
+        gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+        self.twins = []
+        for j, flat in enumerate(picks):
+            l, h = divmod(flat, w.Hkv)
+            C = int(cap[l, h]); n = C - 1
+            K = synth.normal_bf16(w.seed, 40, (n, w.D), gen_dev, None, j << 24).double().cpu().numpy()
+            V = synth.normal_bf16(w.seed, 41, (n, w.D), gen_dev, None, j << 24).double().cpu().numpy()
+            sc = synth.uniform_f64(w.seed, 42, j << 20, n).numpy()
+            hc = HeadCache(C, w.D, w.n_sink, w.recent_num, w.recent_den)
+            hc.load(K, V, np.arange(n), sc)
+            self.twins.append(hc)
+        self.steps_done = 0
+        self.limits = threadpoolctl.threadpool_limits
+
+    def describe(self, steps):
+        return "%d of %d heads x %d decode steps (fp64 numpy, one thread per head)" % (
+            self.n_heads, self.w.L * self.w.Hkv * self.w.B, steps)
+
+    def step(self):
+        from concurrent.futures import ThreadPoolExecutor
+
+        from paper_2502_13176_b200 import synth
+        w, s = self.w, self.steps_done
+        feeds = [synth.normal_bf16(w.seed, 43, (w.g + 2, w.D), "cpu", None, (s * self.n_heads + j) * 4096).double().numpy()
+                 for j in range(self.n_heads)]
+
+        def one(args):
+            hc, feed = args
+            hc.step(feed[:w.g], feed[w.g], feed[w.g + 1], w.T + s)
+            return hc.C * w.D * 4
+
+        t0 = time.perf_counter()
+        with self.limits(limits=1):
+            with ThreadPoolExecutor(max_workers=self.cores) as pool:
+                nbytes = sum(pool.map(one, zip(self.twins, feeds)))
+        self.steps_done += 1
+        return nbytes, time.perf_counter() - t0
+
+
+def oracle_sample(w, seconds_target=12.0, max_steps=32):
     """Time the CPU oracle's decode step on sampled heads of the workload.  Returns a cpu_baseline dict."""
-    from concurrent.futures import ThreadPoolExecutor
-
-    import threadpoolctl
-
-    from oracle import allocation as oalloc
-    from oracle.cache import HeadCache
-    from paper_2502_13176_b200 import synth
-
-    imp = wl.importance(w).numpy()
-    cap, _, _ = oalloc.allocate(imp, w.t, w.r_num, w.r_den, w.total_pages, w.min_pages, w.max_pages, w.page)
-    cores = os.cpu_count() or 1
-    n_heads = min(w.L * w.Hkv * w.B, max(cores, 16))
-    rng_heads = [(i * (w.L * w.Hkv) // n_heads) for i in range(n_heads)]
-    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
-    twins, feeds = [], []
-    for j, flat in enumerate(rng_heads):
-        l, h = divmod(flat, w.Hkv)
-        C = int(cap[l, h]); n = C - 1
-        K = synth.normal_bf16(w.seed, 40, (n, w.D), gen_dev, None, j * 1 << 24).double().cpu().numpy()
-        V = synth.normal_bf16(w.seed, 41, (n, w.D), gen_dev, None, j * 1 << 24).double().cpu().numpy()
-        sc = synth.uniform_f64(w.seed, 42, j * 1 << 20, n).numpy()
-        hc = HeadCache(C, w.D, w.n_sink, w.recent_num, w.recent_den)
-        hc.load(K, V, np.arange(n), sc)
-        twins.append(hc)
-        feeds.append([synth.normal_bf16(w.seed, 43 + i, (w.g + 2, w.D), "cpu", None, j * 4096).double().numpy()
-                      for i in range(3)])
-
-    def one(args):
-        hc, feed, s = args
-        hc.step(feed[:w.g], feed[w.g], feed[w.g + 1], w.T + s)
-        return hc.C * w.D * 4
-
-    total_bytes, steps_done = 0, 0
-    t0 = time.perf_counter()
-    with threadpoolctl.threadpool_limits(limits=1):
-        with ThreadPoolExecutor(max_workers=cores) as pool:
-            while steps_done < 3:
-                total_bytes += sum(pool.map(one, [(hc, f[steps_done], steps_done) for hc, f in zip(twins, feeds)]))
-                steps_done += 1
-                if time.perf_counter() - t0 > seconds_target:
-                    break
-    dt = time.perf_counter() - t0
-    return {"value": total_bytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-            "sample": "%d of %d heads x %d decode steps (fp64 numpy, one thread per head)" % (
-                n_heads, w.L * w.Hkv * w.B, steps_done), "seconds": dt}
+    sample = OracleSample(w)
+    total_bytes, total_s, steps = 0, 0.0, 0
+    while steps < max_steps and total_s < seconds_target:
+        nb, dt = sample.step()
+        total_bytes += nb; total_s += dt; steps += 1
+    return {"value": total_bytes / total_s / 1e9, "unit": "GB/s", "cores": sample.cores, "kind": "oracle",
+            "sample": sample.describe(steps), "seconds": total_s}
 
 
 def run_reference(args, w):
+    """The reference arm: the oracle as it stands on the host cores; one step = one oracle decode step over the
+    bounded sample of heads (built once, untimed).  Rank 0 alone runs it."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    vals = []
+    sample = OracleSample(w)
     for _ in range(args.warmup):
-        oracle_sample(w, seconds_target=2.0)
-    t_all = time.perf_counter()
+        sample.step()
+    total_bytes, total_s = 0, 0.0
     for _ in range(args.steps):
-        vals.append(oracle_sample(w, seconds_target=5.0))
-    dt = time.perf_counter() - t_all
-    v = statistics.mean(x["value"] for x in vals)
+        nb, dt = sample.step()
+        total_bytes += nb; total_s += dt
+    v = total_bytes / total_s / 1e9
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": "GB/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(1, args.steps) * 1e3,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_s / max(1, args.steps) * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name},
-        "cpu_baseline": {"value": v, "unit": "GB/s", "cores": vals[-1]["cores"], "kind": "oracle",
-                         "sample": vals[-1]["sample"]},
+        "config": {"workload": w.name, "layers": w.L, "batch": w.B, "context": w.T, "budget": w.budget},
+        "cpu_baseline": {"value": v, "unit": "GB/s", "cores": sample.cores, "kind": "oracle",
+                         "sample": sample.describe(args.steps)},
         "e2e": {"value": v, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 

@@ -22,15 +22,23 @@
 
 #include "baklava.h"
 #include "common.h"
+#include "ptx.cuh"
 
 namespace {
+
+using ptx::ldmatrix_x4;
+using ptx::mbar_arrive_expect_tx;
+using ptx::mbar_init;
+using ptx::mbar_wait;
+using ptx::smem_u32;
+using ptx::tile_offset;          // tiles here are 64 tokens of 64-element boxes: the same swizzled layout
+using tc::mbar_arrive;
 
 constexpr int kConsumerWarps = 4;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;     // + one producer warp
 constexpr int kTileTokens = kTile;                      // 64 tokens per stage
 constexpr int kWarpTokens = kTileTokens / kConsumerWarps;
 constexpr int kStages = 2;                              // 64 KB per CTA, three CTAs per SM
-constexpr uint32_t kWaitLimit = 1u << 22;               // bounded mbarrier waits
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 static_assert(kWarpTokens == 16, "a consumer warp owns one 16-token MMA block of each tile");
@@ -115,33 +123,6 @@ __device__ __forceinline__ HeadState head_state(const DecodeParams& p, const Uni
 __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-__device__ __forceinline__ uint32_t smem_u32(const void* ptr) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    return done != 0;
-}
-// Waits for the phase with the given parity; gives up after kWaitLimit polls and returns false.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
 // K and V are read once per step and never fit in L2: ask L2 to drop them first, so that the
 // step's logits, scores and positions (which the score pass re-reads) stay resident.
 __device__ __forceinline__ uint64_t l2_evict_first_policy() {
@@ -155,10 +136,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
         "[%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -176,13 +153,6 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
-}
-
-// Byte offset of 16-byte piece `piece` of row `row` inside a [64 rows][D] bf16 tile that TMA wrote with
-// the 128-byte swizzle: the tile is D/64 boxes of 64 rows x 128 bytes, each 1024-byte aligned, and piece
-// c of a box row sits at piece position c ^ (row % 8).
-__device__ __forceinline__ uint32_t tile_offset(int row, int piece) {
-    return (uint32_t)((piece >> 3) * (kTileTokens * 128) + row * 128 + (((piece & 7) ^ (row & 7)) << 4));
 }
 
 // ---------------------------------------------------------------- steps 2-4
@@ -250,7 +220,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             mbar_init(smem_u32(&bar_empty[s]), kConsumerWarps);
         }
         sm_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        ptx::fence_mbar_init();
     }
     __syncthreads();
 
