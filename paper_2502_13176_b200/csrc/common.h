@@ -8,6 +8,11 @@
 constexpr int kTile = 64;          // chunk lengths are multiples of this many tokens
 constexpr int kCtasPerSm = 3;       // resident CTAs of the attention kernel per SM (its launch bounds)
 constexpr int kMinChunk = 256;      // shortest chunk the automatic plan makes
+// chunks of a head x group size that the merge of partials can stage in the attention kernel's idle ring
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+constexpr int max_merge_entries(int D) { return 64 * D; }
 constexpr int kScoreChunk = 4096;  // target length of a piece of the score / eviction pass
 
 // Byte offsets of the regions of the decode workspace.
@@ -20,6 +25,13 @@ struct DecodeWorkspace {
     size_t logit_off;      // fp32 [B * seq_stride_tokens][g]: log2-domain logits of this step
     size_t total;
 };
+
+// floats of one chunk's partial result: o [g][D], m [g], l [g], (pos, slot) of its oldest evictable row; padded
+// so that every record starts 16-byte aligned
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+constexpr int partial_floats(int g, int D) { return (g * D + 2 * g + 2 + 3) / 4 * 4; }
 
 int baklava_check_shape(const baklava_shape* s);
 size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_score_items, int64_t n_units, int32_t B,

@@ -400,7 +400,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         }
     }
     __syncthreads();
-    const int psz = G * D + 2 * G + 2;                      // o, m, l, and the chunk's oldest evictable row
+    const int psz = partial_floats(G, D);                   // o, m, l, and the chunk's oldest evictable row
     float* part = p.partial + (int64_t)blockIdx.x * psz;
     for (int i = tid; i < G * D; i += kThreads) {
         const int a = i / D, d = i - a * D;
@@ -437,14 +437,25 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     // ---- this CTA delivered the head's last partial: merge them in chunk order, write the output
     // and leave the final (max, 1 / sum) of every query head for the score kernel
     const float* part0 = p.partial + (int64_t)(blockIdx.x - piece) * psz;
+    // every chunk's (max, sum) into shared memory with one round of loads (the ring is idle now; the plan
+    // keeps chunks x group within max_merge_entries(D))
+    float* sm_mc = reinterpret_cast<float*>(ring_ptr);
+    float* sm_lc = sm_mc + max_merge_entries(D);
+    const int n_ml = active * G;
+    for (int i = tid; i < n_ml; i += kThreads) {
+        const int c = i / G, a = i - c * G;
+        const float* pc = part0 + (int64_t)c * psz + G * D;
+        sm_mc[i] = __ldcg(pc + a);
+        sm_lc[i] = __ldcg(pc + G + a);
+    }
+    __syncthreads();
     if (tid < G) {
         float mm = -INFINITY;
-        for (int c = 0; c < active; ++c) mm = fmaxf(mm, __ldcg(part0 + (int64_t)c * psz + G * D + tid));
+        for (int c = 0; c < active; ++c) mm = fmaxf(mm, sm_mc[c * G + tid]);
         float ll = 0.0f;
         for (int c = 0; c < active; ++c) {
-            const float* pc = part0 + (int64_t)c * psz;
-            const float mc = __ldcg(pc + G * D + tid);
-            if (mc != -INFINITY) ll = fmaf(__ldcg(pc + G * D + G + tid), exp2f(mc - mm), ll);
+            const float mc = sm_mc[c * G + tid];
+            if (mc != -INFINITY) ll = fmaf(sm_lc[c * G + tid], exp2f(mc - mm), ll);
         }
         const float inv = ll > 0.0f ? 1.0f / ll : 0.0f;
         sm_M[tid] = mm;
@@ -455,30 +466,42 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             p.lse[(int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + tid] = ll > 0.0f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
     }
     __syncthreads();
+    for (int i = tid; i < n_ml; i += kThreads) {            // each chunk's weight in the merged output
+        const int a = i % G;
+        const float mc = sm_mc[i];
+        sm_lc[i] = (mc == -INFINITY) ? 0.0f : exp2f(mc - sm_M[a]);
+    }
+    __syncthreads();
     __nv_bfloat16* orow = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
-    for (int i = tid; i < G * D; i += kThreads) {
-        const int a = i / D;
-        const float Ma = sm_M[a];
-        float acc = 0.0f;
+    for (int grp = tid; grp < G * D / 4; grp += kThreads) { // four output elements per thread, chunks in order
+        const int a = (grp * 4) / D;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         int c = 0;
-        for (; c + 4 <= active; c += 4) {                   // four chunks' loads in flight, summed in order
-            float mc[4], oc[4];
+        for (; c + 8 <= active; c += 8) {                   // eight chunks' loads in flight
+            float4 oc[8];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float* pc = part0 + (int64_t)(c + k) * psz;
-                mc[k] = __ldcg(pc + G * D + a);
-                oc[k] = __ldcg(pc + i);
+            for (int k = 0; k < 8; ++k)
+                oc[k] = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)(c + k) * psz) + grp);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float wgt = sm_lc[(c + k) * G + a];
+                acc.x = fmaf(oc[k].x, wgt, acc.x); acc.y = fmaf(oc[k].y, wgt, acc.y);
+                acc.z = fmaf(oc[k].z, wgt, acc.z); acc.w = fmaf(oc[k].w, wgt, acc.w);
             }
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (mc[k] != -INFINITY) acc = fmaf(oc[k], exp2f(mc[k] - Ma), acc);
         }
         for (; c < active; ++c) {
-            const float* pc = part0 + (int64_t)c * psz;
-            const float mc = __ldcg(pc + G * D + a);
-            if (mc != -INFINITY) acc = fmaf(__ldcg(pc + i), exp2f(mc - Ma), acc);
+            const float4 oc = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)c * psz) + grp);
+            const float wgt = sm_lc[c * G + a];
+            acc.x = fmaf(oc.x, wgt, acc.x); acc.y = fmaf(oc.y, wgt, acc.y);
+            acc.z = fmaf(oc.z, wgt, acc.z); acc.w = fmaf(oc.w, wgt, acc.w);
         }
-        orow[i] = __float2bfloat16_rn(acc * sm_invL[a]);
+        const float inv = sm_invL[a];
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<const uint32_t*>(&lo);
+        packed.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(orow + grp * 4) = packed;
     }
     if (tid == 0) {
         p.arrive[unit] = 0;                                 // the score kernel counts arrivals again

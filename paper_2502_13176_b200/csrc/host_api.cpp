@@ -170,7 +170,7 @@ size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t 
     w.arrive_off = take(sizeof(int32_t) * (size_t)n_units);
     w.stats_off = take(sizeof(float) * (size_t)n_units * 2 * BAKLAVA_MAX_GROUP);
     w.best_off = take(16 * (size_t)n_score_items);
-    w.partial_off = take(sizeof(float) * (size_t)n_items * (g * (s->D + 2) + 2));
+    w.partial_off = take(sizeof(float) * (size_t)n_items * partial_floats(g, s->D));
     w.logit_off = take(sizeof(float) * (size_t)B * (size_t)seq_stride_tokens * g);
     w.total = off;
     if (lay) *lay = w;
@@ -231,7 +231,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
             int64_t pieces = (c + want - 1) / want;
             const int64_t len = ((c + pieces - 1) / pieces + kTile - 1) / kTile * kTile;
             pieces = (c + len - 1) / len;
-            if (pieces > 32767) return BAKLAVA_ERR_UNSUPPORTED;
+            if (pieces > 32767 || pieces * (shape->Hq / Hkv) > max_merge_entries(shape->D)) return BAKLAVA_ERR_UNSUPPORTED;
             const int li = i / Hkv, h = i % Hkv;
             for (int b = 0; b < B; ++b) {
                 const int64_t unit = ((int64_t)li * B + b) * Hkv + h;
