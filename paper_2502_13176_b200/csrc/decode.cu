@@ -546,15 +546,17 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
     launch_dependents();
-    grid_dependency_wait();                               // the attention kernel's scratch and statistics
+    // len and free_slot are not touched by the attention kernel when a score pass follows (this kernel does
+    // the bookkeeping), so the head's state can be read while that kernel is still draining
     const HeadState hs = head_state(p, u);
+    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    grid_dependency_wait();                               // the attention kernel's scratch and statistics
     if (hs.bad) return;                                    // reported by the attention kernel
     const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
     if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
 
-    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
     const __half* prob_h = reinterpret_cast<const __half*>(p.logit + row0 * G);
     const float* mref_h = reinterpret_cast<const float*>(prob_h + (int64_t)G * C);
     float Mq[G], iL[G];
