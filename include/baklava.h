@@ -208,6 +208,17 @@ int baklava_decode_attn(const baklava_shape* shape, const baklava_cache* cache,
                         const int32_t* items, const baklava_plan_info* info,
                         void* ws, size_t ws_bytes, void* stream);
 
+/* The same step for a batch whose sequences are at different positions (requests that joined at
+ * different times, prompts of different lengths).  Eq. 4-7 are per sequence, so nothing in them
+ * changes: sequence b runs the step above with t_pos[b].  A negative t_pos[b] marks a sequence that
+ * sits this step out: none of its cache, out or lse entries is read or written.
+ *   t_pos    device int32 [B]; every other argument as for baklava_decode_attn */
+int baklava_decode_attn_varlen(const baklava_shape* shape, const baklava_cache* cache,
+                               const void* q, const void* k_new, const void* v_new, const int32_t* t_pos,
+                               void* out, float* lse, uint32_t flags,
+                               const int32_t* items, const baklava_plan_info* info,
+                               void* ws, size_t ws_bytes, void* stream);
+
 /* ------------------------------------------------------------------ bulk eviction (Eq. 5-6)
  * Cut dense prefilled heads of T tokens down to their capacities and compact them into
  * the slabs (the MAKE_CACHE of Algorithm 3).  Row t of head (layer, b, h) is token row
@@ -225,6 +236,18 @@ int baklava_evict(const baklava_shape* shape, const baklava_cache* cache,
                   int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
                   void* ws, size_t ws_bytes, void* stream);
 size_t baklava_evict_workspace_size(const baklava_shape* shape, int32_t B, int32_t layers, int32_t T);
+
+/* The same for prompts of different lengths: sequence b has prompt_len[b] tokens (clamped to
+ * 0 .. T; rows at or past it are not tokens and are never read), and the rule above is applied
+ * with that length in place of T.  A sequence of length 0 ends with len = free_slot = 0.
+ *   prompt_len  device int32 [B], or NULL for T everywhere (then identical to baklava_evict)
+ * The workspace is sized for T as in baklava_evict. */
+int baklava_evict_varlen(const baklava_shape* shape, const baklava_cache* cache,
+                         int32_t layer_begin, int32_t layer_end,
+                         const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
+                         const int32_t* prompt_len,
+                         int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
+                         void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------ prompt scores (seed of step 3)
  * The accumulated attention a prompt leaves on its own tokens, for ONE layer: with the causal

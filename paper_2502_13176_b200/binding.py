@@ -70,6 +70,12 @@ def lib():
         L.baklava_decode_attn.argtypes = [POINTER(Shape), POINTER(CacheStruct), c_void_p, c_void_p, c_void_p, c_int32,
                                           c_void_p, c_void_p, c_uint32, c_void_p, POINTER(PlanInfo),
                                           c_void_p, c_size_t, c_void_p]
+        L.baklava_decode_attn_varlen.argtypes = [POINTER(Shape), POINTER(CacheStruct), c_void_p, c_void_p, c_void_p,
+                                                 c_void_p, c_void_p, c_void_p, c_uint32, c_void_p, POINTER(PlanInfo),
+                                                 c_void_p, c_size_t, c_void_p]
+        L.baklava_evict_varlen.argtypes = [POINTER(Shape), POINTER(CacheStruct), c_int32, c_int32, c_void_p, c_void_p,
+                                           c_void_p, c_int32, c_void_p, c_int64, c_int64, c_int64, c_int32, c_void_p,
+                                           c_size_t, c_void_p]
         L.baklava_evict.argtypes = [POINTER(Shape), POINTER(CacheStruct), c_int32, c_int32, c_void_p, c_void_p,
                                     c_void_p, c_int32, c_int64, c_int64, c_int64, c_int32, c_void_p, c_size_t, c_void_p]
         L.baklava_evict_workspace_size.restype = c_size_t
@@ -212,6 +218,16 @@ def baklava_decode_attn(shape, cache, q, k_new, v_new, t_pos, out, lse, flags, p
            "baklava_decode_attn")
 
 
+def baklava_decode_attn_varlen(shape, cache, q, k_new, v_new, t_pos, out, lse, flags, plan, ws, stream=None):
+    """t_pos: device int32 [B]; a negative entry idles that sequence for the step."""
+    assert t_pos.dtype == torch.int32 and t_pos.numel() == cache.B and t_pos.is_cuda
+    _check(lib().baklava_decode_attn_varlen(ctypes.byref(shape), ctypes.byref(cache.struct), _ptr(q), _ptr(k_new),
+                                            _ptr(v_new), _ptr(t_pos), _ptr(out), _ptr(lse), int(flags),
+                                            _ptr(plan.items_dev), ctypes.byref(plan.info), _ptr(ws),
+                                            ws.numel() * ws.element_size(), _stream(stream)),
+           "baklava_decode_attn_varlen")
+
+
 def baklava_evict_workspace_size(shape, B, layers, T):
     return int(lib().baklava_evict_workspace_size(ctypes.byref(shape), B, layers, T))
 
@@ -222,6 +238,15 @@ def baklava_evict(shape, cache, layer_begin, layer_end, k_dense, v_dense, score_
                                _ptr(k_dense), _ptr(v_dense), _ptr(score_dense), int(T), int(stride_layer),
                                int(stride_seq), int(stride_head), int(reserve), _ptr(ws),
                                ws.numel() * ws.element_size(), _stream(stream)), "baklava_evict")
+
+
+def baklava_evict_varlen(shape, cache, layer_begin, layer_end, k_dense, v_dense, score_dense, T, prompt_len,
+                         stride_layer, stride_seq, stride_head, reserve, ws, stream=None):
+    """prompt_len: device int32 [B] or None."""
+    _check(lib().baklava_evict_varlen(ctypes.byref(shape), ctypes.byref(cache.struct), layer_begin, layer_end,
+                                      _ptr(k_dense), _ptr(v_dense), _ptr(score_dense), int(T), _ptr(prompt_len),
+                                      int(stride_layer), int(stride_seq), int(stride_head), int(reserve), _ptr(ws),
+                                      ws.numel() * ws.element_size(), _stream(stream)), "baklava_evict_varlen")
 
 
 EVICT_STATIC_MAX_ENTRIES = 1 << 20

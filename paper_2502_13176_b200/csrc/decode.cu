@@ -62,6 +62,7 @@ struct DecodeParams {
     __nv_bfloat16* out;
     float* lse;
     int32_t t_pos;
+    const int32_t* t_pos_seq;      // per-sequence positions [B] (negative: the sequence sits this step out) or NULL
     uint32_t flags;
     int32_t window_evict;          // 1: no scores are kept and the policy is sinks + window: evict by position
     const int4* items;             // attention items, then score items
@@ -185,8 +186,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const int4 item = p.items[blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
-    launch_dependents();
     grid_dependency_wait();                               // len / free_slot / slab rows come from earlier kernels
+    // Only now may the score kernel's CTAs become resident: they read len / free_slot before their own
+    // dependency wait, and this order guarantees that the previous step's bookkeeping is complete by then
+    // even when the whole grid is resident at once.
+    launch_dependents();
+    const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
+    if (t_pos < 0) return;                                // idle sequence: nothing of it is read or written
     const HeadState hs = head_state(p, u);
     if (hs.bad) {
         if (tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
@@ -201,7 +207,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
     // sinks + window without scores: the one row that is neither a sink nor in the window (the oldest) goes
     const bool pos_evict = kByPosition && hs.do_append && n_hi > C - 1;
-    const int window_from = p.t_pos - max(0, (int)(((int64_t)(C - 1 - p.n_sink) * p.recent_num) / p.recent_den));
+    const int window_from = t_pos - max(0, (int)(((int64_t)(C - 1 - p.n_sink) * p.recent_num) / p.recent_den));
     int old_pos = INT32_MAX, old_slot = -1;                // per lane, then per warp: oldest evictable row seen
 
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
@@ -296,7 +302,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                         *reinterpret_cast<uint4*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c)) = val;
                         *(reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c) = val;
                     }
-                    if (lane == 0) { p.pos[row] = p.t_pos; p.score[row] = 0.0f; }
+                    if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
                     __syncwarp();
                 }
                 if (kByPosition && pos_evict && lane < valid && tok0 + lane != hs.f) {
@@ -549,9 +555,10 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
     // len and free_slot are not touched by the attention kernel when a score pass follows (this kernel does
     // the bookkeeping), so the head's state can be read while that kernel is still draining
     const HeadState hs = head_state(p, u);
+    const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
     grid_dependency_wait();                               // the attention kernel's scratch and statistics
-    if (hs.bad) return;                                    // reported by the attention kernel
+    if (hs.bad || t_pos < 0) return;                       // reported by the attention kernel / idle sequence
     const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
     if (piece >= active) return;
@@ -569,7 +576,7 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
     const int R = C - 1;
     const bool evict = appended && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n_hi > R;
     const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
-    const int newest_candidate = p.t_pos - W;              // rows with pos > this are in the recent window
+    const int newest_candidate = t_pos - W;              // rows with pos > this are in the recent window
 
     unsigned long long best = ~0ull;
     int best_slot = -1;
@@ -742,9 +749,10 @@ cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CU
 
 }  // namespace
 
-extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
+namespace {
+int decode_attn_impl(
         const baklava_shape* shape, const baklava_cache* cache,
-        const void* q, const void* k_new, const void* v_new, int32_t t_pos,
+        const void* q, const void* k_new, const void* v_new, int32_t t_pos, const int32_t* t_pos_seq,
         void* out, float* lse, uint32_t flags,
         const int32_t* items, const baklava_plan_info* info,
         void* ws, size_t ws_bytes, void* stream) {
@@ -797,6 +805,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lse = lse;
     p.t_pos = t_pos;
+    p.t_pos_seq = t_pos_seq;
     // without scores only the pure sinks + window policy can still choose a victim (by position)
     p.window_evict = (flags & BAKLAVA_FLAG_NO_SCORE) && !(flags & BAKLAVA_FLAG_NO_EVICT) &&
                      shape->recent_num == shape->recent_den;
@@ -843,4 +852,27 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
         if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
     }
     return BAKLAVA_OK;
+}
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) int baklava_decode_attn(
+        const baklava_shape* shape, const baklava_cache* cache,
+        const void* q, const void* k_new, const void* v_new, int32_t t_pos,
+        void* out, float* lse, uint32_t flags,
+        const int32_t* items, const baklava_plan_info* info,
+        void* ws, size_t ws_bytes, void* stream) {
+    if (t_pos < 0) return BAKLAVA_ERR_INVALID_ARG;
+    return decode_attn_impl(shape, cache, q, k_new, v_new, t_pos, nullptr, out, lse, flags, items, info, ws, ws_bytes,
+                            stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int baklava_decode_attn_varlen(
+        const baklava_shape* shape, const baklava_cache* cache,
+        const void* q, const void* k_new, const void* v_new, const int32_t* t_pos,
+        void* out, float* lse, uint32_t flags,
+        const int32_t* items, const baklava_plan_info* info,
+        void* ws, size_t ws_bytes, void* stream) {
+    if (!t_pos) return BAKLAVA_ERR_INVALID_ARG;
+    return decode_attn_impl(shape, cache, q, k_new, v_new, 0, t_pos, out, lse, flags, items, info, ws, ws_bytes,
+                            stream);
 }

@@ -36,12 +36,13 @@ struct EvictParams {
     const __nv_bfloat16* v_dense;
     const float* score_dense;
     int32_t T, reserve;
+    const int32_t* seq_len;   // [B] tokens of each sequence's prompt (clamped to 0 .. T) or NULL: T for all
     int64_t stride_layer, stride_seq, stride_head;
     int32_t* kept;   // [n_units][T]
 };
 
 struct Where {
-    int head, st;
+    int head, st, b;
     int64_t dense0, slab0;
 };
 
@@ -52,6 +53,7 @@ __device__ __forceinline__ Where locate(const EvictParams& p, int unit) {
     const int l = p.layer_begin + li;
     Where w;
     w.head = l * p.Hkv + h;
+    w.b = b;
     w.st = (b * p.L + l) * p.Hkv + h;
     w.dense0 = (int64_t)li * p.stride_layer + (int64_t)b * p.stride_seq + (int64_t)h * p.stride_head;
     w.slab0 = (int64_t)b * p.seq_stride + p.slab_off[w.head];
@@ -102,7 +104,7 @@ __global__ void __launch_bounds__(kSelThreads) evict_select_kernel(const EvictPa
     const int C = p.cap[w.head];
     const int R = C - p.reserve;
     int32_t* kept = p.kept + (int64_t)unit * p.T;
-    const int T = p.T;
+    const int T = p.seq_len ? min(max(p.seq_len[w.b], 0), p.T) : p.T;
     if (R < 1) {
         if (tid == 0) { atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE); p.len[w.st] = 0; p.free_slot[w.st] = 0; }
         return;
@@ -206,26 +208,19 @@ extern "C" __attribute__((visibility("default"))) size_t baklava_evict_workspace
     return (size_t)B * layers * shape->Hkv * (size_t)T * sizeof(int32_t);
 }
 
-extern "C" __attribute__((visibility("default"))) int baklava_evict(const baklava_shape* shape, const baklava_cache* cache,
-                             int32_t layer_begin, int32_t layer_end,
-                             const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
-                             int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
-                             void* ws, size_t ws_bytes, void* stream) {
-    int rc = baklava_check_shape(shape);
-    if (rc) return rc;
-    if (!cache || !ws) return BAKLAVA_ERR_INVALID_ARG;
+namespace {
+
+// Argument checks and launches shared by the three entry points; `kept` has room for units * T entries.
+int evict_impl(const baklava_shape* shape, const baklava_cache* cache, int32_t layer_begin, int32_t layer_end,
+               const void* k_dense, const void* v_dense, const float* score_dense, int32_t T, const int32_t* seq_len,
+               int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
+               int32_t* kept, void* stream) {
     if (!k_dense || !v_dense) return BAKLAVA_ERR_UNSUPPORTED;   // in-place compaction of a slab
-    if (!cache->k_slab || !cache->v_slab || !cache->pos || !cache->score || !cache->len || !cache->free_slot ||
-        !cache->cap || !cache->slab_off || !cache->status || cache->B <= 0 || cache->seq_stride_tokens <= 0)
-        return BAKLAVA_ERR_INVALID_ARG;
-    if (layer_begin < 0 || layer_end > shape->L || layer_begin >= layer_end) return BAKLAVA_ERR_INVALID_ARG;
     if (T <= 0 || reserve < 1 || stride_layer < 0 || stride_seq < 0 || stride_head < T) return BAKLAVA_ERR_INVALID_ARG;
-    const void* ptrs[] = {k_dense, v_dense, cache->k_slab, cache->v_slab, ws};
+    const void* ptrs[] = {k_dense, v_dense, cache->k_slab, cache->v_slab};
     for (const void* ptr : ptrs)
         if (!baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
-    const int layers = layer_end - layer_begin;
-    if (ws_bytes < baklava_evict_workspace_size(shape, cache->B, layers, T)) return BAKLAVA_ERR_WORKSPACE;
-    const int64_t units = (int64_t)layers * cache->B * shape->Hkv;
+    const int64_t units = (int64_t)(layer_end - layer_begin) * cache->B * shape->Hkv;
     const int64_t row_blocks = ((int64_t)T + kCopyRows - 1) / kCopyRows;
     if (units > INT32_MAX || row_blocks > 65535) return BAKLAVA_ERR_UNSUPPORTED;
 
@@ -242,8 +237,9 @@ extern "C" __attribute__((visibility("default"))) int baklava_evict(const baklav
     p.v_dense = static_cast<const __nv_bfloat16*>(v_dense);
     p.score_dense = score_dense;
     p.T = T; p.reserve = reserve;
+    p.seq_len = seq_len;
     p.stride_layer = stride_layer; p.stride_seq = stride_seq; p.stride_head = stride_head;
-    p.kept = static_cast<int32_t*>(ws);
+    p.kept = kept;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     evict_select_kernel<<<(unsigned)units, kSelThreads, 0, s>>>(p);
@@ -252,6 +248,43 @@ extern "C" __attribute__((visibility("default"))) int baklava_evict(const baklav
     if (shape->D == 128) evict_copy_kernel<128><<<grid, kCopyThreads, 0, s>>>(p);
     else evict_copy_kernel<64><<<grid, kCopyThreads, 0, s>>>(p);
     return cudaGetLastError() == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
+}
+
+int check_cache_and_layers(const baklava_shape* shape, const baklava_cache* cache, int32_t layer_begin,
+                           int32_t layer_end) {
+    int rc = baklava_check_shape(shape);
+    if (rc) return rc;
+    if (!cache) return BAKLAVA_ERR_INVALID_ARG;
+    if (!cache->k_slab || !cache->v_slab || !cache->pos || !cache->score || !cache->len || !cache->free_slot ||
+        !cache->cap || !cache->slab_off || !cache->status || cache->B <= 0 || cache->seq_stride_tokens <= 0)
+        return BAKLAVA_ERR_INVALID_ARG;
+    if (layer_begin < 0 || layer_end > shape->L || layer_begin >= layer_end) return BAKLAVA_ERR_INVALID_ARG;
+    return BAKLAVA_OK;
+}
+
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) int baklava_evict_varlen(
+        const baklava_shape* shape, const baklava_cache* cache, int32_t layer_begin, int32_t layer_end,
+        const void* k_dense, const void* v_dense, const float* score_dense, int32_t T, const int32_t* prompt_len,
+        int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
+        void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_cache_and_layers(shape, cache, layer_begin, layer_end);
+    if (rc) return rc;
+    if (!ws || !baklava_aligned16(ws)) return BAKLAVA_ERR_INVALID_ARG;
+    if (T > 0 && ws_bytes < baklava_evict_workspace_size(shape, cache->B, layer_end - layer_begin, T))
+        return BAKLAVA_ERR_WORKSPACE;
+    return evict_impl(shape, cache, layer_begin, layer_end, k_dense, v_dense, score_dense, T, prompt_len,
+                      stride_layer, stride_seq, stride_head, reserve, static_cast<int32_t*>(ws), stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int baklava_evict(const baklava_shape* shape, const baklava_cache* cache,
+                             int32_t layer_begin, int32_t layer_end,
+                             const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
+                             int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
+                             void* ws, size_t ws_bytes, void* stream) {
+    return baklava_evict_varlen(shape, cache, layer_begin, layer_end, k_dense, v_dense, score_dense, T, nullptr,
+                                stride_layer, stride_seq, stride_head, reserve, ws, ws_bytes, stream);
 }
 
 // ---------------------------------------------------------------- bulk eviction without a workspace
@@ -287,46 +320,14 @@ extern "C" __attribute__((visibility("default"))) int baklava_evict_static(
         const baklava_shape* shape, const baklava_cache* cache, int32_t layer_begin, int32_t layer_end,
         const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
         int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve, void* stream) {
-    int rc = baklava_check_shape(shape);
+    int rc = check_cache_and_layers(shape, cache, layer_begin, layer_end);
     if (rc) return rc;
-    if (!cache || !k_dense || !v_dense) return BAKLAVA_ERR_INVALID_ARG;
-    if (!cache->k_slab || !cache->v_slab || !cache->pos || !cache->score || !cache->len || !cache->free_slot ||
-        !cache->cap || !cache->slab_off || !cache->status || cache->B <= 0 || cache->seq_stride_tokens <= 0)
-        return BAKLAVA_ERR_INVALID_ARG;
-    if (layer_begin < 0 || layer_end > shape->L || layer_begin >= layer_end) return BAKLAVA_ERR_INVALID_ARG;
-    if (T <= 0 || reserve < 1 || stride_layer < 0 || stride_seq < 0 || stride_head < T) return BAKLAVA_ERR_INVALID_ARG;
-    const void* ptrs[] = {k_dense, v_dense, cache->k_slab, cache->v_slab};
-    for (const void* ptr : ptrs)
-        if (!baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
+    if (!k_dense || !v_dense || T <= 0) return BAKLAVA_ERR_INVALID_ARG;
     const int64_t units = (int64_t)(layer_end - layer_begin) * cache->B * shape->Hkv;
-    const int64_t row_blocks = ((int64_t)T + kCopyRows - 1) / kCopyRows;
     if (units * (int64_t)T > (int64_t)kStaticKeptEntries) return BAKLAVA_ERR_WORKSPACE;   // beyond the fixed array
-    if (units > INT32_MAX || row_blocks > 65535) return BAKLAVA_ERR_UNSUPPORTED;
     int32_t* kept = nullptr;
     rc = static_kept_address(&kept);
     if (rc) return rc;
-
-    EvictParams p;
-    p.k_slab = static_cast<__nv_bfloat16*>(cache->k_slab);
-    p.v_slab = static_cast<__nv_bfloat16*>(cache->v_slab);
-    p.pos = cache->pos; p.score = cache->score; p.len = cache->len; p.free_slot = cache->free_slot;
-    p.cap = cache->cap; p.slab_off = cache->slab_off; p.seq_stride = cache->seq_stride_tokens;
-    p.status = cache->status;
-    p.B = cache->B; p.L = shape->L; p.Hkv = shape->Hkv;
-    p.n_sink = shape->n_sink; p.recent_num = shape->recent_num; p.recent_den = shape->recent_den;
-    p.layer_begin = layer_begin;
-    p.k_dense = static_cast<const __nv_bfloat16*>(k_dense);
-    p.v_dense = static_cast<const __nv_bfloat16*>(v_dense);
-    p.score_dense = score_dense;
-    p.T = T; p.reserve = reserve;
-    p.stride_layer = stride_layer; p.stride_seq = stride_seq; p.stride_head = stride_head;
-    p.kept = kept;
-
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    evict_select_kernel<<<(unsigned)units, kSelThreads, 0, s>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
-    const dim3 grid((unsigned)units, (unsigned)row_blocks);
-    if (shape->D == 128) evict_copy_kernel<128><<<grid, kCopyThreads, 0, s>>>(p);
-    else evict_copy_kernel<64><<<grid, kCopyThreads, 0, s>>>(p);
-    return cudaGetLastError() == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
+    return evict_impl(shape, cache, layer_begin, layer_end, k_dense, v_dense, score_dense, T, nullptr,
+                      stride_layer, stride_seq, stride_head, reserve, kept, stream);
 }
