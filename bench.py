@@ -288,6 +288,9 @@ def main():
     ap.add_argument("--policy", default="heavy", choices=["heavy", "window"],
                     help="heavy: sinks + window + accumulated-attention heavy hitters (default); "
                          "window: the paper's evaluated sinks + window policy, run without scores")
+    ap.add_argument("--mixed-lengths", action="store_true",
+                    help="prompts of different lengths (seeded, uniform in [T/8, T]) decoded at per-sequence "
+                         "positions through baklava_decode_attn_varlen")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.workload == "profile":
@@ -317,8 +320,23 @@ def main():
     bk.lib()                                             # fail now if the library is missing
     step_flags = bk.FLAG_NO_SCORE if args.policy == "window" else 0
     sess = DecodeSession(w, dev, chunk_tokens=args.chunk)
-    sess.prefill_synthetic()
     total = args.warmup + args.steps
+    if args.mixed_lengths:
+        from paper_2502_13176_b200 import synth
+        u = synth.uniform_f64(w.seed, 50, 0, w.B).numpy()
+        prompt_len = [int(w.T // 8 + x * (w.T - w.T // 8)) for x in u]
+        sess.prefill_synthetic(prompt_len)
+        # positions of every step, made ahead so that no other kernel runs between the steps
+        t_steps = (sess.t_seq[None, :] + torch.arange(4 * total, device=dev, dtype=torch.int32)[:, None]).contiguous()
+        counter = [0]
+
+        def varlen_step(q, k, v, flags=0):
+            i = counter[0]; counter[0] += 1
+            return sess.step_varlen(q, k, v, t_steps[i], flags)
+        sess.step = varlen_step
+        w = wl.scaled(w, name=w.name + "-mixed")
+    else:
+        sess.prefill_synthetic()
     feeds = [wl.decode_inputs(w, i, sess.scales, dev) for i in range(2 * total)]
     torch.cuda.synchronize(dev)
 
@@ -385,7 +403,8 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "layers": w.L, "batch": w.B, "context": w.T, "budget": w.budget,
                        "kv_bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (no flush)",
-                       "launch": "one baklava_decode_attn call per step covering all layers", "policy": args.policy,
+                       "launch": "one baklava_decode_attn%s call per step covering all layers" % (
+                           "_varlen" if args.mixed_lengths else ""), "policy": args.policy,
                        "replicas": world},
             "tokens_per_s": whole_job_rate(world, w.B, args.steps, elapsed_ms),
             "pct_of_hbm_peak": 100.0 * gbs / world / peak,

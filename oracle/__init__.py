@@ -13,9 +13,12 @@ the paper's order and notation:
   allocation.py  Algorithm 2             threshold / reduction budget reallocation
   eviction.py    Eq. 5-6 + policy        which entries stay, bulk compaction
   cache.py       Eq. 4-7 iterated        one head's slab and one decode step
+  prefill.py     Eq. 1 column sums       accumulated attention a prompt leaves on its tokens
+  search.py      Algorithm 3             parameter search loop with an attention-output loss
 
 Parity status: every function is pinned by the CPU tests (closed forms,
-library routines, brute force, invariants) except the choice of the search
-parameters (t, r) and anything that needs model weights or benchmark data:
-those are "parity unpinned" and are not part of this oracle.
+library routines, brute force, invariants).  The search loop and its loss are
+pinned as arithmetic; which (t, r) is best for a real model, and anything else
+that needs model weights or benchmark data, is "parity unpinned" and is not
+part of this oracle.
 """

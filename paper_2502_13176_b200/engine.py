@@ -32,17 +32,20 @@ class DecodeSession:
         self.lse = torch.zeros((nl, w.B, w.Hq), dtype=torch.float32, device=self.device)
         self.t = 0
 
-    def prefill_synthetic(self):
-        """Fill every head from the workload's dense synthetic prompt through baklava_evict, a layer at a time."""
+    def prefill_synthetic(self, prompt_len=None):
+        """Fill every head from the workload's dense synthetic prompt through baklava_evict, a layer at a time.
+        `prompt_len` (B ints) keeps only that many tokens of each sequence's prompt."""
         w = self.w
         ews = torch.empty((bk.baklava_evict_workspace_size(self.shape, w.B, 1, w.T),), dtype=torch.uint8,
                           device=self.device)
+        plen = None if prompt_len is None else torch.tensor(list(prompt_len), dtype=torch.int32, device=self.device)
         for l in range(self.lb, self.le):
             k, v = wl.dense_kv_layer(w, l, self.scales, self.device)
             sc = wl.prefill_scores(w, l, self.device)
-            bk.baklava_evict(self.shape, self.cache, l, l + 1, k, v, sc, w.T, 0, w.Hkv * w.T, w.T, 1, ews)
+            bk.baklava_evict_varlen(self.shape, self.cache, l, l + 1, k, v, sc, w.T, plen, 0, w.Hkv * w.T, w.T, 1, ews)
             torch.cuda.synchronize(self.device)
         self.t = w.T
+        self.t_seq = plen
 
     def step(self, q, k_new, v_new, flags=0):
         """One decode step for the session's layer range; returns the output tensor (device, bf16)."""
@@ -50,6 +53,12 @@ class DecodeSession:
                                self.plan, self.ws)
         if not (flags & bk.FLAG_NO_APPEND):
             self.t += 1
+        return self.out
+
+    def step_varlen(self, q, k_new, v_new, t_pos, flags=0):
+        """One decode step with per-sequence positions `t_pos` (device int32 [B]; negative = idle)."""
+        bk.baklava_decode_attn_varlen(self.shape, self.cache, q, k_new, v_new, t_pos, self.out, self.lse, flags,
+                                      self.plan, self.ws)
         return self.out
 
     def retained_kv_bytes(self):
