@@ -265,6 +265,27 @@ int baklava_prefill_scores(const baklava_shape* shape, const void* q, const void
                            float* score, void* ws, size_t ws_bytes, void* stream);
 size_t baklava_prefill_workspace_size(const baklava_shape* shape, int32_t B, int32_t T);
 
+/* ------------------------------------------------------------------ Algorithm 3 (parameter search)
+ * The search evaluates every candidate (t, r): make the cache (baklava_allocate + baklava_evict),
+ * run the evaluation chunks through it, average the chunk losses, keep the best.  The paper's
+ * loss is a model's perplexity; this library has no model, so it offers the loss that can be
+ * computed from the attention path alone: how far the budgeted cache moves the attention outputs
+ * away from those of the dense cache,
+ *     loss = mean over rows i of ||out_i - ref_i||^2 / max(||ref_i||^2, 1e-30),
+ * rows being the output vectors of every (layer, sequence, query head) of one or more steps.
+ *   out, ref   device bf16 [rows, D], D even
+ *   loss       device fp64 [1], overwritten (0 for rows = 0)
+ *   ws         device workspace >= baklava_output_error_workspace_size(rows) bytes
+ * Row sums are taken in fp32, the mean over rows in fp64, both in a fixed order. */
+int baklava_output_error(const void* out, const void* ref, int64_t rows, int32_t D, double* loss,
+                         void* ws, size_t ws_bytes, void* stream);
+size_t baklava_output_error_workspace_size(int64_t rows);
+
+/* The search's selection rule, on the host: *best = index of the first strictly smallest average
+ * loss (a later equal loss does not replace it, a NaN never wins), -1 if no entry is below +inf.
+ *   avg_loss   host fp64 [n] */
+int baklava_search_pick(const double* avg_loss, int32_t n, int32_t* best);
+
 /* ------------------------------------------------------------------ bulk eviction, no workspace
  * (No counterpart in the paper: this is a packaging variant of baklava_evict.)
  * Same operation, arguments and results as baklava_evict, for callers that cannot provide a

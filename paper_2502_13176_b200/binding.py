@@ -88,6 +88,10 @@ def lib():
                                              c_void_p, c_void_p, c_size_t, c_void_p]
         L.baklava_prefill_workspace_size.restype = c_size_t
         L.baklava_prefill_workspace_size.argtypes = [POINTER(Shape), c_int32, c_int32]
+        L.baklava_output_error.argtypes = [c_void_p, c_void_p, c_int64, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]
+        L.baklava_output_error_workspace_size.restype = c_size_t
+        L.baklava_output_error_workspace_size.argtypes = [c_int64]
+        L.baklava_search_pick.argtypes = [POINTER(c_double), c_int32, POINTER(c_int32)]
         L.baklava_profile_workspace_size.restype = c_size_t
         L.baklava_profile_workspace_size.argtypes = [POINTER(Shape), c_int32, c_int32]
         _lib = L
@@ -281,3 +285,25 @@ def baklava_prefill_scores(shape, q, k, prompt_len, B, T, score, ws, stream=None
     _check(lib().baklava_prefill_scores(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(prompt_len), B, T, _ptr(score),
                                         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
            "baklava_prefill_scores")
+
+
+def baklava_output_error(out, ref, loss, ws, stream=None):
+    """out, ref: bf16 tensors of the same shape [..., D]; loss: float64 tensor [1] (device), overwritten."""
+    assert out.shape == ref.shape and out.dtype == torch.bfloat16 and ref.dtype == torch.bfloat16
+    assert out.is_contiguous() and ref.is_contiguous() and loss.dtype == torch.float64
+    D = out.shape[-1]
+    rows = out.numel() // D
+    _check(lib().baklava_output_error(_ptr(out), _ptr(ref), rows, D, _ptr(loss), _ptr(ws),
+                                      ws.numel() * ws.element_size(), _stream(stream)), "baklava_output_error")
+
+
+def baklava_output_error_workspace_size(rows):
+    return int(lib().baklava_output_error_workspace_size(int(rows)))
+
+
+def baklava_search_pick(avg_loss):
+    a = np.ascontiguousarray(avg_loss, dtype=np.float64)
+    best = c_int32(-2)
+    _check(lib().baklava_search_pick(a.ctypes.data_as(POINTER(c_double)), len(a), ctypes.byref(best)),
+           "baklava_search_pick")
+    return int(best.value)

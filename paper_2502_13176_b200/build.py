@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbaklava.so")
-SOURCES = ["host_api.cpp", "decode.cu", "evict.cu", "profile.cu", "prefill.cu"]
+SOURCES = ["host_api.cpp", "decode.cu", "evict.cu", "profile.cu", "prefill.cu", "search.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fvisibility=hidden", "-Xptxas", "-v"]
 

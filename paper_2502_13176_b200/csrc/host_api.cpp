@@ -265,3 +265,15 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
     info->ws_bytes = (int64_t)baklava_decode_ws_bytes(shape, n_items, n_score, info->n_units, B, seq_stride_tokens, nullptr);
     return BAKLAVA_OK;
 }
+
+// ---------------------------------------------------------------- Algorithm 3: which configuration wins
+extern "C" __attribute__((visibility("default"))) int baklava_search_pick(const double* avg_loss, int32_t n,
+                                                                          int32_t* best) {
+    if (!best || n < 0 || (n > 0 && !avg_loss)) return BAKLAVA_ERR_INVALID_ARG;
+    int32_t at = -1;
+    double min_loss = __builtin_inf();
+    for (int32_t i = 0; i < n; ++i)
+        if (avg_loss[i] < min_loss) { min_loss = avg_loss[i]; at = i; }   // strict: the first minimum stays; NaN never wins
+    *best = at;
+    return BAKLAVA_OK;
+}

@@ -13,13 +13,18 @@ def shape_of(w):
 
 
 class DecodeSession:
-    def __init__(self, w, device="cuda", layers=None, chunk_tokens=0, uniform=False):
+    def __init__(self, w, device="cuda", layers=None, chunk_tokens=0, uniform=False, alloc=None, importance=None,
+                 total_tokens=None):
+        """`alloc` = (t, r_num, r_den) overrides the workload's Algorithm 2 parameters, `importance` its
+        synthetic importances, `total_tokens` its budget (e.g. the dense length for a reference run)."""
         self.w, self.device = w, torch.device(device)
         self.shape = shape_of(w)
         self.scales = wl.kv_scales(w)
-        self.importance = wl.importance(w).numpy()
+        self.importance = wl.importance(w).numpy() if importance is None else np.asarray(importance, dtype=np.float64)
+        t, r_num, r_den = (w.t, w.r_num, w.r_den) if alloc is None else alloc
+        total = w.total_pages * w.page if total_tokens is None else int(total_tokens)
         self.cap, self.off, self.stride = bk.baklava_allocate(
-            self.shape, self.importance, w.t, 0 if uniform else w.r_num, w.r_den, w.total_pages * w.page,
+            self.shape, self.importance, t, 0 if uniform else r_num, r_den, total,
             w.min_pages * w.page, w.max_pages * w.page)
         self.cache = bk.Cache(self.shape, self.cap, self.off, self.stride, w.B, self.device)
         self.lb, self.le = (0, w.L) if layers is None else layers
@@ -32,10 +37,11 @@ class DecodeSession:
         self.lse = torch.zeros((nl, w.B, w.Hq), dtype=torch.float32, device=self.device)
         self.t = 0
 
-    def prefill_synthetic(self, prompt_len=None):
+    def prefill_synthetic(self, prompt_len=None, data=None):
         """Fill every head from the workload's dense synthetic prompt through baklava_evict, a layer at a time.
-        `prompt_len` (B ints) keeps only that many tokens of each sequence's prompt."""
-        w = self.w
+        `prompt_len` (B ints) keeps only that many tokens of each sequence's prompt; `data` is a copy of the
+        workload with another seed (another prompt through the same heads)."""
+        w = self.w if data is None else data
         ews = torch.empty((bk.baklava_evict_workspace_size(self.shape, w.B, 1, w.T),), dtype=torch.uint8,
                           device=self.device)
         plen = None if prompt_len is None else torch.tensor(list(prompt_len), dtype=torch.int32, device=self.device)

@@ -138,3 +138,12 @@ def test_argument_errors_are_codes_not_crashes():
     L = bk.lib()
     assert L.baklava_decode_attn(None, None, None, None, None, 0, None, None, 0, None, None, None, 0, None) == -1
     assert L.baklava_evict(ctypes.byref(shape), None, 0, 1, None, None, None, 4, 0, 0, 4, 1, None, 0, None) == -1
+
+
+def test_search_pick_matches_oracle_rule():
+    from oracle import search as osearch
+    rng = np.random.default_rng(9)
+    cases = [[3.0, 1.0, 2.0, 1.0], [np.nan, 2.0, np.nan, 1.5], [np.inf, np.inf], [], [0.0], [np.nan]]
+    cases += [list(rng.integers(0, 4, size=n).astype(float)) for n in (2, 5, 17)]
+    for c in cases:
+        assert bk.baklava_search_pick(c) == osearch.pick_best(c), c
