@@ -18,7 +18,7 @@ constexpr int kScoreChunk = 4096;  // target length of a piece of the score / ev
 // Byte offsets of the regions of the decode workspace.
 struct DecodeWorkspace {
     size_t control_off;    // 64 int32: launch-wide counters
-    size_t arrive_off;     // int32 [n_units]: chunks of a head that have delivered their partial result
+    size_t arrive_off;     // int32 [2][n_units]: chunks of a head that have delivered their partial result; head ready flags
     size_t stats_off;      // fp32 [n_units][2 * 8]: final (max, 1 / sum) of each query head, log2 domain
     size_t best_off;       // uint64 [n_score_items] + int32 [n_score_items]: each score piece's eviction candidate
     size_t partial_off;    // fp32 [n_items][g * D + 2 * g + 2]: per-chunk (o, m, l) and its oldest evictable row (pos, slot)

@@ -69,6 +69,7 @@ struct DecodeParams {
     int32_t n_items;
     int32_t n_score_items;
     int32_t* arrive;
+    int32_t* ready;                // [n_units]: 1 once a head's partials are merged and its statistics are final
     float* partial;
     float* logit;
     float* stats;                  // [n_units][2 * kG]
@@ -123,6 +124,14 @@ __device__ __forceinline__ HeadState head_state(const DecodeParams& p, const Uni
 // grid_dependency_wait returns once the previous grid has completed and its writes are visible.
 __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ int ld_acquire(const int32_t* ptr) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int32_t* ptr, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
 
 // K and V are read once per step and never fit in L2: ask L2 to drop them first, so that the
 // step's logits, scores and positions (which the score pass re-reads) stay resident.
@@ -509,8 +518,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         packed.y = *reinterpret_cast<const uint32_t*>(&hi);
         *reinterpret_cast<uint2*>(orow + grp * 4) = packed;
     }
+    __syncthreads();                                        // every thread's share of the output is written
     if (tid == 0) {
         p.arrive[unit] = 0;                                 // the score kernel counts arrivals again
+        // the head is final: its score pieces may start although other heads are still being attended
+        if (keep_logits) st_release(p.ready + unit, 1);
         if (!keep_logits && hs.do_append) {                 // no score pass follows: finish the bookkeeping here
             int victim = -1;
             if (kByPosition && pos_evict) {
@@ -539,6 +551,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
 // the latest token.  The CTA that finishes a head last picks the head's victim among the chunks'
 // candidates and updates len / free_slot.
 constexpr int kScoreThreads = 128;                       // eight rows per thread and sweep
+constexpr int kReadyPolls = 1 << 14;                     // polls of a head's ready flag before falling back
 
 template <int G>
 __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const DecodeParams p) {
@@ -546,6 +559,7 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
     __shared__ unsigned long long sm_key[kScoreThreads / 32];
     __shared__ int sm_slot[kScoreThreads / 32];
     __shared__ int sm_last;
+    __shared__ int sm_ready;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int4 item = p.items[p.n_items + blockIdx.x];
@@ -557,12 +571,25 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
     const HeadState hs = head_state(p, u);
     const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
-    grid_dependency_wait();                               // the attention kernel's scratch and statistics
     if (hs.bad || t_pos < 0) return;                       // reported by the attention kernel / idle sequence
     const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
     if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
+    // This kernel's CTAs become resident while the last attention CTAs are still running.  A piece needs
+    // only its own head: it watches the head's ready flag (set with release semantics by the CTA that merged
+    // the head) instead of waiting for the whole attention grid.  The watch is bounded; if it runs out, the
+    // grid-wide dependency wait below is always sufficient.
+    if (tid == 0) {
+        int ok = 0;
+        for (int i = 0; i < kReadyPolls && !ok; ++i) {
+            ok = ld_acquire(p.ready + unit) != 0;
+            if (!ok) __nanosleep(64);
+        }
+        sm_ready = ok;
+    }
+    __syncthreads();
+    if (!sm_ready) grid_dependency_wait();                // the attention kernel's scratch and statistics
 
     const __half* prob_h = reinterpret_cast<const __half*>(p.logit + row0 * G);
     const float* mref_h = reinterpret_cast<const float*>(prob_h + (int64_t)G * C);
@@ -695,6 +722,7 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
             }
         }
         p.arrive[unit] = 0;
+        p.ready[unit] = 0;                                  // every piece of the head is past its watch
     }
 }
 
@@ -815,6 +843,7 @@ int decode_attn_impl(
     p.n_score_items = info->n_score_items;
     char* base = static_cast<char*>(ws);
     p.arrive = reinterpret_cast<int32_t*>(base + lay.arrive_off);
+    p.ready = p.arrive + info->n_units;
     p.partial = reinterpret_cast<float*>(base + lay.partial_off);
     p.logit = reinterpret_cast<float*>(base + lay.logit_off);
     p.stats = reinterpret_cast<float*>(base + lay.stats_off);
