@@ -13,7 +13,7 @@ constexpr int kMinChunk = 256;      // shortest chunk the automatic plan makes
 __host__ __device__
 #endif
 constexpr int max_merge_entries(int D) { return 64 * D; }
-constexpr int kScoreChunk = 4096;  // target length of a piece of the score / eviction pass
+constexpr int kScoreChunk = 2048;  // target length of a piece of the score / eviction pass
 
 // Byte offsets of the regions of the decode workspace.
 struct DecodeWorkspace {

@@ -63,8 +63,8 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     constexpr int kStageBytes = 2 * kTileBytes;              // K then V
     constexpr uint32_t kOColumn = 2 * kTileRows;             // O sits after the two S buffers in tensor memory
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q, bar_full[2], bar_empty[2], bar_s_full[2], bar_s_empty[2], bar_p_full[2],
-        bar_p_empty[2], bar_o_full;
+    __shared__ __align__(8) uint64_t bar_q, bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2], bar_s_full[2],
+        bar_s_empty[2], bar_p_full[2], bar_p_empty[2], bar_o_full;
     __shared__ uint32_t tmem_slot;
     __shared__ float sm_warp_sum[kSoftmaxWarps];
     __shared__ int sm_abort;
@@ -90,8 +90,10 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
         mbar_init(smem_u32(&bar_q), 1);
         mbar_init(smem_u32(&bar_o_full), 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), 1);
+            mbar_init(smem_u32(&bar_k_full[s]), 1);
+            mbar_init(smem_u32(&bar_k_empty[s]), 1);
+            mbar_init(smem_u32(&bar_v_full[s]), 1);
+            mbar_init(smem_u32(&bar_v_empty[s]), 1);
             mbar_init(smem_u32(&bar_s_full[s]), 1);
             mbar_init(smem_u32(&bar_s_empty[s]), kSoftmaxWarps);
             mbar_init(smem_u32(&bar_p_full[s]), kSoftmaxWarps);
@@ -116,19 +118,25 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
 #pragma unroll
             for (int bx = 0; bx < D / 64; ++bx)
                 tma_load_3d(q_tile + bx * kBoxBytes, &q_map, bx * 64, qb * kTileRows, pr * p.Hq + h, smem_u32(&bar_q));
-            for (int it = 0; it < n_it; ++it) {
+            // K and V rings are released separately: a K tile is free as soon as its S = Q K^T has been
+            // formed (one tile ahead of the softmax), a V tile only after O += P V.  Loads are issued in
+            // the order the MMA thread needs them: K(0), K(1), V(0), K(2), V(1), ...
+            auto load = [&](const CUtensorMap* map, uint64_t* full, uint64_t* empty, uint32_t dst, int it) {
                 const int s = it & 1;
-                if (it >= 2 && !mbar_wait(smem_u32(&bar_empty[s]), ((it >> 1) - 1) & 1)) { sm_abort = 1; break; }
-                const uint32_t bar = smem_u32(&bar_full[s]);
-                mbar_arrive_expect_tx(bar, kStageBytes);
+                if (it >= 2 && !mbar_wait(smem_u32(&empty[s]), ((it >> 1) - 1) & 1)) return false;
+                const uint32_t bar = smem_u32(&full[s]);
+                mbar_arrive_expect_tx(bar, kTileBytes);
 #pragma unroll
-                for (int bx = 0; bx < D / 64; ++bx) {
-                    tma_load_3d(stage0 + s * kStageBytes + bx * kBoxBytes, &k_map, bx * 64, it * kTileRows,
-                                pr * p.Hkv + kvh, bar);
-                    tma_load_3d(stage0 + s * kStageBytes + kTileBytes + bx * kBoxBytes, &v_map, bx * 64, it * kTileRows,
-                                pr * p.Hkv + kvh, bar);
-                }
+                for (int bx = 0; bx < D / 64; ++bx)
+                    tma_load_3d(dst + s * kStageBytes + bx * kBoxBytes, map, bx * 64, it * kTileRows, pr * p.Hkv + kvh, bar);
+                return true;
+            };
+            bool ok = true;
+            for (int it = 0; it <= n_it && ok; ++it) {
+                if (it < n_it) ok = load(&k_map, bar_k_full, bar_k_empty, stage0, it);
+                if (ok && it >= 1) ok = load(&v_map, bar_v_full, bar_v_empty, stage0 + kTileBytes, it - 1);
             }
+            if (!ok) sm_abort = 1;
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer
@@ -138,7 +146,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
             bool ok = mbar_wait(smem_u32(&bar_q), 0);
             auto issue_s = [&](int it) {                     // S_it = Q K_it^T into S buffer it & 1
                 const int s = it & 1;
-                if (!mbar_wait(smem_u32(&bar_full[s]), (it >> 1) & 1)) return false;
+                if (!mbar_wait(smem_u32(&bar_k_full[s]), (it >> 1) & 1)) return false;
                 if (it >= 2 && !mbar_wait(smem_u32(&bar_s_empty[s]), ((it >> 1) - 1) & 1)) return false;
                 tc::fence_after_sync();
                 const uint32_t k_tile = stage0 + s * kStageBytes;
@@ -148,6 +156,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                     tc::umma_bf16(tmem_base + s * kTileRows, tc::desc_k_major_sw128(q_tile + off),
                                   tc::desc_k_major_sw128(k_tile + off), idesc_s, ks > 0);
                 }
+                tc::umma_commit(smem_u32(&bar_k_empty[s]));  // the K tile may be overwritten
                 tc::umma_commit(smem_u32(&bar_s_full[s]));
                 return true;
             };
@@ -155,6 +164,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
             for (int it = 0; it < n_it && ok; ++it) {
                 const int s = it & 1;
                 if (it + 1 < n_it) ok = issue_s(it + 1);     // the next tile's logits while this tile's softmax runs
+                if (ok) ok = mbar_wait(smem_u32(&bar_v_full[s]), (it >> 1) & 1);
                 if (ok) ok = mbar_wait(smem_u32(&bar_p_full[s]), (it >> 1) & 1);
                 if (!ok) break;
                 tc::fence_after_sync();
@@ -166,7 +176,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                     tc::umma_bf16(tmem_base + kOColumn, tc::desc_k_major_sw128(p_tile + p_off),
                                   tc::desc_mn_major_sw128(v_tile + ks * 2048, kBoxBytes), idesc_o, (it > 0) || (ks > 0));
                 }
-                tc::umma_commit(smem_u32(&bar_empty[s]));    // K and V of this stage are consumed
+                tc::umma_commit(smem_u32(&bar_v_empty[s]));  // the V tile of this stage is consumed
                 tc::umma_commit(smem_u32(&bar_p_empty[s]));  // so is the probability tile
             }
             if (ok) tc::umma_commit(smem_u32(&bar_o_full));
