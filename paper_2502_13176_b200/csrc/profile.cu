@@ -6,9 +6,11 @@
 // (the row pass of the prompt-score kernels).  The second owns 128 query rows per CTA: the Q tile stays
 // in shared memory, K and V tiles of 128 keys stream through a two-stage TMA ring; one thread issues
 // S = Q K^T into tensor memory (double-buffered), sixteen softmax warps read S back, form the already
-// normalised probabilities exp2(s - lse) in bf16 and store them as the next MMA's A operand in shared
-// memory, and the same thread issues O += P V with V as an MN-major B operand; O accumulates in tensor
-// memory over all key tiles and is never written.  The last key tile is the diagonal one, whose V rows
+// normalised probabilities exp2(s - lse) in bf16 and write them back to tensor memory, from where the next
+// MMA takes them as its A operand (shared-memory bandwidth is the scarce resource of this kernel: a
+// 128 x 128 MMA with both operands in shared memory uses all of it), and the same thread issues
+// O += P V with V as an MN-major B operand; O accumulates in tensor memory over all key tiles and is
+// never written.  The last key tile is the diagonal one, whose V rows
 // are exactly the rows the cosine needs, so the final epilogue reads them from shared memory.
 // Per-CTA cosine sums go to the workspace and a small kernel adds them in a fixed order.
 #include <cmath>
@@ -25,7 +27,7 @@ using namespace ptx;
 constexpr int kTileRows = 128;        // query rows per CTA = keys per streamed tile
 constexpr int kSoftmaxWarps = 16;     // four threads per query row, 32 keys of a tile each
 constexpr int kThreads = (2 + kSoftmaxWarps) * 32;   // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, then softmax
-constexpr uint32_t kTmemColumns = 512;    // S: 2 x 128 columns, O: D columns
+constexpr uint32_t kTmemColumns = 512;    // S: 2 x 128 columns, O: D columns (at most 128), P: 2 x 64 columns
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kCosEps = 1e-12f;
 
@@ -59,9 +61,10 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     constexpr int kPvSteps = kTileRows / 16;                 // MMA steps over the keys (O += P V)
     constexpr int kBoxBytes = kTileRows * 128;               // one TMA box: 128 rows x 64 elements
     constexpr int kTileBytes = kTileRows * D * 2;            // a Q, K or V tile
-    constexpr int kPBytes = kTileRows * kTileRows * 2;       // a probability tile: 128 queries x 128 keys, bf16
     constexpr int kStageBytes = 2 * kTileBytes;              // K then V
     constexpr uint32_t kOColumn = 2 * kTileRows;             // O sits after the two S buffers in tensor memory
+    constexpr uint32_t kPColumn = 3 * kTileRows;             // then two probability tiles: 128 keys in bf16 = 64 columns
+    constexpr uint32_t kPColumns = kTileRows / 2;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_q, bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2], bar_s_full[2],
         bar_s_empty[2], bar_p_full[2], bar_p_empty[2], bar_o_full;
@@ -84,7 +87,6 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t q_tile = base;
     const uint32_t stage0 = base + kTileBytes;
-    const uint32_t p_tile0 = stage0 + 2 * kStageBytes;
 
     if (tid == 0) {
         mbar_init(smem_u32(&bar_q), 1);
@@ -169,12 +171,10 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                 if (!ok) break;
                 tc::fence_after_sync();
                 const uint32_t v_tile = stage0 + s * kStageBytes + kTileBytes;
-                const uint32_t p_tile = p_tile0 + s * kPBytes;
 #pragma unroll
-                for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step
-                    const uint32_t p_off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-                    tc::umma_bf16(tmem_base + kOColumn, tc::desc_k_major_sw128(p_tile + p_off),
-                                  tc::desc_mn_major_sw128(v_tile + ks * 2048, kBoxBytes), idesc_o, (it > 0) || (ks > 0));
+                for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step = 8 columns of the probability tile
+                    tc::umma_bf16_ts(tmem_base + kOColumn, tmem_base + kPColumn + s * kPColumns + ks * 8,
+                                     tc::desc_mn_major_sw128(v_tile + ks * 2048, kBoxBytes), idesc_o, (it > 0) || (ks > 0));
                 }
                 tc::umma_commit(smem_u32(&bar_v_empty[s]));  // the V tile of this stage is consumed
                 tc::umma_commit(smem_u32(&bar_p_empty[s]));  // so is the probability tile
@@ -205,27 +205,20 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                 for (int c = 0; c < 32; ++c)
                     if (col_base + c > row) v[c] = 0xff800000u;
             }
-            // probabilities of this thread's 32 keys -> bf16 -> the K-major, 128-byte-swizzled A tile
-            uint8_t* p_row = base_ptr + (p_tile0 - base) + s * kPBytes + (part >> 1) * kBoxBytes + row * 128;
-#pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {                  // 16-byte pieces of 8 keys
-                uint32_t w[4];
-#pragma unroll
-                for (int k2 = 0; k2 < 4; ++k2) {
-                    const int c = cc * 8 + k2 * 2;
-                    w[k2] = pack_bf16(fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -lse)),
-                                      fast_exp2(fmaf(__uint_as_float(v[c + 1]), p.scale_log2, -lse)));
-                }
-                const int piece = (part & 1) * 4 + cc;        // inside the 64-key box
-                *reinterpret_cast<uint4*>(p_row + ((piece ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            tc::fence_proxy_async_smem();
             tc::fence_before_sync();
             __syncwarp();
-            if (lane == 0) {
-                tc::mbar_arrive(smem_u32(&bar_p_full[s]));
-                tc::mbar_arrive(smem_u32(&bar_s_empty[s]));
-            }
+            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_s_empty[s]));    // the logits are in registers
+            // probabilities of this thread's 32 keys -> bf16, two per 32-bit column of the A operand
+            uint32_t w[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+                w[c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(v[2 * c]), p.scale_log2, -lse)),
+                                 fast_exp2(fmaf(__uint_as_float(v[2 * c + 1]), p.scale_log2, -lse)));
+            tc::tmem_st_32x32_x16(lane_addr + kPColumn + s * kPColumns + part * 16, w);
+            tc::tmem_st_wait();
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_p_full[s]));
         }
         // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile.
         // Four threads per row take 32 columns of the head dimension each (two of them when D = 64).
@@ -253,8 +246,8 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                 }
             }
         }
-        // join the four parts of every row through shared memory (the probability tiles are idle now)
-        float* sm_part = reinterpret_cast<float*>(base_ptr + (p_tile0 - base));      // [3][4][128]
+        // join the four parts of every row through shared memory (the stage without the diagonal tile is idle)
+        float* sm_part = reinterpret_cast<float*>(base_ptr + (stage0 - base) + ((qb & 1) ^ 1) * kStageBytes);   // [3][4][128]
         sm_part[(0 * 4 + part) * kTileRows + row] = dot;
         sm_part[(1 * 4 + part) * kTileRows + row] = vv;
         sm_part[(2 * 4 + part) * kTileRows + row] = oo;
@@ -301,8 +294,8 @@ __global__ void profile_mean_kernel(const ProfileParams p) {
 template <int D>
 cudaError_t launch_profile(const ProfileParams& p, const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
                            cudaStream_t s) {
-    // Q tile, two (K, V) stages, two probability tiles
-    constexpr int kSmem = kTileRows * D * 2 * 5 + 2 * kTileRows * kTileRows * 2 + 1024;
+    // Q tile and two (K, V) stages
+    constexpr int kSmem = kTileRows * D * 2 * 5 + 1024;
     cudaError_t e = cudaFuncSetAttribute(profile_pv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const dim3 grid(p.n_blk, p.Hq, p.P);
