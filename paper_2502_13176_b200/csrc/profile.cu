@@ -4,7 +4,7 @@
 //
 // Two launches on the 5th-generation tensor cores.  The first gives every query row its log-sum-exp
 // (the row pass of the prompt-score kernels).  The second owns 128 query rows per CTA: the Q tile stays
-// in shared memory, K and V tiles of 128 keys stream through a two-stage TMA ring; one thread issues
+// in shared memory, K and V tiles of 128 keys stream through three-stage TMA rings; one thread issues
 // S = Q K^T into tensor memory (double-buffered), sixteen softmax warps read S back, form the already
 // normalised probabilities exp2(s - lse) in bf16 and write them back to tensor memory, from where the next
 // MMA takes them as its A operand (shared-memory bandwidth is the scarce resource of this kernel: a
@@ -27,6 +27,8 @@ using namespace ptx;
 constexpr int kTileRows = 128;        // query rows per CTA = keys per streamed tile
 constexpr int kSoftmaxWarps = 16;     // four threads per query row, 32 keys of a tile each
 constexpr int kThreads = (2 + kSoftmaxWarps) * 32;   // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, then softmax
+constexpr int kGroupRing = 4;         // mbarriers that track the MMA groups in flight
+constexpr int kKvStages = 3;          // K and V tiles in flight: the streamed operands come from L2 at a bounded rate
 constexpr uint32_t kTmemColumns = 512;    // S: 2 x 128 columns, O: D columns (at most 128), P: 2 x 64 columns
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kCosEps = 1e-12f;
@@ -66,8 +68,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     constexpr uint32_t kPColumn = 3 * kTileRows;             // then two probability tiles: 128 keys in bf16 = 64 columns
     constexpr uint32_t kPColumns = kTileRows / 2;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q, bar_k_full[2], bar_k_empty[2], bar_v_full[2], bar_v_empty[2], bar_s_full[2],
-        bar_s_empty[2], bar_p_full[2], bar_p_empty[2], bar_o_full;
+    __shared__ __align__(8) uint64_t bar_q, bar_k01[2], bar_in[kGroupRing], bar_group[kGroupRing];
     __shared__ uint32_t tmem_slot;
     __shared__ float sm_warp_sum[kSoftmaxWarps];
     __shared__ int sm_abort;
@@ -90,16 +91,10 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
 
     if (tid == 0) {
         mbar_init(smem_u32(&bar_q), 1);
-        mbar_init(smem_u32(&bar_o_full), 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&bar_k_full[s]), 1);
-            mbar_init(smem_u32(&bar_k_empty[s]), 1);
-            mbar_init(smem_u32(&bar_v_full[s]), 1);
-            mbar_init(smem_u32(&bar_v_empty[s]), 1);
-            mbar_init(smem_u32(&bar_s_full[s]), 1);
-            mbar_init(smem_u32(&bar_s_empty[s]), kSoftmaxWarps);
-            mbar_init(smem_u32(&bar_p_full[s]), kSoftmaxWarps);
-            mbar_init(smem_u32(&bar_p_empty[s]), 1);
+        for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&bar_k01[s]), 1);
+        for (int s = 0; s < kGroupRing; ++s) {
+            mbar_init(smem_u32(&bar_in[s]), kSoftmaxWarps + 2);   // P(it) written, V(it) landed, K(it + 2) landed
+            mbar_init(smem_u32(&bar_group[s]), 1);
         }
         sm_abort = 0;
         fence_mbar_init();
@@ -112,6 +107,9 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     __syncthreads();
     tc::fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
+    // completion of MMA group g (see the MMA issuer); a slot of the ring is reused four groups later,
+    // and no waiter can be that far behind
+    auto group_wait = [&](int g) { return mbar_wait(smem_u32(&bar_group[g % kGroupRing]), (g / kGroupRing) & 1); };
 
     if (warp == 0) {
         // ---------------- TMA producer
@@ -120,23 +118,28 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
 #pragma unroll
             for (int bx = 0; bx < D / 64; ++bx)
                 tma_load_3d(q_tile + bx * kBoxBytes, &q_map, bx * 64, qb * kTileRows, pr * p.Hq + h, smem_u32(&bar_q));
-            // K and V rings are released separately: a K tile is free as soon as its S = Q K^T has been
-            // formed (one tile ahead of the softmax), a V tile only after O += P V.  Loads are issued in
-            // the order the MMA thread needs them: K(0), K(1), V(0), K(2), V(1), ...
-            auto load = [&](const CUtensorMap* map, uint64_t* full, uint64_t* empty, uint32_t dst, int it) {
-                const int s = it & 1;
-                if (it >= 2 && !mbar_wait(smem_u32(&empty[s]), ((it >> 1) - 1) & 1)) return false;
-                const uint32_t bar = smem_u32(&full[s]);
+            // The single MMA thread pays well over a hundred cycles for every mbarrier it looks at, so
+            // everything group it + 2 = { P(it) V(it), S(it + 2) } needs arrives on ONE barrier, bar_in[it % 4]:
+            // the sixteen softmax warps (P(it) written) and the two loads V(it) and K(it + 2).
+            // K(j) reuses the stage of K(j - 3), consumed by S(j - 3) = MMA group j - 3; V(j) the stage of
+            // V(j - 3), consumed by P V of tile j - 3 = MMA group j - 1: both loads of bar_in[j % 4] wait for
+            // group j - 1.
+            auto load = [&](const CUtensorMap* map, uint32_t bar, uint32_t dst, int it) {
                 mbar_arrive_expect_tx(bar, kTileBytes);
 #pragma unroll
                 for (int bx = 0; bx < D / 64; ++bx)
-                    tma_load_3d(dst + s * kStageBytes + bx * kBoxBytes, map, bx * 64, it * kTileRows, pr * p.Hkv + kvh, bar);
-                return true;
+                    tma_load_3d(dst + (it % kKvStages) * kStageBytes + bx * kBoxBytes, map, bx * 64, it * kTileRows,
+                                pr * p.Hkv + kvh, bar);
             };
+            for (int j = 0; j < 2 && j < n_it; ++j) load(&k_map, smem_u32(&bar_k01[j]), stage0, j);
             bool ok = true;
-            for (int it = 0; it <= n_it && ok; ++it) {
-                if (it < n_it) ok = load(&k_map, bar_k_full, bar_k_empty, stage0, it);
-                if (ok && it >= 1) ok = load(&v_map, bar_v_full, bar_v_empty, stage0 + kTileBytes, it - 1);
+            for (int j = 0; j < n_it && ok; ++j) {
+                if (j >= 1) ok = group_wait(j - 1);           // (K(3) and K(4) already reuse a stage)
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&bar_in[j % kGroupRing]);
+                load(&v_map, bar, stage0 + kTileBytes, j);
+                if (j + 2 < n_it) load(&k_map, bar, stage0, j + 2);
+                else tc::mbar_arrive(bar);
             }
             if (!ok) sm_abort = 1;
         }
@@ -145,42 +148,45 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
         if (lane == 0) {
             constexpr uint32_t idesc_s = tc::idesc_bf16_f32(kTileRows, kTileRows);      // S[128 q x 128 keys]
             constexpr uint32_t idesc_o = tc::idesc_bf16_f32_b_mn(kTileRows, D);         // O[128 q x D]
+            // A tcgen05.commit occupies the tensor pipe for about as long as a quarter of a 128 x 128 x 128
+            // MMA, so the work is issued in groups with ONE commit each: group 0 = S(0), group 1 = S(1),
+            // group it + 2 = { O += P(it) V(it), S(it + 2) }.  Completion of group g therefore tells the
+            // softmax warps that S(g) is ready and that the probability buffer of tile g - 2 is free, and
+            // the producer that K(g) and V(g - 2) are consumed.
             bool ok = mbar_wait(smem_u32(&bar_q), 0);
             auto issue_s = [&](int it) {                     // S_it = Q K_it^T into S buffer it & 1
-                const int s = it & 1;
-                if (!mbar_wait(smem_u32(&bar_k_full[s]), (it >> 1) & 1)) return false;
-                if (it >= 2 && !mbar_wait(smem_u32(&bar_s_empty[s]), ((it >> 1) - 1) & 1)) return false;
-                tc::fence_after_sync();
-                const uint32_t k_tile = stage0 + s * kStageBytes;
+                const int s = it & 1, kv = it % kKvStages;
+                const uint32_t k_tile = stage0 + kv * kStageBytes;
 #pragma unroll
                 for (int ks = 0; ks < kKSteps; ++ks) {
                     const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
                     tc::umma_bf16(tmem_base + s * kTileRows, tc::desc_k_major_sw128(q_tile + off),
                                   tc::desc_k_major_sw128(k_tile + off), idesc_s, ks > 0);
                 }
-                tc::umma_commit(smem_u32(&bar_k_empty[s]));  // the K tile may be overwritten
-                tc::umma_commit(smem_u32(&bar_s_full[s]));
-                return true;
             };
-            if (ok) ok = issue_s(0);
-            for (int it = 0; it < n_it && ok; ++it) {
-                const int s = it & 1;
-                if (it + 1 < n_it) ok = issue_s(it + 1);     // the next tile's logits while this tile's softmax runs
-                if (ok) ok = mbar_wait(smem_u32(&bar_v_full[s]), (it >> 1) & 1);
-                if (ok) ok = mbar_wait(smem_u32(&bar_p_full[s]), (it >> 1) & 1);
+            for (int g = 0; g < 2 && g < n_it && ok; ++g) {
+                ok = mbar_wait(smem_u32(&bar_k01[g]), 0);
                 if (!ok) break;
                 tc::fence_after_sync();
-                const uint32_t v_tile = stage0 + s * kStageBytes + kTileBytes;
+                issue_s(g);
+                tc::umma_commit(smem_u32(&bar_group[g % kGroupRing]));
+            }
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int s = it & 1, kv = it % kKvStages;
+                // P(it) is written (so S(it) has been read), V(it) and K(it + 2) have landed
+                ok = mbar_wait(smem_u32(&bar_in[it % kGroupRing]), (it / kGroupRing) & 1);
+                if (!ok) break;
+                tc::fence_after_sync();
+                const uint32_t v_tile = stage0 + kv * kStageBytes + kTileBytes;
 #pragma unroll
                 for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step = 8 columns of the probability tile
                     tc::umma_bf16_ts(tmem_base + kOColumn, tmem_base + kPColumn + s * kPColumns + ks * 8,
                                      tc::desc_mn_major_sw128(v_tile + ks * 2048, kBoxBytes), idesc_o, (it > 0) || (ks > 0));
                 }
-                tc::umma_commit(smem_u32(&bar_v_empty[s]));  // the V tile of this stage is consumed
-                tc::umma_commit(smem_u32(&bar_p_empty[s]));  // so is the probability tile
+                if (it + 2 < n_it) issue_s(it + 2);          // into the S buffer tile `it` has just left
+                tc::umma_commit(smem_u32(&bar_group[(it + 2) % kGroupRing]));
             }
-            if (ok) tc::umma_commit(smem_u32(&bar_o_full));
-            else sm_abort = 1;
+            if (!ok) sm_abort = 1;
         }
     } else {
         // ---------------- softmax warps: a warp reads its quarter of the TMEM lanes (thread = query row);
@@ -194,8 +200,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
         bool ok = true;
         for (int it = 0; it < n_it; ++it) {
             const int s = it & 1;
-            if (!mbar_wait(smem_u32(&bar_s_full[s]), (it >> 1) & 1)) { ok = false; break; }
-            if (it >= 2 && !mbar_wait(smem_u32(&bar_p_empty[s]), ((it >> 1) - 1) & 1)) { ok = false; break; }
+            if (!group_wait(it)) { ok = false; break; }        // S(it) is ready and P V of tile it - 2 has read its P
             tc::fence_after_sync();
             uint32_t v[32];
             tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base, v);
@@ -205,9 +210,6 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                 for (int c = 0; c < 32; ++c)
                     if (col_base + c > row) v[c] = 0xff800000u;
             }
-            tc::fence_before_sync();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_s_empty[s]));    // the logits are in registers
             // probabilities of this thread's 32 keys -> bf16, two per 32-bit column of the A operand
             uint32_t w[16];
 #pragma unroll
@@ -218,15 +220,15 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
             tc::tmem_st_wait();
             tc::fence_before_sync();
             __syncwarp();
-            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_p_full[s]));
+            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_in[it % kGroupRing]));
         }
         // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile.
         // Four threads per row take 32 columns of the head dimension each (two of them when D = 64).
-        if (ok) ok = mbar_wait(smem_u32(&bar_o_full), 0);
+        if (ok) ok = group_wait(n_it + 1);                    // the last group: O is complete
         float dot = 0.0f, vv = 0.0f, oo = 0.0f;
         if (ok && part * 32 < D) {
             tc::fence_after_sync();
-            const uint8_t* v_row = base_ptr + (stage0 - base) + (qb & 1) * kStageBytes + kTileBytes + row * 128;
+            const uint8_t* v_row = base_ptr + (stage0 - base) + (qb % kKvStages) * kStageBytes + kTileBytes + row * 128;
             uint32_t o[32];
             tc::tmem_ld_32x32(lane_addr + kOColumn + part * 32, o);
             tc::tmem_ld_wait();
@@ -247,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
             }
         }
         // join the four parts of every row through shared memory (the stage without the diagonal tile is idle)
-        float* sm_part = reinterpret_cast<float*>(base_ptr + (stage0 - base) + ((qb & 1) ^ 1) * kStageBytes);   // [3][4][128]
+        float* sm_part = reinterpret_cast<float*>(base_ptr + (stage0 - base) + ((qb + 1) % kKvStages) * kStageBytes);   // [3][4][128]
         sm_part[(0 * 4 + part) * kTileRows + row] = dot;
         sm_part[(1 * 4 + part) * kTileRows + row] = vv;
         sm_part[(2 * 4 + part) * kTileRows + row] = oo;
@@ -294,8 +296,8 @@ __global__ void profile_mean_kernel(const ProfileParams p) {
 template <int D>
 cudaError_t launch_profile(const ProfileParams& p, const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
                            cudaStream_t s) {
-    // Q tile and two (K, V) stages
-    constexpr int kSmem = kTileRows * D * 2 * 5 + 1024;
+    // Q tile and the (K, V) stages
+    constexpr int kSmem = kTileRows * D * 2 * (1 + 2 * kKvStages) + 1024;
     cudaError_t e = cudaFuncSetAttribute(profile_pv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const dim3 grid(p.n_blk, p.Hq, p.P);
