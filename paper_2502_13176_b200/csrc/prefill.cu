@@ -26,7 +26,7 @@ constexpr int kThreads = 320;        // warp 0: TMA producer, warp 1: MMA issuer
 constexpr int kEpilogueThreads = 256; // two threads per accumulator row, 64 columns each
 constexpr uint32_t kTmemColumns = 256;   // two 128-column accumulators
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kPassLse = 0, kPassColumnSums = 1;
+constexpr int kPassLse = 0, kPassColumnSums = 1, kPassRowMax = 2;   // row passes: kPassLse and kPassRowMax
 
 // 2^x on the special-function unit (one instruction; -inf gives 0)
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
     const int b = blockIdx.z;
     const int len = p.prompt_len ? min(max(p.prompt_len[b], 0), p.T) : p.T;
     int blk, n_it, nq = 1, head_res, head_first;            // resident block, streamed tiles, heads
-    if (PASS == kPassLse) {
+    if (PASS != kPassColumnSums) {
         blk = p.n_blk - 1 - blockIdx.x;                     // long rows of the causal triangle first
         const int h = blockIdx.y;
         head_res = b * p.Hq + h;
@@ -109,14 +109,14 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
     const uint32_t tmem_base = tmem_slot;
 
     // which streamed tile iteration `it` is: (head of the group, row block)
-    auto stream_head = [&](int it) { return PASS == kPassLse ? head_first : head_first + it / nq; };
-    auto stream_blk = [&](int it) { return PASS == kPassLse ? it : blk + it % nq; };
+    auto stream_head = [&](int it) { return PASS != kPassColumnSums ? head_first : head_first + it / nq; };
+    auto stream_blk = [&](int it) { return PASS != kPassColumnSums ? it : blk + it % nq; };
 
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            const CUtensorMap* res_map = PASS == kPassLse ? &q_map : &k_map;
-            const CUtensorMap* str_map = PASS == kPassLse ? &k_map : &q_map;
+            const CUtensorMap* res_map = PASS != kPassColumnSums ? &q_map : &k_map;
+            const CUtensorMap* str_map = PASS != kPassColumnSums ? &k_map : &q_map;
             mbar_arrive_expect_tx(smem_u32(&bar_res), kTileBytes);
 #pragma unroll
             for (int bx = 0; bx < D / 64; ++bx)
@@ -150,8 +150,9 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
                     tc::umma_bf16(tmem_base + s * kTileRows, tc::desc_k_major_sw128(res_tile + off),
                                   tc::desc_k_major_sw128(str_tile + off), idesc, ks > 0);
                 }
-                tc::umma_commit(smem_u32(&bar_empty[s]));        // the stage may be overwritten
-                tc::umma_commit(smem_u32(&bar_acc_full[s]));     // the accumulator may be read
+                // one commit per tile (a commit costs the tensor pipe about as much as a third of this tile's
+                // MMAs): the epilogue, which sees the accumulator complete, releases the stage for the producer
+                tc::umma_commit(smem_u32(&bar_acc_full[s]));
             }
             if (!ok) sm_abort = 1;
         }
@@ -178,10 +179,28 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
             float next_lse = 0.0f;
             if (PASS == kPassColumnSums && e < kTileRows && it + 1 < n_it) next_lse = fetch_lse(it + 1);
             if (!mbar_wait(smem_u32(&bar_acc_full[s]), (it >> 1) & 1)) { ok = false; break; }
+            if (tid == 64) tc::mbar_arrive(smem_u32(&bar_empty[s]));       // the MMAs have read the streamed tile
             tc::fence_after_sync();
             const bool diagonal = stream_blk(it) == blk;
             const uint32_t acc = lane_addr + s * kTileRows;
-            if (PASS == kPassLse) {
+            if (PASS == kPassRowMax) {
+                // row = query, columns = keys: only the largest logit of the row is wanted (no exponentials)
+#pragma unroll
+                for (int c0 = 0; c0 < kTileRows / 2; c0 += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld_32x32(acc + c0, v);
+                    tc::tmem_ld_wait();
+                    if (diagonal) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (col_base + c0 + c > row) v[c] = 0xff800000u;    // -inf
+                    }
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) mx[c & 3] = fmaxf(mx[c & 3], __uint_as_float(v[c]));
+                    m_run = fmaxf(m_run, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])));
+                }
+            } else if (PASS == kPassLse) {
                 // row = query, columns = keys: keys above the query are masked on the diagonal tile.
                 // Online softmax statistics, 32 columns at a time.
 #pragma unroll
@@ -240,13 +259,16 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
         }
         // join the two halves of every row: the upper half hands its state over through shared memory
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (half == 1) { sm_lse[0][row] = PASS == kPassLse ? m_run : colsum; sm_lse[1][row] = l_run; }
+        if (half == 1) { sm_lse[0][row] = PASS != kPassColumnSums ? m_run : colsum; sm_lse[1][row] = l_run; }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (!ok) {
             sm_abort = 1;
         } else if (half == 0) {
             const int t = blk * kTileRows + row;
-            if (PASS == kPassLse) {
+            if (PASS == kPassRowMax) {
+                // scaled to the log2 domain like the log-sum-exp it stands in for
+                if (t < p.T) p.lse2[(int64_t)head_res * p.T + t] = t < len ? fmaxf(m_run, sm_lse[0][row]) * p.scale_log2 : INFINITY;
+            } else if (PASS == kPassLse) {
                 const float m_hi = sm_lse[0][row], l_hi = sm_lse[1][row];
                 const float m_all = fmaxf(m_run, m_hi);      // m_run is finite: column 0 belongs to the lower half
                 const float l_all = l_run * exp2f(m_run - m_all) + (m_hi == -INFINITY ? 0.0f : l_hi * exp2f(m_hi - m_all));
@@ -284,8 +306,10 @@ cudaError_t launch_prefill(const PrefillParams& p, const CUtensorMap& qm, const 
 
 }  // namespace
 
-// Pass 1 alone, for the profiling kernel: log2-domain log-sum-exp of every causal query row.
-int baklava_launch_row_lse(const baklava_shape* shape, const void* q, const void* k, const int32_t* prompt_len,
+// A row pass alone, for the profiling kernel: log2-domain largest logit of every causal query row
+// (+inf past the prompt).  The cosine of Algorithm 1 does not depend on the scale of a head's output
+// row, so the row maximum serves as the softmax's stabiliser and its sum is never needed.
+int baklava_launch_row_max(const baklava_shape* shape, const void* q, const void* k, const int32_t* prompt_len,
                            int32_t B, int32_t T, float* lse2, uint32_t* error, cudaStream_t s) {
     PrefillParams p;
     p.prompt_len = prompt_len;
@@ -299,8 +323,8 @@ int baklava_launch_row_lse(const baklava_shape* shape, const void* q, const void
     if (!make_head_map(&qm, q, (int64_t)B * shape->Hq, T, shape->D, kTileRows) ||
         !make_head_map(&km, k, (int64_t)B * shape->Hkv, T, shape->D, kTileRows))
         return BAKLAVA_ERR_CUDA;
-    cudaError_t e = shape->D == 128 ? launch_pass<128, kPassLse>(p, qm, km, dim3(p.n_blk, p.Hq, B), s)
-                                    : launch_pass<64, kPassLse>(p, qm, km, dim3(p.n_blk, p.Hq, B), s);
+    cudaError_t e = shape->D == 128 ? launch_pass<128, kPassRowMax>(p, qm, km, dim3(p.n_blk, p.Hq, B), s)
+                                    : launch_pass<64, kPassRowMax>(p, qm, km, dim3(p.n_blk, p.Hq, B), s);
     return e == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
 }
 

@@ -2,16 +2,17 @@
 // causal softmax attention O = softmax(Q K^T / sqrt(D)) V and the token-wise cosine between the
 // head's input V_t and its output O_t, averaged over the prompt's tokens.
 //
-// Two launches on the 5th-generation tensor cores.  The first gives every query row its log-sum-exp
-// (the row pass of the prompt-score kernels).  The second owns 128 query rows per CTA: the Q tile stays
-// in shared memory, K and V tiles of 128 keys stream through three-stage TMA rings; one thread issues
-// S = Q K^T into tensor memory (double-buffered), sixteen softmax warps read S back, form the already
-// normalised probabilities exp2(s - lse) in bf16 and write them back to tensor memory, from where the next
-// MMA takes them as its A operand (shared-memory bandwidth is the scarce resource of this kernel: a
-// 128 x 128 MMA with both operands in shared memory uses all of it), and the same thread issues
-// O += P V with V as an MN-major B operand; O accumulates in tensor memory over all key tiles and is
-// never written.  The last key tile is the diagonal one, whose V rows
-// are exactly the rows the cosine needs, so the final epilogue reads them from shared memory.
+// Two launches on the 5th-generation tensor cores.  The first gives every query row its largest logit
+// (a row pass of the prompt-score kernels, without exponentials).  That is all the softmax needs here:
+// the cosine does not change when a row of O is scaled, so the probabilities are left unnormalised,
+// p = exp2(s - max) <= 1, and O never needs rescaling or dividing.  The second launch owns 128 query rows
+// per CTA: the Q tile stays in shared memory, K and V tiles of 128 keys stream through three-stage TMA
+// rings; one thread issues S = Q K^T into tensor memory (double-buffered), sixteen softmax warps read S
+// back, form the probabilities in bf16 and write them back to tensor memory, from where the next MMA takes
+// them as its A operand, and the same thread issues O += P V with V as an MN-major B operand; O
+// accumulates in tensor memory over all key tiles and is never written.  The last key tile is the
+// diagonal one, whose V rows are exactly the rows the cosine needs, so the final epilogue reads them from
+// shared memory.
 // Per-CTA cosine sums go to the workspace and a small kernel adds them in a fixed order.
 #include <cmath>
 #include <cstdint>
@@ -35,7 +36,7 @@ constexpr float kCosEps = 1e-12f;
 
 struct ProfileParams {
     const int32_t* prompt_len;   // [P] or null
-    const float* lse2;           // [P, Hq, T] from the row pass
+    const float* lse2;           // [P, Hq, T] from the row pass: every row's largest logit, log2 domain
     float* head_cos;             // [P, Hq]
     float* token_cos;            // [P, Hq, T] or null
     float* block_sum;            // [P, Hq, n_blk]
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
         const int col_base = part * 32;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
         const int t = qb * kTileRows + row;
-        const float lse = t < p.T ? p.lse2[((int64_t)pr * p.Hq + h) * p.T + t] : INFINITY;   // +inf past the prompt
+        const float lse = t < p.T ? p.lse2[((int64_t)pr * p.Hq + h) * p.T + t] : INFINITY;   // row maximum; +inf past the prompt
         bool ok = true;
         for (int it = 0; it < n_it; ++it) {
             const int s = it & 1;
@@ -347,7 +348,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_profile_heads(
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 256, s) != cudaSuccess) return BAKLAVA_ERR_CUDA;
-    rc = baklava_launch_row_lse(shape, q, k, prompt_len, P, T, lse2, p.error, s);
+    rc = baklava_launch_row_max(shape, q, k, prompt_len, P, T, lse2, p.error, s);
     if (rc) return rc;
     cudaError_t err = shape->D == 128 ? launch_profile<128>(p, qm, km, vm, s) : launch_profile<64>(p, qm, km, vm, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
