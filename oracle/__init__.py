@@ -15,6 +15,7 @@ the paper's order and notation:
   cache.py       Eq. 4-7 iterated        one head's slab and one decode step
   prefill.py     Eq. 1 column sums       accumulated attention a prompt leaves on its tokens
   search.py      Algorithm 3             parameter search loop with an attention-output loss
+  fp8.py         quantised slabs         FP8 E4M3 codec and the per-head scale rule
 
 Parity status: every function is pinned by the CPU tests (closed forms,
 library routines, brute force, invariants).  The search loop and its loss are
