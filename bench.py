@@ -288,6 +288,8 @@ def main():
     ap.add_argument("--policy", default="heavy", choices=["heavy", "window"],
                     help="heavy: sinks + window + accumulated-attention heavy hitters (default); "
                          "window: the paper's evaluated sinks + window policy, run without scores")
+    ap.add_argument("--kv", default="bf16", choices=["bf16", "fp8"],
+                    help="slab format: bf16 (the headline) or FP8 E4M3 with per-head scales (half the bytes per row)")
     ap.add_argument("--mixed-lengths", action="store_true",
                     help="prompts of different lengths (seeded, uniform in [T/8, T]) decoded at per-sequence "
                          "positions through baklava_decode_attn_varlen")
@@ -319,7 +321,10 @@ def main():
 
     bk.lib()                                             # fail now if the library is missing
     step_flags = bk.FLAG_NO_SCORE if args.policy == "window" else 0
-    sess = DecodeSession(w, dev, chunk_tokens=args.chunk)
+    sess = DecodeSession(w, dev, chunk_tokens=args.chunk,
+                         kv_dtype=bk.KV_FP8_E4M3 if args.kv == "fp8" else bk.KV_BF16)
+    if args.kv == "fp8":
+        w = wl.scaled(w, name=w.name + "-fp8")
     total = args.warmup + args.steps
     if args.mixed_lengths:
         from paper_2502_13176_b200 import synth
@@ -391,7 +396,7 @@ def main():
     elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e_ms], dev)
 
     if rank == 0:
-        bytes_per_step = rows_per_step * w.D * 2 * 2          # K and V rows, bf16
+        bytes_per_step = rows_per_step * w.D * 2 * (1 if args.kv == "fp8" else 2)   # K and V rows, bf16 or one byte
         gbs = whole_job_rate(world, bytes_per_step, args.steps, elapsed_ms) / 1e9
         e2e_gbs = whole_job_rate(world, bytes_per_step, args.steps, e2e_ms) / 1e9
         peak, peak_kind = measured_peaks()
@@ -400,7 +405,8 @@ def main():
         line = {
             "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if args.kv == "bf16" else "fp8-e4m3 slabs, fp16 MMA",
+            "data": "synthetic",
             "config": {"workload": w.name, "layers": w.L, "batch": w.B, "context": w.T, "budget": w.budget,
                        "kv_bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (no flush)",
                        "launch": "one baklava_decode_attn%s call per step covering all layers" % (

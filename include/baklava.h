@@ -62,6 +62,9 @@ extern "C" {
 
 #define BAKLAVA_MAX_GROUP          8
 
+#define BAKLAVA_KV_BF16            0
+#define BAKLAVA_KV_FP8_E4M3        1
+
 /* Model attention shape and retention policy. */
 typedef struct baklava_shape {
     int32_t L;           /* layers                                                            */
@@ -80,11 +83,20 @@ typedef struct baklava_shape {
  *
  * Row `slot` of head (l, h) of sequence b is token row
  *     b * seq_stride_tokens + slab_off[l * Hkv + h] + slot          (0 <= slot < cap[l * Hkv + h])
- * of k_slab / v_slab (D bf16 each) and the same index of pos / score.
+ * of k_slab / v_slab (D bf16 each, or D bytes with BAKLAVA_KV_FP8_E4M3) and the same index of pos / score.
  * len[(b * L + l) * Hkv + h] rows are valid.  They are the slots 0 .. len without
  * free_slot (just 0 .. len-1 while free_slot == len, i.e. until the cache first
  * fills).  The next appended token is written at free_slot.  A cache reset
  * (the RESET_CACHE of Algorithm 3) is len = free_slot = 0.
+ *
+ * Quantised slabs (the paper names quantisation as a complement to budget allocation and fixes no
+ * scheme): with kv_dtype = BAKLAVA_KV_FP8_E4M3 a row element x of head (l, h) is stored as the FP8
+ * E4M3 code of fl32(x) * (1 / scale), rounded to nearest even and saturated to +-448, and stands for
+ * code * scale from then on, with one caller-chosen fp32 scale for K and one for V per (l, h); the
+ * reciprocals are passed alongside so that every implementation multiplies by the same number.
+ * baklava_decode_attn(_varlen) and baklava_evict(_varlen) quantise the rows they write (k_new / v_new,
+ * the dense prompt) and read the slabs accordingly; queries stay bf16 (they must be finite in fp16:
+ * |q| < 65504).  Only D = 128.  Everything else (positions, scores, policy) is unchanged.
  */
 typedef struct baklava_cache {
     void*          k_slab;             /* bf16 [B * seq_stride_tokens, D]        */
@@ -98,6 +110,8 @@ typedef struct baklava_cache {
     int64_t        seq_stride_tokens;  /* rows per sequence                      */
     int32_t        B;
     uint32_t*      status;             /* one word, OR of BAKLAVA_STATUS_* bits  */
+    int32_t        kv_dtype;           /* BAKLAVA_KV_BF16 or BAKLAVA_KV_FP8_E4M3 */
+    const float*   kv_scale;           /* FP8 only: [L, Hkv, 4] = K scale, 1 / K scale, V scale, 1 / V scale */
 } baklava_cache;
 
 /* Parameters of Algorithm 2 (threshold t, reduction r) and the bounds the paper leaves open. */

@@ -16,6 +16,7 @@ OK = 0
 FLAG_NO_APPEND, FLAG_NO_SCORE, FLAG_NO_EVICT = 1, 2, 4
 SCOPE_LAYER, SCOPE_MODEL = 0, 1
 STATUS_OVERFLOW, STATUS_BAD_STATE, STATUS_TIMEOUT = 1, 2, 4
+KV_BF16, KV_FP8_E4M3 = 0, 1
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbaklava.so")
 _lib = None
@@ -38,7 +39,8 @@ class Shape(ctypes.Structure):
 class CacheStruct(ctypes.Structure):
     _fields_ = [("k_slab", c_void_p), ("v_slab", c_void_p), ("pos", c_void_p), ("score", c_void_p),
                 ("len", c_void_p), ("free_slot", c_void_p), ("cap", c_void_p), ("slab_off", c_void_p),
-                ("seq_stride_tokens", c_int64), ("B", c_int32), ("status", c_void_p)]
+                ("seq_stride_tokens", c_int64), ("B", c_int32), ("status", c_void_p), ("kv_dtype", c_int32),
+                ("kv_scale", c_void_p)]
 
 
 class AllocParams(ctypes.Structure):
@@ -177,13 +179,25 @@ def baklava_decode_plan(shape, cap, B, layer_begin, layer_end, seq_stride_tokens
 class Cache:
     """Device buffers of a budgeted cache plus the struct the library reads.  Memory only."""
 
-    def __init__(self, shape, cap, slab_off, seq_stride, B, device="cuda"):
+    def __init__(self, shape, cap, slab_off, seq_stride, B, device="cuda", kv_dtype=KV_BF16, kv_scale=None):
+        """kv_scale: float32 array [L, Hkv, 2] = (K scale, V scale) per head, for FP8 slabs."""
         self.shape, self.B, self.seq_stride = shape, int(B), int(seq_stride)
+        self.kv_dtype = int(kv_dtype)
         self.cap_host = np.ascontiguousarray(cap, dtype=np.int32).reshape(shape.L, shape.Hkv)
         self.off_host = np.ascontiguousarray(slab_off, dtype=np.int64).reshape(shape.L, shape.Hkv)
         rows = self.B * self.seq_stride
-        self.k_slab = torch.empty((rows, shape.D), dtype=torch.bfloat16, device=device)
-        self.v_slab = torch.empty((rows, shape.D), dtype=torch.bfloat16, device=device)
+        slab_type = torch.uint8 if self.kv_dtype == KV_FP8_E4M3 else torch.bfloat16
+        self.k_slab = torch.empty((rows, shape.D), dtype=slab_type, device=device)
+        self.v_slab = torch.empty((rows, shape.D), dtype=slab_type, device=device)
+        self.kv_scale = None
+        if self.kv_dtype == KV_FP8_E4M3:
+            sc = np.ascontiguousarray(kv_scale, dtype=np.float32).reshape(shape.L, shape.Hkv, 2)
+            four = np.empty((shape.L, shape.Hkv, 4), dtype=np.float32)
+            four[..., 0], four[..., 2] = sc[..., 0], sc[..., 1]
+            four[..., 1] = np.float32(1.0) / sc[..., 0]        # float32 division, rounded once
+            four[..., 3] = np.float32(1.0) / sc[..., 1]
+            self.kv_scale_host = four
+            self.kv_scale = torch.from_numpy(four).to(device)
         self.pos = torch.full((rows,), -1, dtype=torch.int32, device=device)
         self.score = torch.zeros((rows,), dtype=torch.float32, device=device)
         self.len = torch.zeros((self.B, shape.L, shape.Hkv), dtype=torch.int32, device=device)
@@ -194,7 +208,8 @@ class Cache:
         self.struct = CacheStruct(self.k_slab.data_ptr(), self.v_slab.data_ptr(), self.pos.data_ptr(),
                                   self.score.data_ptr(), self.len.data_ptr(), self.free_slot.data_ptr(),
                                   self.cap.data_ptr(), self.slab_off.data_ptr(), self.seq_stride, self.B,
-                                  self.status.data_ptr())
+                                  self.status.data_ptr(), self.kv_dtype,
+                                  None if self.kv_scale is None else self.kv_scale.data_ptr())
 
     def reset(self):
         self.len.zero_()
@@ -208,7 +223,7 @@ class Cache:
 
     def kv_bytes_retained(self):
         """Bytes of K and V rows currently valid (the metric's numerator for one step)."""
-        return int(self.len.sum().item()) * self.shape.D * 2 * 2
+        return int(self.len.sum().item()) * self.shape.D * 2 * (1 if self.kv_dtype == KV_FP8_E4M3 else 2)
 
 
 def decode_workspace(plan, device="cuda"):

@@ -22,6 +22,7 @@
 
 #include "baklava.h"
 #include "common.h"
+#include "fp8.cuh"
 #include "ptx.cuh"
 
 namespace {
@@ -76,6 +77,7 @@ struct DecodeParams {
     unsigned long long* best_key;  // [n_score_items]
     int32_t* best_slot;            // [n_score_items]
     float scale_log2;   // log2(e) / sqrt(D)
+    const float* kv_scale;   // FP8 slabs: [L, Hkv, 4] (K scale, its reciprocal, V scale, its reciprocal)
 };
 
 struct Unit {
@@ -160,6 +162,19 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(zero), "r"(a2), "r"(zero), "r"(b0), "r"(b1));
 }
+// the same with fp16 operands (FP8 slabs: the codes convert to fp16 exactly)
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    const uint32_t zero = 0u;
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(zero), "r"(a2), "r"(zero), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
@@ -168,13 +183,23 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // ---------------------------------------------------------------- steps 2-4
 // kByPosition: the score-free sinks + window policy (a second instantiation, so that the default
 // path carries none of its registers or branches).
-template <int D, bool kByPosition>
+// kFp8: K and V rows are FP8 E4M3 codes (one byte per element, per-head scales).  A stage then holds 128
+// tokens (the same 32 KB), every consumer warp takes two 16-token blocks of it, the codes are widened to fp16
+// in registers (exactly) and the MMAs run in fp16 with the scales applied to the fp32 results.  The
+// contraction index of an MMA may be permuted freely as long as both operands agree, which is what lets
+// ldmatrix (16-bit granules) serve one-byte data: four consecutive bytes of a K row land in one register
+// and become two fp16 pairs; V comes through ldmatrix.trans as two tokens x two adjacent channels per
+// register, which a byte permute splits into an even-channel and an odd-channel operand.
+template <int D, bool kByPosition, bool kFp8>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(const DecodeParams p,
                                                                 const __grid_constant__ CUtensorMap k_map,
                                                                 const __grid_constant__ CUtensorMap v_map) {
     constexpr int kKSteps = D / 16;                    // MMA k-steps over the head dimension
     constexpr int kNTiles = D / 8;                     // 8-wide output column blocks
-    constexpr int kTileBytes = kTileTokens * D * 2;    // one K (or V) tile
+    constexpr int kTT = kFp8 ? 2 * kTileTokens : kTileTokens;       // tokens per stage
+    constexpr int kBlocks = kTT / (kConsumerWarps * kWarpTokens);    // 16-token blocks per warp and stage
+    constexpr int kRowBytes = kFp8 ? D : 2 * D;
+    constexpr int kTileBytes = kTT * kRowBytes;        // one K (or V) tile
     constexpr int kStageBytes = 2 * kTileBytes;
     constexpr int kG = BAKLAVA_MAX_GROUP;
 
@@ -212,7 +237,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
     if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
-    const int n_tiles = end > begin ? (end - begin + kTileTokens - 1) / kTileTokens : 0;
+    const int n_tiles = end > begin ? (end - begin + kTT - 1) / kTT : 0;
     const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
     // sinks + window without scores: the one row that is neither a sink nor in the window (the oldest) goes
     const bool pos_evict = kByPosition && hs.do_append && n_hi > C - 1;
@@ -220,6 +245,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     int old_pos = INT32_MAX, old_slot = -1;                // per lane, then per warp: oldest evictable row seen
 
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    const float scale_k = kFp8 ? p.scale_log2 * p.kv_scale[u.head * 4 + 0] : p.scale_log2;   // logits -> log2 domain
     // this head's share of the scratch: unnormalised probabilities [G][C] in fp16, each relative to the
     // running maximum its 16-token block was computed under, and those maxima [G][C / 16] in fp32
     __half* prob_h = reinterpret_cast<__half*>(p.logit + row0 * G);
@@ -261,12 +287,17 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                 }
                 const uint32_t full = smem_u32(&bar_full[s]);
                 const uint32_t dst = ring + s * kStageBytes;
-                const int y = (int)(row0 + begin + it * kTileTokens);
+                const int y = (int)(row0 + begin + it * kTT);
                 mbar_arrive_expect_tx(full, kStageBytes);
+                if (kFp8) {                                  // one 128-byte-wide box holds the whole row
+                    tma_load_2d(dst, &k_map, 0, y, full, stream_policy);
+                    tma_load_2d(dst + kTileBytes, &v_map, 0, y, full, stream_policy);
+                } else {
 #pragma unroll
-                for (int bx = 0; bx < D / 64; ++bx) {
-                    tma_load_2d(dst + bx * (kTileTokens * 128), &k_map, bx * 64, y, full, stream_policy);
-                    tma_load_2d(dst + kTileBytes + bx * (kTileTokens * 128), &v_map, bx * 64, y, full, stream_policy);
+                    for (int bx = 0; bx < D / 64; ++bx) {
+                        tma_load_2d(dst + bx * (kTileTokens * 128), &k_map, bx * 64, y, full, stream_policy);
+                        tma_load_2d(dst + kTileBytes + bx * (kTileTokens * 128), &v_map, bx * 64, y, full, stream_policy);
+                    }
                 }
             }
         }
@@ -278,11 +309,19 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             const __nv_bfloat16* qrow_ptr = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + qrow) * D;
 #pragma unroll
             for (int ks = 0; ks < kKSteps; ++ks) {
-                qa0[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + qcol) : 0u;
-                qa2[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + 8 + qcol) : 0u;
+                if (kFp8) {
+                    // channels 16 ks + 4 (lane % 4) + {0, 1} and + {2, 3}: the order the K bytes arrive in
+                    const uint2 raw = qrow < G ? *reinterpret_cast<const uint2*>(qrow_ptr + ks * 16 + 2 * qcol) : make_uint2(0u, 0u);
+                    const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+                    const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+                    qa0[ks] = pack_f16(f0.x, f0.y);
+                    qa2[ks] = pack_f16(f1.x, f1.y);
+                } else {
+                    qa0[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + qcol) : 0u;
+                    qa2[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + 8 + qcol) : 0u;
+                }
             }
         }
-        const int r0 = warp * kWarpTokens;                 // this warp's rows inside a tile
         const int lm = lane >> 3, li8 = lane & 7;          // ldmatrix: matrix index and row inside it
         bool alive = true;
         for (int it = 0; it < n_tiles && alive; ++it) {
@@ -294,7 +333,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             }
             const uint32_t k_tile = ring + s * kStageBytes;
             const uint32_t v_tile = k_tile + kTileBytes;
-            const int tok0 = begin + it * kTileTokens + r0;          // first token of this warp's block
+#pragma unroll
+            for (int blk = 0; blk < kBlocks; ++blk) {
+            const int r0 = (warp * kBlocks + blk) * kWarpTokens;     // this block's rows inside the tile
+            const int tok0 = begin + it * kTT + r0;                  // first token of the block
             const int valid = min(kWarpTokens, end - tok0);          // rows of the block inside the chunk
             if (valid > 0) {
                 if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + kWarpTokens) {
@@ -304,12 +346,25 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                     const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
                     const int64_t row = row0 + hs.f;
                     uint8_t* k_ptr = ring_ptr + s * kStageBytes;
+                    if (kFp8) {                              // quantise the row: eight elements per lane and operand
+                        for (int i = lane; i < 2 * kVec; i += 32) {
+                            const bool is_v = i >= kVec;
+                            const int c = is_v ? i - kVec : i;
+                            const uint4 raw = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
+                            const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + (is_v ? 3 : 1)]);
+                            *reinterpret_cast<uint2*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c >> 1) +
+                                                      (c & 1) * 8) = val;
+                            uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
+                            *(reinterpret_cast<uint2*>(slab + row * D) + c) = val;
+                        }
+                    } else {
                     for (int i = lane; i < 2 * kVec; i += 32) {
                         const bool is_v = i >= kVec;
                         const int c = is_v ? i - kVec : i;
                         const uint4 val = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
                         *reinterpret_cast<uint4*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c)) = val;
                         *(reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c) = val;
+                    }
                     }
                     if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
                     __syncwarp();
@@ -321,8 +376,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                 // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
                 if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
                     uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
-                    for (int i = lane; i < kWarpTokens * (D / 8); i += 32) {
-                        const int r = i / (D / 8), c = i % (D / 8);
+                    constexpr int kPieces = kRowBytes / 16;     // 16-byte pieces of a row
+                    for (int i = lane; i < kWarpTokens * kPieces; i += 32) {
+                        const int r = i / kPieces, c = i % kPieces;
                         if (r >= valid || tok0 + r == hole)
                             *reinterpret_cast<uint4*>(v_ptr + tile_offset(r0 + r, c)) = make_uint4(0, 0, 0, 0);
                     }
@@ -330,12 +386,27 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                 }
                 // S = Q K^T for 16 tokens: two 8-token column blocks
                 float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+                if (kFp8) {
+#pragma unroll
+                    for (int kk = 0; kk < D / 32; ++kk) {     // 32 channels per load: two k-steps for both token blocks
+                        uint32_t kb[4];
+                        ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * kk + (lm & 1)), kb);
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            const int ks = 2 * kk + c;
+                            mma_f16(sacc[0], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[c]), fp8::f16x2_from_e4m3x2(kb[c] >> 16));
+                            mma_f16(sacc[1], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[2 + c]),
+                                    fp8::f16x2_from_e4m3x2(kb[2 + c] >> 16));
+                        }
+                    }
+                } else {
 #pragma unroll
                 for (int ks = 0; ks < kKSteps; ++ks) {
                     uint32_t kb[4];
                     ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kb);
                     mma_bf16(sacc[0], qa0[ks], qa2[ks], kb[0], kb[1]);
                     mma_bf16(sacc[1], qa0[ks], qa2[ks], kb[2], kb[3]);
+                }
                 }
                 // this thread: row qrow, tokens tok0 + 8 t + qcol + {0, 1}
                 float sv[4];
@@ -345,7 +416,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const int tok = tok0 + 8 * t + qcol + e;
-                        sv[2 * t + e] = sacc[t][e] * p.scale_log2;
+                        sv[2 * t + e] = sacc[t][e] * scale_k;
                         ok[2 * t + e] = tok < end && tok != hole;
                     }
                 float mx = -INFINITY;
@@ -374,6 +445,24 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
 #pragma unroll
                     for (int j = 0; j < kNTiles; ++j) { o[j][0] *= corr; o[j][1] *= corr; }
                 }
+                if (kFp8) {
+                    const uint32_t pa0 = pack_f16(pv[0], pv[1]), pa2 = pack_f16(pv[2], pv[3]);
+                    // a register of the transposed load = two tokens x two adjacent channels; the permute puts the
+                    // even channel's token pair in the low half and the odd channel's in the high half.
+                    // o[2 c] collects channels 16 c + 0, 2, .., 14 and o[2 c + 1] channels 16 c + 1, 3, .., 15.
+#pragma unroll
+                    for (int c2 = 0; c2 < D / 32; ++c2) {
+                        uint32_t vb[4];
+                        ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * c2 + (lm >> 1)), vb);
+#pragma unroll
+                        for (int h2 = 0; h2 < 2; ++h2) {
+                            const uint32_t lo = __byte_perm(vb[2 * h2], 0u, 0x3120), hi = __byte_perm(vb[2 * h2 + 1], 0u, 0x3120);
+                            const int c = 2 * c2 + h2;
+                            mma_f16(o[2 * c], pa0, pa2, fp8::f16x2_from_e4m3x2(lo), fp8::f16x2_from_e4m3x2(hi));
+                            mma_f16(o[2 * c + 1], pa0, pa2, fp8::f16x2_from_e4m3x2(lo >> 16), fp8::f16x2_from_e4m3x2(hi >> 16));
+                        }
+                    }
+                } else {
                 const uint32_t pa0 = pack_bf16(pv[0], pv[1]), pa2 = pack_bf16(pv[2], pv[3]);
                 // O += P V: V^T fragments through ldmatrix.trans, two 8-wide column blocks per load
 #pragma unroll
@@ -383,6 +472,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                     mma_bf16(o[2 * j2], pa0, pa2, vb[0], vb[1]);
                     mma_bf16(o[2 * j2 + 1], pa0, pa2, vb[2], vb[3]);
                 }
+                }
+            }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
@@ -408,9 +499,17 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         lq += __shfl_xor_sync(0xffffffffu, lq, 1);
         lq += __shfl_xor_sync(0xffffffffu, lq, 2);
         if (qrow < G) {
+            if (kFp8) {                                         // four consecutive channels per thread and 16-channel group
+                const float sv_ = p.kv_scale[u.head * 4 + 2];
+#pragma unroll
+                for (int c = 0; c < D / 16; ++c)
+                    *reinterpret_cast<float4*>(sm_o + ((warp * G + qrow) * D + 16 * c + 2 * qcol)) =
+                        make_float4(o[2 * c][0] * sv_, o[2 * c + 1][0] * sv_, o[2 * c][1] * sv_, o[2 * c + 1][1] * sv_);
+            } else {
 #pragma unroll
             for (int j = 0; j < kNTiles; ++j)
                 *reinterpret_cast<float2*>(sm_o + ((warp * G + qrow) * D + 8 * j + qcol)) = make_float2(o[j][0], o[j][1]);
+            }
             if ((lane & 3) == 0) { sm_m[warp][qrow] = m_run; sm_l[warp][qrow] = lq; }
         }
     }
@@ -757,10 +856,23 @@ bool make_slab_map(CUtensorMap* map, void* base, int64_t rows, int D) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool kByPosition>
+// FP8 slabs: one byte per element, boxes of 128 rows x 128 bytes (the whole row), 128-byte swizzle
+bool make_slab_map_fp8(CUtensorMap* map, void* base, int64_t rows, int D) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)D};
+    const cuuint32_t box[2] = {128, (cuuint32_t)(2 * kTileTokens)};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, bool kByPosition, bool kFp8 = false>
 cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
-    constexpr int kSmem = kStages * 2 * kTileTokens * D * 2 + 1024;
-    cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D, kByPosition>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    constexpr int kSmem = kStages * 2 * kTileTokens * D * 2 + 1024;      // the same 32 KB stages for both formats
+    cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D, kByPosition, kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -772,7 +884,7 @@ cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CU
     cfg.stream = s;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_chunk_kernel<D, kByPosition>, p, km, vm);
+    return cudaLaunchKernelEx(&cfg, decode_chunk_kernel<D, kByPosition, kFp8>, p, km, vm);
 }
 
 }  // namespace
@@ -807,9 +919,17 @@ int decode_attn_impl(
                                                 cache->seq_stride_tokens, &lay);
     if (ws_bytes < need) return BAKLAVA_ERR_WORKSPACE;
 
+    const bool quantised = cache->kv_dtype == BAKLAVA_KV_FP8_E4M3;
+    if (cache->kv_dtype != BAKLAVA_KV_BF16 && !quantised) return BAKLAVA_ERR_INVALID_ARG;
+    if (quantised && !cache->kv_scale) return BAKLAVA_ERR_INVALID_ARG;
+    if (quantised && shape->D != 128) return BAKLAVA_ERR_UNSUPPORTED;
     CUtensorMap k_map, v_map;
-    if (!make_slab_map(&k_map, cache->k_slab, rows, shape->D) || !make_slab_map(&v_map, cache->v_slab, rows, shape->D))
+    if (quantised) {
+        if (!make_slab_map_fp8(&k_map, cache->k_slab, rows, shape->D) || !make_slab_map_fp8(&v_map, cache->v_slab, rows, shape->D))
+            return BAKLAVA_ERR_CUDA;
+    } else if (!make_slab_map(&k_map, cache->k_slab, rows, shape->D) || !make_slab_map(&v_map, cache->v_slab, rows, shape->D)) {
         return BAKLAVA_ERR_CUDA;
+    }
 
     DecodeParams p;
     p.k_slab = static_cast<__nv_bfloat16*>(cache->k_slab);
@@ -850,10 +970,12 @@ int decode_attn_impl(
     p.best_key = reinterpret_cast<unsigned long long*>(base + lay.best_off);
     p.best_slot = reinterpret_cast<int32_t*>(base + lay.best_off + 8 * (size_t)info->n_score_items);
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
+    p.kv_scale = cache->kv_scale;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
-    if (p.window_evict) err = shape->D == 128 ? launch_chunks<128, true>(p, k_map, v_map, s) : launch_chunks<64, true>(p, k_map, v_map, s);
+    if (quantised) err = p.window_evict ? launch_chunks<128, true, true>(p, k_map, v_map, s) : launch_chunks<128, false, true>(p, k_map, v_map, s);
+    else if (p.window_evict) err = shape->D == 128 ? launch_chunks<128, true>(p, k_map, v_map, s) : launch_chunks<64, true>(p, k_map, v_map, s);
     else err = shape->D == 128 ? launch_chunks<128, false>(p, k_map, v_map, s) : launch_chunks<64, false>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     if (!(p.flags & BAKLAVA_FLAG_NO_SCORE)) {

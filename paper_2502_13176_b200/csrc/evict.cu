@@ -12,6 +12,7 @@
 
 #include "baklava.h"
 #include "common.h"
+#include "fp8.cuh"
 
 namespace {
 
@@ -39,6 +40,7 @@ struct EvictParams {
     const int32_t* seq_len;   // [B] tokens of each sequence's prompt (clamped to 0 .. T) or NULL: T for all
     int64_t stride_layer, stride_seq, stride_head;
     int32_t* kept;   // [n_units][T]
+    const float* kv_scale;   // FP8 slabs: [L, Hkv, 4] (K scale, its reciprocal, V scale, its reciprocal)
 };
 
 struct Where {
@@ -175,7 +177,7 @@ __global__ void __launch_bounds__(kSelThreads) evict_select_kernel(const EvictPa
     if (tid == 0) { p.len[w.st] = R; p.free_slot[w.st] = R; }
 }
 
-template <int D>
+template <int D, bool kFp8>
 __global__ void __launch_bounds__(kCopyThreads) evict_copy_kernel(const EvictParams p) {
     const int unit = blockIdx.x;
     const Where w = locate(p, unit);
@@ -192,8 +194,14 @@ __global__ void __launch_bounds__(kCopyThreads) evict_copy_kernel(const EvictPar
         const bool is_v = piece >= kVec;
         const int c = is_v ? piece - kVec : piece;
         const uint4* from = reinterpret_cast<const uint4*>((is_v ? p.v_dense : p.k_dense) + (w.dense0 + src) * D) + c;
-        uint4* to = reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + (w.slab0 + r) * D) + c;
-        *to = __ldg(from);
+        if (kFp8) {          // the row is quantised on its way into the slab: D bytes per row
+            const float inv_scale = p.kv_scale[w.head * 4 + (is_v ? 3 : 1)];
+            uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
+            *(reinterpret_cast<uint2*>(slab + (w.slab0 + r) * D) + c) = fp8::quantise8(__ldg(from), inv_scale);
+        } else {
+            uint4* to = reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + (w.slab0 + r) * D) + c;
+            *to = __ldg(from);
+        }
         if (piece == 0) {
             p.pos[w.slab0 + r] = src;
             p.score[w.slab0 + r] = p.score_dense ? p.score_dense[w.dense0 + src] + 0.0f : 0.0f;
@@ -240,13 +248,19 @@ int evict_impl(const baklava_shape* shape, const baklava_cache* cache, int32_t l
     p.seq_len = seq_len;
     p.stride_layer = stride_layer; p.stride_seq = stride_seq; p.stride_head = stride_head;
     p.kept = kept;
+    p.kv_scale = cache->kv_scale;
+    const bool quantised = cache->kv_dtype == BAKLAVA_KV_FP8_E4M3;
+    if (cache->kv_dtype != BAKLAVA_KV_BF16 && !quantised) return BAKLAVA_ERR_INVALID_ARG;
+    if (quantised && !cache->kv_scale) return BAKLAVA_ERR_INVALID_ARG;
+    if (quantised && shape->D != 128) return BAKLAVA_ERR_UNSUPPORTED;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     evict_select_kernel<<<(unsigned)units, kSelThreads, 0, s>>>(p);
     if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
     const dim3 grid((unsigned)units, (unsigned)row_blocks);
-    if (shape->D == 128) evict_copy_kernel<128><<<grid, kCopyThreads, 0, s>>>(p);
-    else evict_copy_kernel<64><<<grid, kCopyThreads, 0, s>>>(p);
+    if (quantised) evict_copy_kernel<128, true><<<grid, kCopyThreads, 0, s>>>(p);
+    else if (shape->D == 128) evict_copy_kernel<128, false><<<grid, kCopyThreads, 0, s>>>(p);
+    else evict_copy_kernel<64, false><<<grid, kCopyThreads, 0, s>>>(p);
     return cudaGetLastError() == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
 }
 

@@ -14,7 +14,7 @@ def shape_of(w):
 
 class DecodeSession:
     def __init__(self, w, device="cuda", layers=None, chunk_tokens=0, uniform=False, alloc=None, importance=None,
-                 total_tokens=None):
+                 total_tokens=None, kv_dtype=bk.KV_BF16):
         """`alloc` = (t, r_num, r_den) overrides the workload's Algorithm 2 parameters, `importance` its
         synthetic importances, `total_tokens` its budget (e.g. the dense length for a reference run)."""
         self.w, self.device = w, torch.device(device)
@@ -26,7 +26,10 @@ class DecodeSession:
         self.cap, self.off, self.stride = bk.baklava_allocate(
             self.shape, self.importance, t, 0 if uniform else r_num, r_den, total,
             w.min_pages * w.page, w.max_pages * w.page)
-        self.cache = bk.Cache(self.shape, self.cap, self.off, self.stride, w.B, self.device)
+        self.kv_dtype = kv_dtype
+        fp8_scales = wl.kv_fp8_scales(w, self.scales) if kv_dtype == bk.KV_FP8_E4M3 else None
+        self.cache = bk.Cache(self.shape, self.cap, self.off, self.stride, w.B, self.device, kv_dtype=kv_dtype,
+                              kv_scale=fp8_scales)
         self.lb, self.le = (0, w.L) if layers is None else layers
         n_sm = torch.cuda.get_device_properties(self.device).multi_processor_count
         self.plan = bk.baklava_decode_plan(self.shape, self.cap, w.B, self.lb, self.le, self.stride,
@@ -70,7 +73,7 @@ class DecodeSession:
     def retained_kv_bytes(self):
         """Bytes of K and V in valid rows of the session's layers: what one step must read."""
         n = int(self.cache.len[:, self.lb:self.le].sum().item())
-        return n * self.w.D * 2 * 2
+        return n * self.w.D * 2 * (1 if self.kv_dtype == bk.KV_FP8_E4M3 else 2)
 
     def check_status(self):
         code = int(self.cache.status.item())

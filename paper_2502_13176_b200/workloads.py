@@ -110,6 +110,13 @@ def kv_scales(w):
     raise ValueError(w.kv_recipe)
 
 
+def kv_fp8_scales(w, scales):
+    """Per-head FP8 scales (K, V) as float32 [L, Hkv, 2]: six standard deviations of the head's widest
+    channel map to the largest finite E4M3 value (448)."""
+    widest = torch.stack([scales[0].amax(dim=2), scales[1].amax(dim=2)], dim=2)      # [L, Hkv, 2]
+    return (widest * (6.0 / 448.0)).to(torch.float32).numpy()
+
+
 def dense_kv(w, l, b, h, scales, device="cpu", T=None):
     """Prefilled K and V of one (layer, sequence, KV head): two bf16 [T, D] tensors."""
     T = w.T if T is None else T

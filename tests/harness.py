@@ -8,6 +8,7 @@ import torch
 
 from oracle import allocation as oalloc
 from oracle import eviction as oevict
+from oracle import fp8 as ofp8
 from oracle.cache import HeadCache
 from paper_2502_13176_b200 import binding as bk
 from paper_2502_13176_b200 import workloads as wl
@@ -37,8 +38,10 @@ def f64(t):
 class Session:
     """One workload on the device (library) with oracle twins for the heads in `heads`."""
 
-    def __init__(self, w, heads=None, chunk_tokens=0, layers=None, prefill=True, device="cuda", caps=None):
+    def __init__(self, w, heads=None, chunk_tokens=0, layers=None, prefill=True, device="cuda", caps=None,
+                 kv_dtype=bk.KV_BF16):
         self.w, self.device = w, device
+        self.kv_dtype = kv_dtype
         self.shape = shape_of(w)
         self.scales = wl.kv_scales(w)
         self.imp = wl.importance(w).numpy()
@@ -56,7 +59,9 @@ class Session:
             flat = self.cap.reshape(-1).astype(np.int64)
             self.off = np.concatenate([[0], np.cumsum(flat)[:-1]]).reshape(w.L, w.Hkv)
             self.stride = int(flat.sum())
-        self.cache = bk.Cache(self.shape, self.cap, self.off, self.stride, w.B, device)
+        self.fp8_scales = wl.kv_fp8_scales(w, self.scales) if kv_dtype == bk.KV_FP8_E4M3 else None
+        self.cache = bk.Cache(self.shape, self.cap, self.off, self.stride, w.B, device, kv_dtype=kv_dtype,
+                              kv_scale=self.fp8_scales)
         self.lb, self.le = (0, w.L) if layers is None else layers
         self.plan = bk.baklava_decode_plan(self.shape, self.cap, w.B, self.lb, self.le, self.stride,
                                            chunk_tokens=chunk_tokens,
@@ -75,6 +80,14 @@ class Session:
             for (b, l, h) in self.heads:
                 self.twins[(b, l, h)] = HeadCache(int(self.cap[l, h]), w.D, w.n_sink, w.recent_num, w.recent_den)
 
+    def as_stored(self, rows, l, h, which):
+        """The values the cache holds for `rows` (float64) of head (l, h): themselves, or their FP8 round trip.
+        which: 0 = K, 1 = V."""
+        if self.kv_dtype != bk.KV_FP8_E4M3:
+            return rows
+        four = self.cache.kv_scale_host[l, h]
+        return ofp8.quantise_rows(rows, four[2 * which], four[2 * which + 1])[1]
+
     def _prefill(self):
         w = self.w
         ews = torch.empty((bk.baklava_evict_workspace_size(self.shape, w.B, 1, w.T),), dtype=torch.uint8,
@@ -89,7 +102,8 @@ class Session:
             k, v = wl.dense_kv(w, l, b, h, self.scales)
             sc = wl.prefill_scores(w, l)[b, h]
             C = int(self.cap[l, h])
-            K2, V2, pos2, s2, _ = oevict.bulk_evict(f64(k), f64(v), np.arange(w.T), f64(sc), C - 1,
+            K2, V2, pos2, s2, _ = oevict.bulk_evict(self.as_stored(f64(k), l, h, 0), self.as_stored(f64(v), l, h, 1),
+                                                   np.arange(w.T), f64(sc), C - 1,
                                                    w.n_sink, w.recent_num, w.recent_den)
             hc = HeadCache(C, w.D, w.n_sink, w.recent_num, w.recent_den)
             hc.load(K2, V2, pos2, s2)
@@ -99,7 +113,13 @@ class Session:
     def head_state(self, b, l, h):
         lo, hi = self.cache.rows(b, l, h)
         c = self.cache
-        return dict(K=f64(c.k_slab[lo:hi]), V=f64(c.v_slab[lo:hi]), pos=c.pos[lo:hi].cpu().numpy().astype(np.int64),
+        if self.kv_dtype == bk.KV_FP8_E4M3:
+            four = c.kv_scale_host[l, h]
+            K = ofp8.decode(c.k_slab[lo:hi].cpu().numpy()) * float(four[0])
+            V = ofp8.decode(c.v_slab[lo:hi].cpu().numpy()) * float(four[2])
+        else:
+            K, V = f64(c.k_slab[lo:hi]), f64(c.v_slab[lo:hi])
+        return dict(K=K, V=V, pos=c.pos[lo:hi].cpu().numpy().astype(np.int64),
                     score=c.score[lo:hi].cpu().numpy(), len=int(c.len[b, l, h]), free=int(c.free_slot[b, l, h]))
 
     def valid_slots(self, st):
@@ -136,7 +156,8 @@ class Session:
         for (b, l, h) in self.heads:
             tw = self.twins[(b, l, h)]
             li = l - self.lb
-            o_ref, lse_ref, ev = tw.step(qh[li, b, h * g:(h + 1) * g], knh[li, b, h], vnh[li, b, h], t_pos,
+            o_ref, lse_ref, ev = tw.step(qh[li, b, h * g:(h + 1) * g], self.as_stored(knh[li, b, h], l, h, 0),
+                                         self.as_stored(vnh[li, b, h], l, h, 1), t_pos,
                                          append=append, update_score=not (flags & bk.FLAG_NO_SCORE),
                                          evict=not (flags & bk.FLAG_NO_EVICT) and
                                          (not (flags & bk.FLAG_NO_SCORE) or w.recent_num == w.recent_den))
