@@ -39,7 +39,10 @@ size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t 
 
 inline bool baklava_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// prefill.cu: log2-domain largest logit of every causal query row, lse2 [B, Hq, T] (+inf past the prompt)
+// prefill.cu: log2-domain largest logit of every causal query row (+inf past the prompt) into lse2 [B, Hq, T],
+// for the 128-row blocks listed in `list` (flat index ((b * Hq + h) * n_blk + blk), *list_count entries, both on
+// the device); `grid` CTAs share the list
 struct CUstream_st;
 int baklava_launch_row_max(const baklava_shape* shape, const void* q, const void* k, const int32_t* prompt_len,
-                           int32_t B, int32_t T, float* lse2, uint32_t* error, CUstream_st* stream);
+                           int32_t B, int32_t T, float* lse2, const int32_t* list, const int32_t* list_count,
+                           int32_t grid, uint32_t* error, CUstream_st* stream);

@@ -44,10 +44,10 @@ struct PrefillParams {
     float scale_log2;
 };
 
+// One CTA's work: the row block / key block (bx, by, bz) of the grid the pass is normally launched with.
 template <int D, int PASS>
-__global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParams p,
-                                                           const __grid_constant__ CUtensorMap q_map,
-                                                           const __grid_constant__ CUtensorMap k_map) {
+__device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                              const int bx, const int by, const int bz) {
     constexpr int kKSteps = D / 16;                         // one MMA covers 16 elements of the head dimension
     constexpr int kBoxBytes = kTileRows * 128;              // one TMA box: 128 rows x 64 elements
     constexpr int kTileBytes = kTileRows * D * 2;
@@ -59,12 +59,12 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = p.Hq / p.Hkv;
-    const int b = blockIdx.z;
+    const int b = bz;
     const int len = p.prompt_len ? min(max(p.prompt_len[b], 0), p.T) : p.T;
     int blk, n_it, nq = 1, head_res, head_first;            // resident block, streamed tiles, heads
     if (PASS != kPassColumnSums) {
-        blk = p.n_blk - 1 - blockIdx.x;                     // long rows of the causal triangle first
-        const int h = blockIdx.y;
+        blk = p.n_blk - 1 - bx;                             // long rows of the causal triangle first
+        const int h = by;
         head_res = b * p.Hq + h;
         head_first = b * p.Hkv + h / g;
         n_it = blk + 1;
@@ -74,8 +74,8 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
             return;
         }
     } else {
-        blk = blockIdx.x;                                   // early key blocks meet the most query tiles: first
-        const int kvh = blockIdx.y;
+        blk = bx;                                           // early key blocks meet the most query tiles: first
+        const int kvh = by;
         head_res = b * p.Hkv + kvh;
         head_first = b * p.Hq + kvh * g;
         if (blk * kTileRows >= len) {                       // keys past the prompt receive nothing
@@ -285,6 +285,38 @@ __global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParam
         tc::tmem_dealloc(tmem_base, kTmemColumns);
     }
     if (tid == 0 && sm_abort) atomicOr(p.error, 1u);
+    if (tid == 0) {                                         // the barriers may be set up again by the next block of this CTA
+        mbar_inval(smem_u32(&bar_res));
+        for (int s = 0; s < 2; ++s) {
+            mbar_inval(smem_u32(&bar_full[s]));
+            mbar_inval(smem_u32(&bar_empty[s]));
+            mbar_inval(smem_u32(&bar_acc_full[s]));
+            mbar_inval(smem_u32(&bar_acc_empty[s]));
+        }
+    }
+    __syncthreads();
+}
+
+template <int D, int PASS>
+__global__ void __launch_bounds__(kThreads, 2) qk_pass_kernel(const PrefillParams p,
+                                                           const __grid_constant__ CUtensorMap q_map,
+                                                           const __grid_constant__ CUtensorMap k_map) {
+    qk_pass_block<D, PASS>(p, q_map, k_map, blockIdx.x, blockIdx.y, blockIdx.z);
+}
+
+// The row-maximum pass over a list of row blocks (entries = flat index ((b * Hq + h) * n_blk + blk), count
+// in *list_count): a small fixed grid whose CTAs take the entries in turn, so that an empty list costs nothing.
+template <int D>
+__global__ void __launch_bounds__(kThreads, 2) row_max_list_kernel(const PrefillParams p, const int32_t* list,
+                                                                const int32_t* list_count,
+                                                                const __grid_constant__ CUtensorMap q_map,
+                                                                const __grid_constant__ CUtensorMap k_map) {
+    const int n = *list_count;
+    for (int w = blockIdx.x; w < n; w += gridDim.x) {
+        const int flat = list[w];
+        const int blk = flat % p.n_blk, h = (flat / p.n_blk) % p.Hq, b = flat / (p.n_blk * p.Hq);
+        qk_pass_block<D, kPassRowMax>(p, q_map, k_map, p.n_blk - 1 - blk, h, b);
+    }
 }
 
 template <int D, int PASS>
@@ -310,7 +342,8 @@ cudaError_t launch_prefill(const PrefillParams& p, const CUtensorMap& qm, const 
 // (+inf past the prompt).  The cosine of Algorithm 1 does not depend on the scale of a head's output
 // row, so the row maximum serves as the softmax's stabiliser and its sum is never needed.
 int baklava_launch_row_max(const baklava_shape* shape, const void* q, const void* k, const int32_t* prompt_len,
-                           int32_t B, int32_t T, float* lse2, uint32_t* error, cudaStream_t s) {
+                           int32_t B, int32_t T, float* lse2, const int32_t* list, const int32_t* list_count,
+                           int32_t grid, uint32_t* error, cudaStream_t s) {
     PrefillParams p;
     p.prompt_len = prompt_len;
     p.error = error;
@@ -323,8 +356,16 @@ int baklava_launch_row_max(const baklava_shape* shape, const void* q, const void
     if (!make_head_map(&qm, q, (int64_t)B * shape->Hq, T, shape->D, kTileRows) ||
         !make_head_map(&km, k, (int64_t)B * shape->Hkv, T, shape->D, kTileRows))
         return BAKLAVA_ERR_CUDA;
-    cudaError_t e = shape->D == 128 ? launch_pass<128, kPassRowMax>(p, qm, km, dim3(p.n_blk, p.Hq, B), s)
-                                    : launch_pass<64, kPassRowMax>(p, qm, km, dim3(p.n_blk, p.Hq, B), s);
+    constexpr int kSmem128 = 100 * 1024, kSmem64 = 100 * 1024;   // as launch_pass: at most two CTAs (2 x 256 TMEM columns) per SM
+    cudaError_t e;
+    if (shape->D == 128) {
+        e = cudaFuncSetAttribute(row_max_list_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem128);
+        if (e == cudaSuccess) row_max_list_kernel<128><<<grid, kThreads, kSmem128, s>>>(p, list, list_count, qm, km);
+    } else {
+        e = cudaFuncSetAttribute(row_max_list_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem64);
+        if (e == cudaSuccess) row_max_list_kernel<64><<<grid, kThreads, kSmem64, s>>>(p, list, list_count, qm, km);
+    }
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
 }
 

@@ -2,14 +2,15 @@
 // causal softmax attention O = softmax(Q K^T / sqrt(D)) V and the token-wise cosine between the
 // head's input V_t and its output O_t, averaged over the prompt's tokens.
 //
-// Two launches on the 5th-generation tensor cores.  The first gives every query row its largest logit
-// (a row pass of the prompt-score kernels, without exponentials).  That is all the softmax needs here:
-// the cosine does not change when a row of O is scaled, so the probabilities are left unnormalised,
-// p = exp2(s - max) <= 1, and O never needs rescaling or dividing.  The second launch owns 128 query rows
-// per CTA: the Q tile stays in shared memory, K and V tiles of 128 keys stream through three-stage TMA
-// rings; one thread issues S = Q K^T into tensor memory (double-buffered), sixteen softmax warps read S
-// back, form the probabilities in bf16 and write them back to tensor memory, from where the next MMA takes
-// them as its A operand, and the same thread issues O += P V with V as an MN-major B operand; O
+// One pass on the 5th-generation tensor cores.  The cosine does not change when a row of O is scaled, so
+// the softmax is left unnormalised and needs only a stabiliser per row, for which the row's largest logit in
+// the first key tile serves: p = exp2(s - reference), no running maximum, no sum, no rescaling of O, no
+// division.  (Rows whose later logits leave the fp32 range that way are detected in the epilogue and redone
+// by a second instantiation that takes the true row maxima from a row pass; see profile_pv_block.)
+// A CTA owns 128 query rows: the Q tile stays in shared memory, K and V tiles of 128 keys stream through
+// three-stage TMA rings; one thread issues S = Q K^T into tensor memory (double-buffered), sixteen softmax
+// warps read S back, form the probabilities in bf16 and write them back to tensor memory, from where the next
+// MMA takes them as its A operand, and the same thread issues O += P V with V as an MN-major B operand; O
 // accumulates in tensor memory over all key tiles and is never written.  The last key tile is the
 // diagonal one, whose V rows are exactly the rows the cosine needs, so the final epilogue reads them from
 // shared memory.
@@ -36,7 +37,9 @@ constexpr float kCosEps = 1e-12f;
 
 struct ProfileParams {
     const int32_t* prompt_len;   // [P] or null
-    const float* lse2;           // [P, Hq, T] from the row pass: every row's largest logit, log2 domain
+    const float* lse2;           // [P, Hq, T] from the row pass: every row's largest logit, log2 domain (exact mode)
+    int32_t* redo_list;          // flat indices ((pr * Hq + h) * n_blk + qb) of the row blocks the one-pass kernel
+    int32_t* redo_count;         //   could not finish in range, and how many there are
     float* head_cos;             // [P, Hq]
     float* token_cos;            // [P, Hq, T] or null
     float* block_sum;            // [P, Hq, n_blk]
@@ -55,11 +58,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfileParams p,
-                                                                 const __grid_constant__ CUtensorMap q_map,
-                                                                 const __grid_constant__ CUtensorMap k_map,
-                                                                 const __grid_constant__ CUtensorMap v_map) {
+// kExact = false: one pass.  The softmax needs a stabiliser per row, not the row's true maximum: the
+// largest logit among the row's keys in the FIRST key tile serves (every row sees key 0, so it exists),
+// probabilities of later keys may then exceed 1, which bf16 and the fp32 accumulator hold up to 2^127.
+// A row whose later logits are so far above that reference that O or its norm leaves the fp32 range
+// shows up as a non-finite cosine term in the epilogue; its row block is flagged in `redo` and done again
+// by the kExact = true instantiation, which takes every row's true maximum from a row pass and runs only
+// on flagged blocks.  Results that stayed finite are exact up to rounding, because scaling a row of O by
+// a power of two changes nothing in its cosine.
+template <int D, bool kExact>
+__device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                                 const CUtensorMap& v_map, const int qb, const int h, const int pr) {
     constexpr int kKSteps = D / 16;                          // MMA steps over the head dimension (S = Q K^T)
     constexpr int kPvSteps = kTileRows / 16;                 // MMA steps over the keys (O += P V)
     constexpr int kBoxBytes = kTileRows * 128;               // one TMA box: 128 rows x 64 elements
@@ -73,10 +82,9 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     __shared__ uint32_t tmem_slot;
     __shared__ float sm_warp_sum[kSoftmaxWarps];
     __shared__ int sm_abort;
+    __shared__ int sm_redo;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int qb = p.n_blk - 1 - blockIdx.x;                 // long rows of the causal triangle first
-    const int h = blockIdx.y, pr = blockIdx.z;
     const int kvh = h / (p.Hq / p.Hkv);
     const int len = p.prompt_len ? min(max(p.prompt_len[pr], 0), p.T) : p.T;
     float* out_sum = p.block_sum + ((int64_t)pr * p.Hq + h) * p.n_blk + qb;
@@ -98,6 +106,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
             mbar_init(smem_u32(&bar_group[s]), 1);
         }
         sm_abort = 0;
+        sm_redo = 0;
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -197,13 +206,28 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
         const int col_base = part * 32;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
         const int t = qb * kTileRows + row;
-        const float lse = t < p.T ? p.lse2[((int64_t)pr * p.Hq + h) * p.T + t] : INFINITY;   // row maximum; +inf past the prompt
+        // the softmax's reference logit of this row, log2 domain (exact mode: the row's maximum; +inf past the prompt)
+        float lse = 0.0f;
+        if (kExact) lse = t < p.T ? p.lse2[((int64_t)pr * p.Hq + h) * p.T + t] : INFINITY;
         bool ok = true;
         for (int it = 0; it < n_it; ++it) {
             const int s = it & 1;
             if (!group_wait(it)) { ok = false; break; }        // S(it) is ready and P V of tile it - 2 has read its P
             tc::fence_after_sync();
             uint32_t v[32];
+            if (!kExact && it == 0) {
+                // reference = largest logit of the row over the whole first key tile (all four column groups)
+                float mx = -INFINITY;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
+                    tc::tmem_ld_32x32(lane_addr + c0, v);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (qb > 0 || c0 + c <= row) mx = fmaxf(mx, __uint_as_float(v[c]));
+                }
+                lse = mx * p.scale_log2;
+            }
             tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base, v);
             tc::tmem_ld_wait();
             if (it == qb) {                                   // diagonal tile: keys above the query do not exist
@@ -265,6 +289,10 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
                 o4 += sm_part[(2 * 4 + k) * kTileRows + row];
             }
             c = d4 / fmaxf(sqrtf(v4) * sqrtf(o4), kCosEps);
+            if (!kExact && !(fabsf(d4) <= 3.0e38f && o4 <= 3.0e38f)) {   // left the fp32 range (or NaN): redo this block
+                sm_redo = 1;
+                c = 0.0f;
+            }
             if (p.token_cos) p.token_cos[((int64_t)pr * p.Hq + h) * p.T + t] = c;
         }
 #pragma unroll
@@ -280,7 +308,41 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
     }
     if (tid == 0) {
         if (sm_abort) atomicOr(p.error, 1u);
-        *out_sum = sm_abort ? 0.0f : (sm_warp_sum[0] + sm_warp_sum[1]) + (sm_warp_sum[2] + sm_warp_sum[3]);
+        const bool again = !kExact && sm_redo != 0;
+        *out_sum = (sm_abort || again) ? 0.0f : (sm_warp_sum[0] + sm_warp_sum[1]) + (sm_warp_sum[2] + sm_warp_sum[3]);
+        if (again) p.redo_list[atomicAdd(p.redo_count, 1)] = (pr * p.Hq + h) * p.n_blk + qb;
+        // the barriers may be set up again by the next row block of this CTA (exact mode)
+        mbar_inval(smem_u32(&bar_q));
+        for (int s = 0; s < 2; ++s) mbar_inval(smem_u32(&bar_k01[s]));
+        for (int s = 0; s < kGroupRing; ++s) {
+            mbar_inval(smem_u32(&bar_in[s]));
+            mbar_inval(smem_u32(&bar_group[s]));
+        }
+    }
+    __syncthreads();
+}
+
+// One pass over every row block of the layer: grid (row blocks, query heads, prompts), long blocks first.
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfileParams p,
+                                                                 const __grid_constant__ CUtensorMap q_map,
+                                                                 const __grid_constant__ CUtensorMap k_map,
+                                                                 const __grid_constant__ CUtensorMap v_map) {
+    profile_pv_block<D, false>(p, q_map, k_map, v_map, p.n_blk - 1 - (int)blockIdx.x, blockIdx.y, blockIdx.z);
+}
+
+// The exact form over the row blocks the one-pass kernel listed: a small fixed grid whose CTAs take the
+// entries in turn, so that the usual empty list costs nothing.
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) profile_pv_redo_kernel(const ProfileParams p,
+                                                                      const __grid_constant__ CUtensorMap q_map,
+                                                                      const __grid_constant__ CUtensorMap k_map,
+                                                                      const __grid_constant__ CUtensorMap v_map) {
+    const int n = *p.redo_count;
+    for (int w = blockIdx.x; w < n; w += gridDim.x) {
+        const int flat = p.redo_list[w];
+        profile_pv_block<D, true>(p, q_map, k_map, v_map, flat % p.n_blk, (flat / p.n_blk) % p.Hq,
+                                  flat / (p.n_blk * p.Hq));
     }
 }
 
@@ -294,11 +356,19 @@ __global__ void profile_mean_kernel(const ProfileParams p) {
     p.head_cos[i] = len > 0 ? acc / (float)len : 0.0f;
 }
 
-template <int D>
+constexpr int kRedoGrid = 148;        // CTAs that share the list of row blocks to redo
+
+template <int D, bool kExact>
 cudaError_t launch_profile(const ProfileParams& p, const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
                            cudaStream_t s) {
     // Q tile and the (K, V) stages
     constexpr int kSmem = kTileRows * D * 2 * (1 + 2 * kKvStages) + 1024;
+    if (kExact) {
+        cudaError_t e = cudaFuncSetAttribute(profile_pv_redo_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        if (e != cudaSuccess) return e;
+        profile_pv_redo_kernel<D><<<kRedoGrid, kThreads, kSmem, s>>>(p, qm, km, vm);
+        return cudaGetLastError();
+    }
     cudaError_t e = cudaFuncSetAttribute(profile_pv_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     const dim3 grid(p.n_blk, p.Hq, p.P);
@@ -312,7 +382,7 @@ extern "C" __attribute__((visibility("default"))) size_t baklava_profile_workspa
                                                                                     int32_t P, int32_t T) {
     if (!shape || P <= 0 || T <= 0) return 0;
     const size_t n_blk = ((size_t)T + kTileRows - 1) / kTileRows;
-    return 256 + sizeof(float) * (size_t)P * shape->Hq * ((size_t)T + n_blk);
+    return 256 + sizeof(float) * (size_t)P * shape->Hq * ((size_t)T + 2 * n_blk);
 }
 
 extern "C" __attribute__((visibility("default"))) int baklava_profile_heads(
@@ -336,6 +406,8 @@ extern "C" __attribute__((visibility("default"))) int baklava_profile_heads(
     float* lse2 = reinterpret_cast<float*>(static_cast<char*>(ws) + 256);
     p.lse2 = lse2;
     p.block_sum = lse2 + (size_t)P * shape->Hq * (size_t)T;
+    p.redo_list = reinterpret_cast<int32_t*>(p.block_sum + (size_t)P * shape->Hq * ((size_t)(T + kTileRows - 1) / kTileRows));
+    p.redo_count = reinterpret_cast<int32_t*>(ws) + 1;       // inside the header that is cleared below
     p.P = P; p.T = T; p.Hq = shape->Hq; p.Hkv = shape->Hkv;
     p.n_blk = (T + kTileRows - 1) / kTileRows;
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
@@ -348,9 +420,13 @@ extern "C" __attribute__((visibility("default"))) int baklava_profile_heads(
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemsetAsync(ws, 0, 256, s) != cudaSuccess) return BAKLAVA_ERR_CUDA;
-    rc = baklava_launch_row_max(shape, q, k, prompt_len, P, T, lse2, p.error, s);
+    // one pass for everything, then the exact two-pass form for the row blocks it listed (normally none:
+    // both follow-up launches then find an empty list and return at once)
+    cudaError_t err = shape->D == 128 ? launch_profile<128, false>(p, qm, km, vm, s) : launch_profile<64, false>(p, qm, km, vm, s);
+    if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    rc = baklava_launch_row_max(shape, q, k, prompt_len, P, T, lse2, p.redo_list, p.redo_count, 2 * kRedoGrid, p.error, s);
     if (rc) return rc;
-    cudaError_t err = shape->D == 128 ? launch_profile<128>(p, qm, km, vm, s) : launch_profile<64>(p, qm, km, vm, s);
+    err = shape->D == 128 ? launch_profile<128, true>(p, qm, km, vm, s) : launch_profile<64, true>(p, qm, km, vm, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
     const int n = P * shape->Hq;
     profile_mean_kernel<<<(n + 127) / 128, 128, 0, s>>>(p);

@@ -12,11 +12,13 @@ from harness import assert_close, f64
 pytestmark = pytest.mark.gpu
 
 
-def _run(P, Hq, Hkv, T, D, lens=None, seed=3, want_tokens=True, v=None):
+def _run(P, Hq, Hkv, T, D, lens=None, seed=3, want_tokens=True, v=None, k_edit=None):
     dev = "cuda"
     shape = bk.make_shape(1, Hq, Hkv, D)
     q = synth.normal_bf16(seed, 1, (P, Hq, T, D), dev)
     k = synth.normal_bf16(seed, 2, (P, Hkv, T, D), dev)
+    if k_edit is not None:
+        k = k_edit(k)
     if v is None:
         v = synth.normal_bf16(seed, 3, (P, Hkv, T, D), dev)
     plen = None if lens is None else torch.tensor(lens, dtype=torch.int32, device=dev)
@@ -52,6 +54,27 @@ def test_many_key_tiles_wrap_the_rings():
     # ten 128-key tiles per row block: every stage, accumulator and probability buffer is reused several times
     _run(P=1, Hq=2, Hkv=1, T=1200, D=128, want_tokens=True, lens=[1170])
     _run(P=1, Hq=2, Hkv=2, T=900, D=64, want_tokens=False)
+
+
+def test_key_far_above_the_first_tile_stays_in_range():
+    # logits of one late key tower over everything in the first key tile, but by less than the fp32 range:
+    # the one-pass kernel's probabilities exceed 1 there and the cosines must still come out right
+    def edit(k):
+        k = k.clone()
+        k[:, :, 300] *= 12.0
+        return k
+    _run(P=1, Hq=4, Hkv=2, T=520, D=128, k_edit=edit)
+
+
+def test_key_beyond_the_range_is_redone_exactly():
+    # here the gap is hundreds of octaves: the one-pass kernel overflows on the rows that see the key, flags
+    # their row blocks, and the exact two-pass kernel redoes them; rows before the key are finished in one pass
+    def edit(k):
+        k = k.clone()
+        k[:, :, 400] *= 300.0
+        return k
+    _run(P=2, Hq=4, Hkv=2, T=650, D=128, k_edit=edit, lens=[650, 500])
+    _run(P=1, Hq=2, Hkv=1, T=300, D=64, k_edit=edit if False else (lambda k: torch.cat([k[:, :, :200], k[:, :, 200:] * 250.0], dim=2)))
 
 
 def test_group_of_seven():
