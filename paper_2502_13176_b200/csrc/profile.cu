@@ -3,8 +3,8 @@
 // head's input V_t and its output O_t, averaged over the prompt's tokens.
 //
 // One pass on the 5th-generation tensor cores.  The cosine does not change when a row of O is scaled, so
-// the softmax is left unnormalised and needs only a stabiliser per row, for which the row's largest logit in
-// the first key tile serves: p = exp2(s - reference), no running maximum, no sum, no rescaling of O, no
+// the softmax is left unnormalised and needs only a stabiliser per row, for which the row's largest logit
+// among its first eight keys serves: p = exp2(s - reference), no running maximum, no sum, no rescaling of O, no
 // division.  (Rows whose later logits leave the fp32 range that way are detected in the epilogue and redone
 // by a second instantiation that takes the true row maxima from a row pass; see profile_pv_block.)
 // A CTA owns 128 query rows: the Q tile stays in shared memory, K and V tiles of 128 keys stream through
@@ -59,7 +59,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // kExact = false: one pass.  The softmax needs a stabiliser per row, not the row's true maximum: the
-// largest logit among the row's keys in the FIRST key tile serves (every row sees key 0, so it exists),
+// largest logit among the row's first eight keys serves (every row sees key 0, so it exists),
 // probabilities of later keys may then exceed 1, which bf16 and the fp32 accumulator hold up to 2^127.
 // A row whose later logits are so far above that reference that O or its norm leaves the fp32 range
 // shows up as a non-finite cosine term in the epilogue; its row block is flagged in `redo` and done again
@@ -216,16 +216,15 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
             tc::fence_after_sync();
             uint32_t v[32];
             if (!kExact && it == 0) {
-                // reference = largest logit of the row over the whole first key tile (all four column groups)
-                float mx = -INFINITY;
-#pragma unroll 1
-                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
-                    tc::tmem_ld_32x32(lane_addr + c0, v);
-                    tc::tmem_ld_wait();
+                // reference = the row's largest logit among the first eight keys (those of them it may see):
+                // every thread of the row reads the same eight columns, so the four agree without talking
+                uint32_t first[8];
+                tc::tmem_ld_32x32_x8(lane_addr, first);
+                tc::tmem_ld_wait();
+                float mx = __uint_as_float(first[0]);
 #pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (qb > 0 || c0 + c <= row) mx = fmaxf(mx, __uint_as_float(v[c]));
-                }
+                for (int c = 1; c < 8; ++c)
+                    if (qb > 0 || c <= row) mx = fmaxf(mx, __uint_as_float(first[c]));
                 lse = mx * p.scale_log2;
             }
             tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base, v);
