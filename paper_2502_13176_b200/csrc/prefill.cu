@@ -144,11 +144,12 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
                 if (!ok) break;
                 tc::fence_after_sync();
                 const uint32_t str_tile = base + (1 + s) * kTileBytes;
+                const uint64_t da = tc::desc_k_major_sw128(res_tile), db = tc::desc_k_major_sw128(str_tile);
 #pragma unroll
                 for (int ks = 0; ks < kKSteps; ++ks) {
-                    const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;    // 64-element span, then 32 B per step
-                    tc::umma_bf16(tmem_base + s * kTileRows, tc::desc_k_major_sw128(res_tile + off),
-                                  tc::desc_k_major_sw128(str_tile + off), idesc, ks > 0);
+                    // 64-element span, then 32 B per step; the descriptor's address field counts 16-byte units
+                    const uint32_t off = ((ks >> 2) * kBoxBytes + (ks & 3) * 32) >> 4;
+                    tc::umma_bf16(tmem_base + s * kTileRows, da + off, db + off, idesc, ks > 0);
                 }
                 // one commit per tile (a commit costs the tensor pipe about as much as a third of this tile's
                 // MMAs): the epilogue, which sees the accumulator complete, releases the stage for the producer

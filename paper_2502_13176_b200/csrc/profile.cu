@@ -167,11 +167,13 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
             auto issue_s = [&](int it) {                     // S_it = Q K_it^T into S buffer it & 1
                 const int s = it & 1, kv = it % kKvStages;
                 const uint32_t k_tile = stage0 + kv * kStageBytes;
+                // a descriptor's address field is (address >> 4), so stepping through a tile is an addition: the
+                // issuing thread's instruction count per MMA is what bounds this kernel
+                const uint64_t dq = tc::desc_k_major_sw128(q_tile), dk = tc::desc_k_major_sw128(k_tile);
 #pragma unroll
                 for (int ks = 0; ks < kKSteps; ++ks) {
-                    const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-                    tc::umma_bf16(tmem_base + s * kTileRows, tc::desc_k_major_sw128(q_tile + off),
-                                  tc::desc_k_major_sw128(k_tile + off), idesc_s, ks > 0);
+                    const uint32_t off = ((ks >> 2) * kBoxBytes + (ks & 3) * 32) >> 4;
+                    tc::umma_bf16(tmem_base + s * kTileRows, dq + off, dk + off, idesc_s, ks > 0);
                 }
             };
             for (int g = 0; g < 2 && g < n_it && ok; ++g) {
@@ -188,10 +190,11 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
                 if (!ok) break;
                 tc::fence_after_sync();
                 const uint32_t v_tile = stage0 + kv * kStageBytes + kTileBytes;
+                const uint64_t dv = tc::desc_mn_major_sw128(v_tile, kBoxBytes);
 #pragma unroll
                 for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step = 8 columns of the probability tile
                     tc::umma_bf16_ts(tmem_base + kOColumn, tmem_base + kPColumn + s * kPColumns + ks * 8,
-                                     tc::desc_mn_major_sw128(v_tile + ks * 2048, kBoxBytes), idesc_o, (it > 0) || (ks > 0));
+                                     dv + (ks * 2048 >> 4), idesc_o, (it > 0) || (ks > 0));
                 }
                 if (it + 2 < n_it) issue_s(it + 2);          // into the S buffer tile `it` has just left
                 tc::umma_commit(smem_u32(&bar_group[(it + 2) % kGroupRing]));
