@@ -4,6 +4,7 @@ the smallest capacities, from the seeded inputs alone."""
 import numpy as np
 import pytest
 
+from paper_2502_13176_b200 import binding as bk
 from paper_2502_13176_b200 import workloads as wl
 
 from harness import Session
@@ -25,13 +26,14 @@ def _sampled_heads(s, count):
     return sorted(set(heads))
 
 
-@pytest.mark.parametrize("w,steps,count", [(wl.LLAMA3_8B_32K, 3, 6), (wl.QWEN25_7B_8K_B16, 2, 6)],
-                         ids=["llama3-8b-32k", "qwen2.5-7b-8k-b16"])
-def test_full_workload_sampled_heads(w, steps, count):
+@pytest.mark.parametrize("w,steps,count,kv", [(wl.LLAMA3_8B_32K, 3, 6, bk.KV_BF16), (wl.QWEN25_7B_8K_B16, 2, 6, bk.KV_BF16),
+                                             (wl.LLAMA3_8B_32K, 2, 4, bk.KV_FP8_E4M3)],
+                         ids=["llama3-8b-32k", "qwen2.5-7b-8k-b16", "llama3-8b-32k-fp8"])
+def test_full_workload_sampled_heads(w, steps, count, kv):
     probe = Session(w, heads=[], prefill=False)            # capacities only, to choose the sample
     heads = _sampled_heads(probe, count)
     del probe
-    s = Session(w, heads=heads)
+    s = Session(w, heads=heads, kv_dtype=kv)
     assert int(s.cap.max()) > 2 * int(s.cap.min())          # the budgets really are ragged
     for (b, l, h) in heads:
         s.check_state(b, l, h, "after prefill")
