@@ -198,6 +198,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     constexpr int kNTiles = D / 8;                     // 8-wide output column blocks
     constexpr int kTT = kFp8 ? 2 * kTileTokens : kTileTokens;       // tokens per stage
     constexpr int kBlocks = kTT / (kConsumerWarps * kWarpTokens);    // 16-token blocks per warp and stage
+    static_assert(kFp8 || kBlocks == 1, "bf16 stages hold one 16-token block per warp");
     constexpr int kRowBytes = kFp8 ? D : 2 * D;
     constexpr int kTileBytes = kTT * kRowBytes;        // one K (or V) tile
     constexpr int kStageBytes = 2 * kTileBytes;
@@ -333,6 +334,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             }
             const uint32_t k_tile = ring + s * kStageBytes;
             const uint32_t v_tile = k_tile + kTileBytes;
+            if constexpr (kBlocks == 1) {
+            // one 16-token block per warp and stage
 #pragma unroll
             for (int blk = 0; blk < kBlocks; ++blk) {
             const int r0 = (warp * kBlocks + blk) * kWarpTokens;     // this block's rows inside the tile
@@ -472,6 +475,173 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                     mma_bf16(o[2 * j2], pa0, pa2, vb[0], vb[1]);
                     mma_bf16(o[2 * j2 + 1], pa0, pa2, vb[2], vb[3]);
                 }
+                }
+            }
+            }
+            } else {
+            // several 16-token blocks per warp and stage (FP8 rows): one softmax update over all of them,
+            // which halves the serial part per token and gives the MMAs of the blocks to the scheduler together
+            const int w0 = warp * kBlocks * kWarpTokens;             // this warp's rows inside the tile
+            const int wtok0 = begin + it * kTT + w0;                 // their first token
+            if (wtok0 < end) {
+#pragma unroll
+                for (int blk = 0; blk < kBlocks; ++blk) {            // per 16-token block: patch the tile where needed
+                    const int r0 = w0 + blk * kWarpTokens;
+                    const int tok0 = wtok0 + blk * kWarpTokens;
+                    const int valid = kBlocks == 1 ? min(kWarpTokens, end - tok0)
+                                                   : max(0, min(kWarpTokens, end - tok0));   // rows of the block inside the chunk
+                    if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
+                        // step 1 (Eq. 4): the new token's row replaces whatever the tile holds at the free slot,
+                        // in shared memory for this pass and in the slab for the steps to come
+                        constexpr int kVec = D / 8;
+                        const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
+                        const int64_t row = row0 + hs.f;
+                        uint8_t* k_ptr = ring_ptr + s * kStageBytes;
+                        if (kFp8) {                          // quantise the row: eight elements per lane and operand
+                            for (int i = lane; i < 2 * kVec; i += 32) {
+                                const bool is_v = i >= kVec;
+                                const int c = is_v ? i - kVec : i;
+                                const uint4 raw = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
+                                const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + (is_v ? 3 : 1)]);
+                                *reinterpret_cast<uint2*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c >> 1) +
+                                                          (c & 1) * 8) = val;
+                                uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
+                                *(reinterpret_cast<uint2*>(slab + row * D) + c) = val;
+                            }
+                        } else {
+                            for (int i = lane; i < 2 * kVec; i += 32) {
+                                const bool is_v = i >= kVec;
+                                const int c = is_v ? i - kVec : i;
+                                const uint4 val = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
+                                *reinterpret_cast<uint4*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c)) = val;
+                                *(reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c) = val;
+                            }
+                        }
+                        if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
+                        __syncwarp();
+                    }
+                    if (kByPosition && pos_evict && lane < valid && tok0 + lane != hs.f) {
+                        const int ps = p.pos[row0 + tok0 + lane];
+                        if (ps >= p.n_sink && ps <= window_from && ps < old_pos) { old_pos = ps; old_slot = tok0 + lane; }
+                    }
+                    // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
+                    if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
+                        uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
+                        constexpr int kPieces = kRowBytes / 16;     // 16-byte pieces of a row
+                        for (int i = lane; i < kWarpTokens * kPieces; i += 32) {
+                            const int r = i / kPieces, c = i % kPieces;
+                            if (r >= valid || tok0 + r == hole)
+                                *reinterpret_cast<uint4*>(v_ptr + tile_offset(r0 + r, c)) = make_uint4(0, 0, 0, 0);
+                        }
+                        __syncwarp();
+                    }
+                }
+                // S = Q K^T for the warp's 16 * kBlocks tokens: 8-token column blocks, all under one softmax update
+                constexpr int kCols = 2 * kBlocks;
+                float sacc[kCols][4];
+#pragma unroll
+                for (int t = 0; t < kCols; ++t) { sacc[t][0] = sacc[t][1] = sacc[t][2] = sacc[t][3] = 0.0f; }
+#pragma unroll
+                for (int sb = 0; sb < kBlocks; ++sb) {
+                    const int r0 = w0 + sb * kWarpTokens;
+                    if (kFp8) {
+#pragma unroll
+                        for (int kk = 0; kk < D / 32; ++kk) {     // 32 channels per load: two k-steps for both token blocks
+                            uint32_t kb[4];
+                            ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * kk + (lm & 1)), kb);
+#pragma unroll
+                            for (int c = 0; c < 2; ++c) {
+                                const int ks = 2 * kk + c;
+                                mma_f16(sacc[2 * sb], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[c]),
+                                        fp8::f16x2_from_e4m3x2(kb[c] >> 16));
+                                mma_f16(sacc[2 * sb + 1], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[2 + c]),
+                                        fp8::f16x2_from_e4m3x2(kb[2 + c] >> 16));
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int ks = 0; ks < kKSteps; ++ks) {
+                            uint32_t kb[4];
+                            ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kb);
+                            mma_bf16(sacc[2 * sb], qa0[ks], qa2[ks], kb[0], kb[1]);
+                            mma_bf16(sacc[2 * sb + 1], qa0[ks], qa2[ks], kb[2], kb[3]);
+                        }
+                    }
+                }
+                // this thread: row qrow, tokens wtok0 + 8 t + qcol + {0, 1}
+                float sv[2 * kCols];
+                bool ok[2 * kCols];
+#pragma unroll
+                for (int t = 0; t < kCols; ++t)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int tok = wtok0 + 8 * t + qcol + e;
+                        sv[2 * t + e] = sacc[t][e] * scale_k;
+                        ok[2 * t + e] = tok < end && tok != hole;
+                    }
+                float mx = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 2 * kCols; ++i) mx = fmaxf(mx, ok[i] ? sv[i] : -INFINITY);
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run, mx);
+                const float corr = (m_new == -INFINITY) ? 1.0f : exp2f(m_run - m_new);
+                float pv[2 * kCols];
+#pragma unroll
+                for (int i = 0; i < 2 * kCols; ++i) pv[i] = ok[i] ? exp2f(sv[i] - m_new) : 0.0f;
+                float psum = (pv[0] + pv[1]) + (pv[2] + pv[3]);
+#pragma unroll
+                for (int sb = 1; sb < kBlocks; ++sb) psum += (pv[4 * sb] + pv[4 * sb + 1]) + (pv[4 * sb + 2] + pv[4 * sb + 3]);
+                l_run = l_run * corr + psum;
+                m_run = m_new;
+                if (keep_logits && qrow < G) {
+#pragma unroll
+                    for (int t = 0; t < kCols; ++t) {
+                        const int tok = wtok0 + 8 * t + qcol;
+                        __half* dst = prob_h + (int64_t)qrow * C + tok;
+                        if (tok + 1 < end) *reinterpret_cast<__half2*>(dst) = __floats2half2_rn(pv[2 * t], pv[2 * t + 1]);
+                        else if (tok < end) dst[0] = __float2half_rn(pv[2 * t]);
+                    }
+                    if ((lane & 3) == 0) {
+#pragma unroll
+                        for (int sb = 0; sb < kBlocks; ++sb)      // the reference maximum of every 16-token block written
+                            if (wtok0 + sb * kWarpTokens < end) mref_h[qrow * (C >> 4) + (wtok0 >> 4) + sb] = m_new;
+                    }
+                }
+                if (__any_sync(0xffffffffu, corr != 1.0f)) {
+#pragma unroll
+                    for (int j = 0; j < kNTiles; ++j) { o[j][0] *= corr; o[j][1] *= corr; }
+                }
+                if (kFp8) {
+                    // a register of the transposed load = two tokens x two adjacent channels; the permute puts the
+                    // even channel's token pair in the low half and the odd channel's in the high half.
+                    // o[2 c] collects channels 16 c + 0, 2, .., 14 and o[2 c + 1] channels 16 c + 1, 3, .., 15.
+#pragma unroll
+                    for (int c2 = 0; c2 < D / 32; ++c2) {
+#pragma unroll
+                        for (int sb = 0; sb < kBlocks; ++sb) {
+                            const uint32_t pa0 = pack_f16(pv[4 * sb], pv[4 * sb + 1]), pa2 = pack_f16(pv[4 * sb + 2], pv[4 * sb + 3]);
+                            uint32_t vb[4];
+                            ldmatrix_x4_trans(v_tile + tile_offset(w0 + sb * kWarpTokens + (lm & 1) * 8 + li8, 2 * c2 + (lm >> 1)), vb);
+#pragma unroll
+                            for (int h2 = 0; h2 < 2; ++h2) {
+                                const uint32_t lo = __byte_perm(vb[2 * h2], 0u, 0x3120), hi = __byte_perm(vb[2 * h2 + 1], 0u, 0x3120);
+                                const int c = 2 * c2 + h2;
+                                mma_f16(o[2 * c], pa0, pa2, fp8::f16x2_from_e4m3x2(lo), fp8::f16x2_from_e4m3x2(hi));
+                                mma_f16(o[2 * c + 1], pa0, pa2, fp8::f16x2_from_e4m3x2(lo >> 16), fp8::f16x2_from_e4m3x2(hi >> 16));
+                            }
+                        }
+                    }
+                } else {
+                    // O += P V: V^T fragments through ldmatrix.trans, two 8-wide column blocks per load
+                    const uint32_t pa0 = pack_bf16(pv[0], pv[1]), pa2 = pack_bf16(pv[2], pv[3]);
+#pragma unroll
+                    for (int j2 = 0; j2 < kNTiles / 2; ++j2) {
+                        uint32_t vb[4];
+                        ldmatrix_x4_trans(v_tile + tile_offset(w0 + (lm & 1) * 8 + li8, 2 * j2 + (lm >> 1)), vb);
+                        mma_bf16(o[2 * j2], pa0, pa2, vb[0], vb[1]);
+                        mma_bf16(o[2 * j2 + 1], pa0, pa2, vb[2], vb[3]);
+                    }
                 }
             }
             }
