@@ -552,10 +552,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
 #pragma unroll
                             for (int c = 0; c < 2; ++c) {
                                 const int ks = 2 * kk + c;
-                                mma_f16(sacc[2 * sb], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[c]),
-                                        fp8::f16x2_from_e4m3x2(kb[c] >> 16));
-                                mma_f16(sacc[2 * sb + 1], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[2 + c]),
-                                        fp8::f16x2_from_e4m3x2(kb[2 + c] >> 16));
+                                uint32_t b0, b1;
+                                fp8::f16x4_from_e4m3x4(kb[c], b0, b1);
+                                mma_f16(sacc[2 * sb], qa0[ks], qa2[ks], b0, b1);
+                                fp8::f16x4_from_e4m3x4(kb[2 + c], b0, b1);
+                                mma_f16(sacc[2 * sb + 1], qa0[ks], qa2[ks], b0, b1);
                             }
                         }
                     } else {
@@ -627,8 +628,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                             for (int h2 = 0; h2 < 2; ++h2) {
                                 const uint32_t lo = __byte_perm(vb[2 * h2], 0u, 0x3120), hi = __byte_perm(vb[2 * h2 + 1], 0u, 0x3120);
                                 const int c = 2 * c2 + h2;
-                                mma_f16(o[2 * c], pa0, pa2, fp8::f16x2_from_e4m3x2(lo), fp8::f16x2_from_e4m3x2(hi));
-                                mma_f16(o[2 * c + 1], pa0, pa2, fp8::f16x2_from_e4m3x2(lo >> 16), fp8::f16x2_from_e4m3x2(hi >> 16));
+                                uint32_t even0, odd0, even1, odd1;               // tokens 0-7 and 8-15 of the block
+                                fp8::f16x4_from_e4m3x4(lo, even0, odd0);
+                                fp8::f16x4_from_e4m3x4(hi, even1, odd1);
+                                mma_f16(o[2 * c], pa0, pa2, even0, even1);
+                                mma_f16(o[2 * c + 1], pa0, pa2, odd0, odd1);
                             }
                         }
                     }

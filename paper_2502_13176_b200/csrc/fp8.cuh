@@ -20,6 +20,14 @@ __device__ __forceinline__ uint32_t f16x2_from_e4m3x2(uint32_t pair) {
     asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(d) : "h"(h));
     return d;
 }
+// four E4M3 codes (one register) -> fp16 pairs of the low and of the high half, exactly
+__device__ __forceinline__ void f16x4_from_e4m3x4(uint32_t four, uint32_t& lo, uint32_t& hi) {
+    asm("{\n\t.reg .b16 l, h;\n\t"
+        "mov.b32 {l, h}, %2;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, l;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
+        : "=r"(lo), "=r"(hi) : "r"(four));
+}
 // eight bf16 values (16 bytes) times `inv_scale` -> eight codes (8 bytes)
 __device__ __forceinline__ uint2 quantise8(uint4 raw, float inv_scale) {
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
