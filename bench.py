@@ -294,6 +294,9 @@ def main():
     ap.add_argument("--mixed-lengths", action="store_true",
                     help="prompts of different lengths (seeded, uniform in [T/8, T]) decoded at per-sequence "
                          "positions through baklava_decode_attn_varlen")
+    ap.add_argument("--per-layer", default="off", choices=["off", "calls", "graph"],
+                    help="one baklava_decode_attn_varlen call per layer instead of one call over all layers: "
+                         "issued one by one (calls) or captured once in a CUDA graph and replayed (graph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.workload == "profile":
@@ -343,6 +346,33 @@ def main():
         w = wl.scaled(w, name=w.name + "-mixed")
     else:
         sess.prefill_synthetic()
+    if args.per_layer != "off":
+        # layer by layer, as a model calls attention; positions live on the device and advance there
+        sess.per_layer_plans()
+        t_dev = torch.full((w.B,), w.T, dtype=torch.int32, device=dev)
+        sq, sk, sv = (torch.empty_like(t) for t in wl.decode_inputs(w, 0, sess.scales, dev))
+
+        def layer_calls():
+            sess.step_layers(sq, sk, sv, t_dev, step_flags)
+            t_dev.add_(1)
+        if args.per_layer == "graph":
+            side = torch.cuda.Stream(dev)
+            with torch.cuda.stream(side):
+                layer_calls()                                # once outside capture: attributes, first-use set-up
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    layer_calls()
+            torch.cuda.current_stream(dev).wait_stream(side)
+
+        def layered_step(q, k, v, flags=0):
+            sq.copy_(q, non_blocking=True); sk.copy_(k, non_blocking=True); sv.copy_(v, non_blocking=True)
+            if args.per_layer == "graph":
+                graph.replay()
+            else:
+                layer_calls()
+            return sess.out
+        sess.step = layered_step
+        w = wl.scaled(w, name=w.name + "-per-layer-" + args.per_layer)
     feeds = [wl.decode_inputs(w, i, sess.scales, dev) for i in range(2 * total)]
     torch.cuda.synchronize(dev)
 
@@ -426,7 +456,7 @@ def main():
                          "peak_kind": peak_kind, "kernel": "decode_chunk_kernel",
                          "note": "events bracket one call = attention kernel + score/evict kernel"},
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": (1 if args.policy == "window" else 2) * args.steps,
+            "gpu_launches": (1 if args.policy == "window" else 2) * args.steps * (w.L if args.per_layer != "off" else 1),
             "clocks": clocks.summary(t_open, t_close),
         }
         if world == 1 and not args.no_cpu_baseline:

@@ -70,6 +70,22 @@ class DecodeSession:
                                       self.plan, self.ws)
         return self.out
 
+    def per_layer_plans(self):
+        """One plan and workspace per layer, for callers that run attention layer by layer (as a model does)."""
+        n_sm = torch.cuda.get_device_properties(self.device).multi_processor_count
+        self.layer_plans = []
+        for l in range(self.lb, self.le):
+            plan = bk.baklava_decode_plan(self.shape, self.cap, self.w.B, l, l + 1, self.stride, n_sm=n_sm).to(self.device)
+            self.layer_plans.append((plan, bk.decode_workspace(plan, self.device)))
+
+    def step_layers(self, q, k_new, v_new, t_pos, flags=0):
+        """One decode step as one call per layer; t_pos: device int32 [B] (so that the sequence of calls can be
+        captured in a CUDA graph and replayed with the positions advanced on the device)."""
+        for i, (plan, ws) in enumerate(self.layer_plans):
+            bk.baklava_decode_attn_varlen(self.shape, self.cache, q[i:i + 1], k_new[i:i + 1], v_new[i:i + 1], t_pos,
+                                          self.out[i:i + 1], self.lse[i:i + 1], flags, plan, ws)
+        return self.out
+
     def retained_kv_bytes(self):
         """Bytes of K and V in valid rows of the session's layers: what one step must read."""
         n = int(self.cache.len[:, self.lb:self.le].sum().item())
