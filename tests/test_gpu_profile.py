@@ -77,6 +77,17 @@ def test_key_beyond_the_range_is_redone_exactly():
     _run(P=1, Hq=2, Hkv=1, T=300, D=64, k_edit=edit if False else (lambda k: torch.cat([k[:, :, :200], k[:, :, 200:] * 250.0], dim=2)))
 
 
+def test_rows_on_both_sides_of_the_range_limit():
+    # a late key whose logits reach a few hundred octaves for some rows and stay small for others: some rows of a
+    # block overflow (the block is redone exactly), others would have been fine either way
+    def edit(k):
+        k = k.clone()
+        k[:, :, 200] *= 40.0
+        return k
+    _run(P=2, Hq=4, Hkv=2, T=400, D=128, k_edit=edit)
+    _run(P=1, Hq=2, Hkv=1, T=300, D=64, k_edit=edit)
+
+
 def test_group_of_seven():
     _run(P=1, Hq=7, Hkv=1, T=150, D=128, want_tokens=False)
 
