@@ -156,3 +156,16 @@ def test_varlen_argument_errors():
     assert rc == -1
     with pytest.raises(bk.BaklavaError):
         bk.baklava_decode_attn(s.shape, s.cache, q, kn, vn, -1, s.out, s.lse, 0, s.plan, s.ws)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_prompt_lengths_and_idle_patterns(seed):
+    rng = np.random.default_rng(500 + seed)
+    B = int(rng.integers(2, 6))
+    w = wl.scaled(wl.TINY, B=B, D=int(rng.choice([64, 128])), budget=float(rng.choice([0.125, 0.25, 0.5])),
+                  seed=wl.MASTER_SEED + 200 + seed)
+    lens = [int(x) for x in rng.integers(0, w.T + 1, size=B)]
+    s = VarlenSession(w, lens, chunk_tokens=int(rng.choice([0, 64, 192])))
+    for i in range(6):
+        idle = tuple(int(b) for b in range(B) if rng.random() < 0.3)
+        s.step_varlen(i, idle=idle)
