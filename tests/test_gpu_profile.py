@@ -117,3 +117,46 @@ def test_importance_from_profile_matches_oracle_end_to_end():
         s_ref[:, l] = op.profile_heads(f64(q), f64(k), f64(v))
     got = bk.baklava_importance(shape, s_dev)
     np.testing.assert_allclose(got, op.kv_importance(s_ref, Hq // Hkv), atol=1e-3)
+
+
+def test_profile_to_budgets_chain_at_four_total_budgets():
+    """The whole one-time pass of the method in small: profile every layer over the prompts (device), reduce to
+    KV-cache importance (host), allocate at 10 / 30 / 50 / 70 % of dense (host) -- against the oracle's chain."""
+    from oracle import allocation as oalloc
+    dev = "cuda"
+    P, L, Hq, Hkv, T, D, page = 4, 3, 8, 2, 256, 128, 16
+    shape = bk.make_shape(L, Hq, Hkv, D)
+    s_dev = np.zeros((P, L, Hq), dtype=np.float32)
+    s_ref = np.zeros((P, L, Hq))
+    ws = torch.empty((bk.baklava_profile_workspace_size(shape, P, T),), dtype=torch.uint8, device=dev)
+    for l in range(L):
+        q = synth.normal_bf16(40 + l, 1, (P, Hq, T, D), dev)
+        k = synth.normal_bf16(40 + l, 2, (P, Hkv, T, D), dev)
+        # heads differ: some value rows share a common direction, so their outputs resemble their inputs more
+        v = synth.normal_bf16(40 + l, 3, (P, Hkv, T, D), dev)
+        common = synth.normal_bf16(40 + l, 4, (1, Hkv, 1, D), dev).float()
+        mix = torch.tensor([0.0, 1.5], device=dev).reshape(1, Hkv, 1, 1) * (l + 1)
+        v = (v.float() + mix * common).to(torch.bfloat16)
+        hc = torch.empty((P, Hq), dtype=torch.float32, device=dev)
+        bk.baklava_profile_heads(shape, q, k, v, None, P, T, hc, None, ws)
+        torch.cuda.synchronize()
+        s_dev[:, l] = hc.cpu().numpy()
+        s_ref[:, l] = op.profile_heads(f64(q), f64(k), f64(v))
+    imp_dev = bk.baklava_importance(shape, s_dev)
+    imp_ref = op.kv_importance(s_ref, Hq // Hkv)
+    np.testing.assert_allclose(imp_dev, imp_ref, atol=1e-3)
+    assert imp_ref.max() - imp_ref.min() > 0.05                     # the heads really differ
+    t = float(np.median(imp_ref))
+    for pct in (10, 30, 50, 70):
+        base_pages = max(1, T * pct // 100 // page)
+        total = base_pages * L * Hkv * page
+        cap, off, stride = bk.baklava_allocate(shape, imp_dev, t, 1, 2, total, page, (T // page) * page)
+        # the host code on the device's importances = the oracle's rule on the same numbers, bit for bit
+        ocap, ooff, ostride = oalloc.allocate(imp_dev, t, 1, 2, base_pages * L * Hkv, 1, T // page, page)
+        np.testing.assert_array_equal(cap, ocap)
+        np.testing.assert_array_equal(off, ooff)
+        assert stride == ostride == total
+        # and, unless an importance sits within the fp32 noise of the threshold, the oracle's own chain agrees
+        if np.abs(imp_ref - t).min() > 2e-3:
+            rcap, _, _ = oalloc.allocate(imp_ref, t, 1, 2, base_pages * L * Hkv, 1, T // page, page)
+            np.testing.assert_array_equal(cap, rcap)
