@@ -399,6 +399,19 @@ def main():
     sess.check_status()
     elapsed_ms = ev[0].elapsed_time(ev[1])
 
+    # ---- per-step spread: the same steps again with an event after each (the events sit between the launches,
+    # so these steps lose the overlap of one step's tail with the next step's start and run a few us longer)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    marks[0].record()
+    for i in range(args.steps):
+        sess.step(*feeds[args.warmup + i], flags=step_flags)
+        marks[i + 1].record()
+    torch.cuda.synchronize(dev)
+    per_step_us = sorted(marks[i].elapsed_time(marks[i + 1]) * 1e3 for i in range(args.steps))
+
+    def pct(q):
+        return per_step_us[min(len(per_step_us) - 1, int(q * len(per_step_us)))]
+
     # ---- end to end: host buffers in, host buffer out, every step.  A step's q / k_new / v_new travel as one
     # pinned buffer (one copy), the output comes back as one
     def packed(ts):
@@ -450,6 +463,7 @@ def main():
                            "_varlen" if args.mixed_lengths else ""), "policy": args.policy,
                        "replicas": world},
             "tokens_per_s": whole_job_rate(world, w.B, args.steps, elapsed_ms),
+            "step_us_with_event_per_step": {"p10": pct(0.1), "median": pct(0.5), "p90": pct(0.9)},
             "pct_of_hbm_peak": 100.0 * gbs / world / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
