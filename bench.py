@@ -27,17 +27,45 @@ from paper_2502_13176_b200 import workloads as wl  # noqa: E402
 
 METRIC = "decode-step retained-KV GB/s"
 WORKLOADS = {"llama": wl.LLAMA3_8B_32K, "qwen": wl.QWEN25_7B_8K_B16, "tiny": wl.TINY}
-# dram bytes (read + write) per launch of the attention kernel from the committed ncu capture under
-# profiles/ (taken on 8 layers and scaled by rows); a workload without a current capture reports null.
-NCU_TRAFFIC_BYTES = {"llama3-8b-32k-30pct": 1318000000}
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+KERNEL_SOURCES = {"decode_chunk_kernel": ["decode.cu", "ptx.cuh", "common.h", "fp8.cuh"],
+                  "profile_pv_kernel": ["profile.cu", "ptx.cuh", "common.h"],
+                  "qk_pass_kernel": ["prefill.cu", "ptx.cuh", "common.h"]}
 
 
-def measured_peaks():
+def source_digest(kernel):
+    """Short hash of the source files a kernel is compiled from: the key that says whether an ncu capture
+    still describes the kernel as it is now."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel]:
+        with open(os.path.join(ROOT, "paper_2502_13176_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_traffic(workload, kernel):
+    """dram bytes (read + write) per launch from the table of ncu captures under profiles/: lines of
+    `workload kernel source-digest bytes`.  None when there is no capture of this workload, or when the
+    kernel's sources have changed since it was taken."""
+    if not os.path.exists(TRAFFIC_TABLE):
+        return None
+    digest = source_digest(kernel)
+    with open(TRAFFIC_TABLE) as f:
+        for line in f:
+            parts = line.split()
+            if len(parts) >= 4 and not line.startswith("#") and parts[0] == workload and parts[1] == kernel \
+                    and parts[2] == digest:
+                return int(parts[3])
+    return None
+
+
+def measured_peaks(key="hbm_gbs", fallback=6650.0):
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+            return float(json.load(f)[key]), "measured"
+    return fallback, "fallback"
 
 
 class ClockSampler:
@@ -140,7 +168,8 @@ class OracleSample:
         return "%d of %d heads x %d decode steps (fp64 numpy, one thread per head)" % (
             self.n_heads, self.w.L * self.w.Hkv * self.w.B, steps)
 
-    def step(self):
+    def step(self, threads=None):
+        """One oracle decode step over the sampled heads, one head per thread (`threads` = 1: one after another)."""
         from concurrent.futures import ThreadPoolExecutor
 
         from paper_2502_13176_b200 import synth
@@ -155,8 +184,11 @@ class OracleSample:
 
         t0 = time.perf_counter()
         with self.limits(limits=1):
-            with ThreadPoolExecutor(max_workers=self.cores) as pool:
-                nbytes = sum(pool.map(one, zip(self.twins, feeds)))
+            if threads == 1:
+                nbytes = sum(one(a) for a in zip(self.twins, feeds))
+            else:
+                with ThreadPoolExecutor(max_workers=self.cores) as pool:
+                    nbytes = sum(pool.map(one, zip(self.twins, feeds)))
         self.steps_done += 1
         return nbytes, time.perf_counter() - t0
 
@@ -168,8 +200,13 @@ def oracle_sample(w, seconds_target=12.0, max_steps=128):
     while steps < max_steps and total_s < seconds_target:
         nb, dt = sample.step()
         total_bytes += nb; total_s += dt; steps += 1
+    one_bytes, one_s, one_steps = 0, 0.0, 0                # the same sample on one core
+    while one_steps < max_steps and one_s < seconds_target / 2:
+        nb, dt = sample.step(threads=1)
+        one_bytes += nb; one_s += dt; one_steps += 1
     return {"value": total_bytes / total_s / 1e9, "unit": "GB/s", "cores": sample.cores, "kind": "oracle",
-            "sample": sample.describe(steps), "seconds": total_s}
+            "sample": sample.describe(steps), "seconds": total_s,
+            "single_thread": {"value": one_bytes / one_s / 1e9, "unit": "GB/s", "cores": 1, "steps": one_steps}}
 
 
 def run_reference(args, w):
@@ -196,6 +233,35 @@ def run_reference(args, w):
         "e2e": {"value": v, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def timed_calls(dev, call, steps, warmup):
+    """`warmup` untimed calls, then `steps` calls between two events; returns (ms per call, clocks summary)."""
+    for _ in range(warmup):
+        call()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    with ClockSampler(dev.index) as clocks:
+        t_open = time.perf_counter()
+        e0.record()
+        for _ in range(steps):
+            call()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        t_close = time.perf_counter()
+    return e0.elapsed_time(e1) / steps, clocks.summary(t_open, t_close)
+
+
+def tensor_line(metric, workload, config, kernel, flop, ms, clocks, args, launches, dtype="bf16"):
+    peak, peak_kind = measured_peaks("bf16_tflops", 1590.0)
+    tf = flop / (ms * 1e-3) / 1e12
+    return {"metric": metric, "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype,
+            "data": "synthetic", "config": dict(workload=workload, **config),
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                         "traffic": ncu_traffic(workload, kernel), "peak_kind": peak_kind, "kernel": kernel},
+            "ms_x_sm_ghz": None if not clocks.get("sm_mhz") else ms * clocks["sm_mhz"] * 1e-3,
+            "gpu_launches": launches * args.steps, "clocks": clocks}
+
+
 def run_profile_pass(args):
     """The one-time profiling pass (Algorithm 1 step 1) on the LLaMA-3-8B attention shape: one step = one
     layer's heads for all prompts.  Reported against the tensor roofline; not the headline benchmark."""
@@ -212,39 +278,44 @@ def run_profile_pass(args):
     del parts
     head_cos = torch.empty((P, w.Hq), dtype=torch.float32, device=dev)
     ws = torch.empty((bk.baklava_profile_workspace_size(shape, P, T),), dtype=torch.uint8, device=dev)
-    for _ in range(args.warmup):
-        bk.baklava_profile_heads(shape, q, k, v, None, P, T, head_cos, None, ws)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize(dev)
-    with ClockSampler(dev.index) as clocks:
-        t_open = time.perf_counter()
-        e0.record()
-        for _ in range(args.steps):
-            bk.baklava_profile_heads(shape, q, k, v, None, P, T, head_cos, None, ws)
-        e1.record()
-        torch.cuda.synchronize(dev)
-        t_close = time.perf_counter()
-    ms = e0.elapsed_time(e1) / args.steps
+    ms, clocks = timed_calls(dev, lambda: bk.baklava_profile_heads(shape, q, k, v, None, P, T, head_cos, None, ws),
+                             args.steps, args.warmup)
+    assert bk.workspace_error(ws) == 0
     flop = P * w.Hq * 2.0 * T * T * w.D          # QK^T and PV under the causal mask: 2 * (T^2 / 2) * D * 2 each
-    peak = 1653.9
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(path):
-        with open(path) as f:
-            peak = float(json.load(f)["bf16_tflops"])
-    tf = flop / (ms * 1e-3) / 1e12
-    print(json.dumps({"metric": "profiling-pass TFLOP/s (causal attention + cosine, one layer)", "value": tf,
-                      "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
-                      "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
-                      "config": {"workload": "profile-llama3-8b", "prompts": P, "prompt_tokens": T, "heads": w.Hq,
-                                 "kv_heads": w.Hkv, "head_dim": w.D},
-                      "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s",
-                                   "frac": tf / peak, "traffic": None,
-                                   "kernel": "profile_pv_kernel (tcgen05; one pass, exact redo of out-of-range row blocks)"},
-                      "gpu_launches": 4 * args.steps, "clocks": clocks.summary(t_open, t_close)}))
+    line = tensor_line("profiling-pass TFLOP/s (causal attention + cosine, one layer)", "profile-llama3-8b",
+                       {"prompts": P, "prompt_tokens": T, "heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D},
+                       "profile_pv_kernel", flop, ms, clocks, args, 4)
+    # end to end: the layer's Q, K, V come from pinned host memory and the head means go back, every step
+    host = [t.cpu().pin_memory() for t in (q, k, v)]
+    back = torch.empty(head_cos.shape, dtype=head_cos.dtype).pin_memory()
+
+    def e2e():
+        for d, h in zip((q, k, v), host):
+            d.copy_(h, non_blocking=True)
+        bk.baklava_profile_heads(shape, q, k, v, None, P, T, head_cos, None, ws)
+        back.copy_(head_cos, non_blocking=True)
+    e2e_ms, _ = timed_calls(dev, e2e, max(1, args.steps // 4), 1)
+    line["e2e"] = {"value": flop / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                   "h2d_bytes_per_step": sum(h.numel() * h.element_size() for h in host),
+                   "d2h_bytes_per_step": back.numel() * back.element_size()}
+    if not args.no_cpu_baseline:
+        from oracle import profiling as oprof
+        n, t0 = 0, time.perf_counter()
+        while n < 4 and time.perf_counter() - t0 < 15.0:       # a few full (prompt, head) instances
+            h = (n * 9) % w.Hq
+            oprof.head_similarity(q[0, h].double().cpu().numpy(), k[0, h // w.g].double().cpu().numpy(),
+                                  v[0, h // w.g].double().cpu().numpy(), T)
+            n += 1
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n * 2.0 * T * T * w.D / dt / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(),
+                                "kind": "oracle", "sample": "%d of %d (prompt, head) instances of %d tokens (fp64 numpy)" % (
+                                    n, P * w.Hq, T)}
+    print(json.dumps(line))
 
 
 def run_prefill_scores(args):
-    """Exact seeding of the heavy-hitter scores for one layer of a 32K prompt (two passes over Q K^T)."""
+    """Exact seeding of the heavy-hitter scores for one layer of a 32K prompt (two passes over Q K^T, or one
+    when the caller already has the rows' log-sum-exp)."""
     from paper_2502_13176_b200 import binding as bk, synth
     from paper_2502_13176_b200.engine import shape_of
 
@@ -257,22 +328,34 @@ def run_prefill_scores(args):
     k = synth.normal_bf16(w.seed, wl.T_PROFILE_K, (B, w.Hkv, T, w.D), dev)
     score = torch.empty((B, w.Hkv, T), dtype=torch.float32, device=dev)
     ws = torch.empty((bk.baklava_prefill_workspace_size(shape, B, T),), dtype=torch.uint8, device=dev)
-    for _ in range(args.warmup):
-        bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize(dev)
-    e0.record()
-    for _ in range(args.steps):
-        bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws)
-    e1.record()
-    torch.cuda.synchronize(dev)
-    ms = e0.elapsed_time(e1) / args.steps
+    ms, clocks = timed_calls(dev, lambda: bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws),
+                             args.steps, args.warmup)
+    assert bk.workspace_error(ws) == 0
     flop = 2 * B * w.Hq * 1.0 * T * T * w.D           # Q K^T under the causal mask, twice
-    tf = flop / (ms * 1e-3) / 1e12
-    print(json.dumps({"metric": "prompt-score seeding TFLOP/s (one layer)", "value": tf, "unit": "TFLOP/s",
-                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "dtype": "bf16",
-                      "config": {"workload": "prefill-scores-llama3-8b", "batch": B, "prompt_tokens": T},
-                      "gpu_launches": 2 * args.steps}))
+    line = tensor_line("prompt-score seeding TFLOP/s (one layer)", "prefill-scores-llama3-8b",
+                       {"batch": B, "prompt_tokens": T}, "qk_pass_kernel", flop, ms, clocks, args, 2)
+    host = [t.cpu().pin_memory() for t in (q, k)]
+    back = torch.empty(score.shape, dtype=score.dtype).pin_memory()
+
+    def e2e():
+        for d, h in zip((q, k), host):
+            d.copy_(h, non_blocking=True)
+        bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws)
+        back.copy_(score, non_blocking=True)
+    e2e_ms, _ = timed_calls(dev, e2e, max(1, args.steps // 4), 1)
+    line["e2e"] = {"value": flop / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                   "h2d_bytes_per_step": sum(h.numel() * h.element_size() for h in host),
+                   "d2h_bytes_per_step": back.numel() * back.element_size()}
+    if not args.no_cpu_baseline:
+        from oracle.prefill import prefill_scores as oracle_scores
+        Tc = min(T, 4096)                                  # the oracle forms a Tc x Tc matrix per query head
+        t0 = time.perf_counter()
+        oracle_scores(q[0, :w.g, :Tc].double().cpu().numpy(), k[0, 0, :Tc].double().cpu().numpy())
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": 2 * w.g * 1.0 * Tc * Tc * w.D / dt / 1e12, "unit": "TFLOP/s",
+                                "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": "one KV group (%d query heads) of the first %d tokens (fp64 numpy)" % (w.g, Tc)}
+    print(json.dumps(line))
 
 
 def main():
@@ -298,6 +381,9 @@ def main():
                     help="one baklava_decode_attn_varlen call per layer instead of one call over all layers: "
                          "issued one by one (calls) or captured once in a CUDA graph and replayed (graph)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustain-seconds", type=float, default=1.0,
+                    help="after the K timed steps, keep stepping for at least this long (cycling the step inputs) "
+                         "and report that region too, with the SM clock seen under it; 0 = skip")
     args = ap.parse_args()
     if args.workload == "profile":
         return run_profile_pass(args)
@@ -399,6 +485,25 @@ def main():
     sess.check_status()
     elapsed_ms = ev[0].elapsed_time(ev[1])
 
+    # ---- sustained: a second or more of continuous stepping, the clock the GPU settles at under it
+    sustained = None
+    if args.sustain_seconds > 0:
+        est = max(elapsed_ms / args.steps, 1e-3)
+        n_sus = int(args.sustain_seconds * 1e3 / est) + 1
+        sv = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        with ClockSampler(local) as sus_clocks:
+            s_open = time.perf_counter()
+            sv[0].record()
+            for i in range(n_sus):
+                sess.step(*feeds[i % total], flags=step_flags)
+            sv[1].record()
+            torch.cuda.synchronize(dev)
+            s_close = time.perf_counter()
+        sus_ms = sv[0].elapsed_time(sv[1])
+        sustained = {"steps": n_sus, "seconds": sus_ms * 1e-3, "ms_per_step": sus_ms / n_sus,
+                     "clocks": sus_clocks.summary(s_open, s_close)}
+        sess.check_status()
+
     # ---- per-step spread: the same steps again with an event after each (the events sit between the launches,
     # so these steps lose the overlap of one step's tail with the next step's start and run a few us longer)
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
@@ -466,13 +571,22 @@ def main():
             "step_us_with_event_per_step": {"p10": pct(0.1), "median": pct(0.5), "p90": pct(0.9)},
             "pct_of_hbm_peak": 100.0 * gbs / world / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                         "frac": achieved / peak, "traffic": ncu_traffic(w.name, "decode_chunk_kernel"),
                          "peak_kind": peak_kind, "kernel": "decode_chunk_kernel",
                          "note": "events bracket one call = attention kernel + score/evict kernel"},
             "e2e": {"value": e2e_gbs, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": (1 if args.policy == "window" else 2) * args.steps * (w.L if args.per_layer != "off" else 1),
             "clocks": clocks.summary(t_open, t_close),
         }
+        mhz = line["clocks"].get("sm_mhz")
+        line["us_x_sm_ghz"] = None if not mhz else kernel_ms * 1e3 * mhz * 1e-3      # clock-normalised step time
+        if sustained:
+            sustained["value"] = bytes_per_step / (sustained["ms_per_step"] * 1e-3) / 1e9
+            sustained["unit"] = "GB/s"
+            sustained["frac_of_peak"] = sustained["value"] / peak
+            smhz = sustained["clocks"].get("sm_mhz")
+            sustained["us_x_sm_ghz"] = None if not smhz else sustained["ms_per_step"] * 1e3 * smhz * 1e-3
+            line["sustained"] = sustained
         if world == 1 and not args.no_cpu_baseline:
             cb = oracle_sample(w)
             cb.pop("seconds")

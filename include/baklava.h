@@ -13,13 +13,29 @@
  *  - "host" / "device" on a pointer says where the memory lives.  The caller owns
  *    every buffer; the library allocates nothing on the device and keeps no
  *    pointer after a call returns.  Scratch comes from a caller-supplied
- *    workspace whose size the *_workspace_size() functions return.
+ *    workspace whose size the *_workspace_size() functions return.  (One
+ *    exception, stated at its declaration: baklava_evict_static keeps its
+ *    scratch in an array inside the library image and remembers that array's
+ *    device address between calls.)
  *  - Device work is enqueued on `stream` (a cudaStream_t passed as void*) and the
  *    call returns without synchronising.  Argument errors are found on the host
  *    before anything is enqueued.  State errors found on the device (append into
  *    a full cache, inconsistent length) set bits in the cache's device `status`
  *    word, skip the offending head's update and leave the rest of the step
  *    intact; the caller reads the word after synchronising.
+ *  - No kernel waits without a limit.  A wait on a tile or on another block that
+ *    does not end within the limit (baklava_set_wait_limit; about 50 ms by default)
+ *    gives up: BAKLAVA_STATUS_TIMEOUT is set, the kernel first lets every copy it
+ *    has requested land, and the head it was working on keeps the state it had
+ *    before the step (no output, no score update, no append bookkeeping).  All
+ *    counters in the workspace return to zero, so the next step may run on the
+ *    same workspace.  The calls that take no cache (baklava_profile_heads,
+ *    baklava_prefill_scores) report the same event in the first 32-bit word of
+ *    their workspace: the call clears it, bit 0 set after synchronising means a
+ *    wait gave up and the results are not to be used.
+ *  - slab_off entries, capacities and seq_stride_tokens are multiples of 16 rows
+ *    (baklava_allocate produces such layouts); seq_stride_tokens is checked on the
+ *    host, a head whose offset or capacity is not is skipped with BAD_STATE.
  *  - bf16 tensors are row-major with the last index fastest; all device pointers
  *    must be 16-byte aligned.
  *  - Supported shapes: D in {64, 128}; Hq a multiple of Hkv with g = Hq / Hkv <= 8;
@@ -56,6 +72,10 @@ extern "C" {
                                         /*   recent_den), where the oldest row outside both is evicted:  */
                                         /*   the paper's evaluated policy, with no score traffic at all  */
 #define BAKLAVA_FLAG_NO_EVICT      4u   /* never evict; a cache that fills up stays full              */
+#define BAKLAVA_FLAG_TEST_STALL  256u   /* test aid, never set it in production: the first chunk of   */
+                                        /*   every head is fed its first 64 (FP8: 128) rows only, so    */
+                                        /*   that the bounded wait for the next ones runs out and the   */
+                                        /*   time-out path runs (use with a short baklava_set_wait_limit) */
 
 #define BAKLAVA_SCOPE_LAYER        0    /* Algorithm 2 inside each layer                              */
 #define BAKLAVA_SCOPE_MODEL        1    /* Algorithm 2 over all L * Hkv caches at once                */
@@ -211,10 +231,12 @@ int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t 
  *   v_new    device bf16 [layers, B, Hkv, D]
  *   out      device bf16 [layers, B, Hq, D]
  *   lse      device fp32 [layers, B, Hq] natural-log normaliser, or NULL
- *   items    device int32, the plan's items;  info: the plan's info
+ *   items    device int32, the plan's items (complete before the call is enqueued, or written by
+ *            earlier work on the same stream);  info: the plan's info
  *   ws       device workspace >= info->ws_bytes; must be zero-filled before its first use
  *            and not shared by steps that overlap in time; the library restores the
- *            parts that must be zero before it returns the stream to the caller.
+ *            parts that must be zero before it returns the stream to the caller, also
+ *            after a step that set BAKLAVA_STATUS_TIMEOUT.
  * A head with no valid row gives out = 0 and lse = -inf. */
 int baklava_decode_attn(const baklava_shape* shape, const baklava_cache* cache,
                         const void* q, const void* k_new, const void* v_new, int32_t t_pos,
@@ -233,6 +255,11 @@ int baklava_decode_attn_varlen(const baklava_shape* shape, const baklava_cache* 
                                const int32_t* items, const baklava_plan_info* info,
                                void* ws, size_t ws_bytes, void* stream);
 
+/* Upper bound, in SM clock cycles, of every wait inside the decode kernels from the next call on
+ * (process-wide; default 100 000 000, about 50 ms).  A wait that runs out sets BAKLAVA_STATUS_TIMEOUT
+ * as the conventions above describe.  sm_cycles > 0. */
+int baklava_set_wait_limit(int64_t sm_cycles);
+
 /* ------------------------------------------------------------------ bulk eviction (Eq. 5-6)
  * Cut dense prefilled heads of T tokens down to their capacities and compact them into
  * the slabs (the MAKE_CACHE of Algorithm 3).  Row t of head (layer, b, h) is token row
@@ -243,7 +270,16 @@ int baklava_decode_attn_varlen(const baklava_shape* shape, const baklava_cache* 
  * positions, and the R - n_sink - W rows of the rest that rank first by (score
  * descending, position ascending).  Kept rows land in slots 0 .. n'-1 in ascending
  * position with their scores; len = free_slot = n'.   reserve >= 1.
- *   ws   device workspace >= baklava_evict_workspace_size() bytes */
+ *   ws   device workspace >= baklava_evict_workspace_size() bytes
+ *
+ * In place (k_dense = v_dense = NULL; score_dense must be NULL too, the strides are ignored): the
+ * same rule applied to the len rows every slab already holds, with their own positions and scores
+ * (the latest position present takes the place of T - 1): a budget that shrank, a cache that filled
+ * up under NO_EVICT, a freed slot to close.  Eq. 5-6 remove rows and keep the order of the others:
+ * the kept rows move down to slots 0 .. n'-1 in the order they have in the slab (ascending position
+ * for a slab that baklava_evict filled); len = free_slot = n'.  Here T only sizes the workspace and
+ * must be at least the largest capacity in the layer range (a larger head is skipped with
+ * BAD_STATE, as is one whose len / free_slot are inconsistent). */
 int baklava_evict(const baklava_shape* shape, const baklava_cache* cache,
                   int32_t layer_begin, int32_t layer_end,
                   const void* k_dense, const void* v_dense, const float* score_dense, int32_t T,
@@ -302,7 +338,7 @@ int baklava_search_pick(const double* avg_loss, int32_t n, int32_t* best);
 
 /* ------------------------------------------------------------------ bulk eviction, no workspace
  * (No counterpart in the paper: this is a packaging variant of baklava_evict.)
- * Same operation, arguments and results as baklava_evict, for callers that cannot provide a
+ * Same operation, arguments, results and return codes as baklava_evict, for callers that cannot provide a
  * workspace because they cannot allocate device memory where the call is made: code running
  * inside a host framework whose memory pool is exhausted or frozen, plug-ins that are handed
  * only their input and output buffers, and start-up code that runs before an allocator exists.
@@ -312,7 +348,9 @@ int baklava_search_pick(const double* avg_loss, int32_t n, int32_t* best);
  *  - Limit: (layer_end - layer_begin) * B * Hkv * T <= BAKLAVA_EVICT_STATIC_MAX_ENTRIES;
  *    larger requests return BAKLAVA_ERR_WORKSPACE before anything is enqueued.
  *  - The first call on each device looks up the array's device address (the device must be
- *    current).  Make that first call outside any stream capture.
+ *    current) and the library remembers it.  Make that first call outside any stream capture.
+ *    The address dies with the device's context: a process that calls cudaDeviceReset must not
+ *    call this entry point afterwards.
  *  - All calls on a device share the one array and it keeps the previous call's contents.
  *    Every entry that is read is written earlier in the same call, so nothing has to be
  *    cleared; but two calls whose kernels overlap on the GPU (different streams) race on it.

@@ -56,3 +56,12 @@ def bulk_evict(K, V, pos, score, R, n_sink, recent_num, recent_den):
     order = keep[np.argsort(np.asarray(pos)[keep], kind="stable")]
     return (np.asarray(K)[order], np.asarray(V)[order], np.asarray(pos)[order],
             np.asarray(score)[order], order)
+
+
+def compact_in_place(K, V, pos, score, R, n_sink, recent_num, recent_den):
+    """The same cut applied to a cache as it stands: Eq. 5-6 take rows out and leave the others in
+    the order they had, whatever that order is.  Returns (K', V', pos', score', kept_index) with
+    kept_index ascending."""
+    keep = select_keep(pos, score, R, n_sink, recent_num, recent_den)
+    return (np.asarray(K)[keep], np.asarray(V)[keep], np.asarray(pos)[keep], np.asarray(score)[keep], keep)
+

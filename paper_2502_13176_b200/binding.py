@@ -14,6 +14,7 @@ import torch
 
 OK = 0
 FLAG_NO_APPEND, FLAG_NO_SCORE, FLAG_NO_EVICT = 1, 2, 4
+FLAG_TEST_STALL = 256
 SCOPE_LAYER, SCOPE_MODEL = 0, 1
 STATUS_OVERFLOW, STATUS_BAD_STATE, STATUS_TIMEOUT = 1, 2, 4
 KV_BF16, KV_FP8_E4M3 = 0, 1
@@ -94,6 +95,7 @@ def lib():
         L.baklava_output_error_workspace_size.restype = c_size_t
         L.baklava_output_error_workspace_size.argtypes = [c_int64]
         L.baklava_search_pick.argtypes = [POINTER(c_double), c_int32, POINTER(c_int32)]
+        L.baklava_set_wait_limit.argtypes = [c_int64]
         L.baklava_profile_workspace_size.restype = c_size_t
         L.baklava_profile_workspace_size.argtypes = [POINTER(Shape), c_int32, c_int32]
         _lib = L
@@ -180,7 +182,8 @@ class Cache:
     """Device buffers of a budgeted cache plus the struct the library reads.  Memory only."""
 
     def __init__(self, shape, cap, slab_off, seq_stride, B, device="cuda", kv_dtype=KV_BF16, kv_scale=None):
-        """kv_scale: float32 array [L, Hkv, 2] = (K scale, V scale) per head, for FP8 slabs."""
+        """kv_scale: float32 array [L, Hkv, 4] = (K scale, 1 / K scale, V scale, 1 / V scale) per head, for FP8
+        slabs; passed to the library as given."""
         self.shape, self.B, self.seq_stride = shape, int(B), int(seq_stride)
         self.kv_dtype = int(kv_dtype)
         self.cap_host = np.ascontiguousarray(cap, dtype=np.int32).reshape(shape.L, shape.Hkv)
@@ -191,13 +194,8 @@ class Cache:
         self.v_slab = torch.empty((rows, shape.D), dtype=slab_type, device=device)
         self.kv_scale = None
         if self.kv_dtype == KV_FP8_E4M3:
-            sc = np.ascontiguousarray(kv_scale, dtype=np.float32).reshape(shape.L, shape.Hkv, 2)
-            four = np.empty((shape.L, shape.Hkv, 4), dtype=np.float32)
-            four[..., 0], four[..., 2] = sc[..., 0], sc[..., 1]
-            four[..., 1] = np.float32(1.0) / sc[..., 0]        # float32 division, rounded once
-            four[..., 3] = np.float32(1.0) / sc[..., 1]
-            self.kv_scale_host = four
-            self.kv_scale = torch.from_numpy(four).to(device)
+            self.kv_scale_host = np.ascontiguousarray(kv_scale, dtype=np.float32).reshape(shape.L, shape.Hkv, 4).copy()
+            self.kv_scale = torch.from_numpy(self.kv_scale_host).to(device)
         self.pos = torch.full((rows,), -1, dtype=torch.int32, device=device)
         self.score = torch.zeros((rows,), dtype=torch.float32, device=device)
         self.len = torch.zeros((self.B, shape.L, shape.Hkv), dtype=torch.int32, device=device)
@@ -245,6 +243,16 @@ def baklava_decode_attn_varlen(shape, cache, q, k_new, v_new, t_pos, out, lse, f
                                             _ptr(plan.items_dev), ctypes.byref(plan.info), _ptr(ws),
                                             ws.numel() * ws.element_size(), _stream(stream)),
            "baklava_decode_attn_varlen")
+
+
+def baklava_set_wait_limit(sm_cycles):
+    _check(lib().baklava_set_wait_limit(int(sm_cycles)), "baklava_set_wait_limit")
+
+
+def workspace_error(ws):
+    """The error word baklava_profile_heads / baklava_prefill_scores leave in their workspace (0 = none);
+    synchronises."""
+    return int(ws[:4].view(torch.int32).item())
 
 
 def baklava_evict_workspace_size(shape, B, layers, T):

@@ -16,6 +16,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <climits>
 #include <cmath>
 #include <cstdint>
@@ -78,6 +79,7 @@ struct DecodeParams {
     int32_t* best_slot;            // [n_score_items]
     float scale_log2;   // log2(e) / sqrt(D)
     const float* kv_scale;   // FP8 slabs: [L, Hkv, 4] (K scale, its reciprocal, V scale, its reciprocal)
+    long long wait_cycles;   // SM clock cycles after which a wait on a tile gives up
 };
 
 struct Unit {
@@ -112,7 +114,8 @@ __device__ __forceinline__ HeadState head_state(const DecodeParams& p, const Uni
     h.n = p.len[u.st];
     h.f = p.free_slot[u.st];
     const bool no_append = (p.flags & BAKLAVA_FLAG_NO_APPEND) != 0;
-    h.bad = h.n < 0 || h.n > h.C || h.f < 0 || h.f > h.C || (!no_append && h.f > h.n);
+    h.bad = h.n < 0 || h.n > h.C || h.f < 0 || h.f > h.C || (!no_append && h.f > h.n) ||
+            (p.slab_off[u.head] & 15) != 0 || (h.C & 15) != 0;   // rows are read in 16-byte vectors of pos / score
     h.overflow = !no_append && h.n >= h.C;
     h.do_append = !no_append && !h.overflow && !h.bad;
     h.hole = (no_append && h.f < h.n) ? h.f : -1;
@@ -213,15 +216,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     __shared__ float sm_invL[kG];
     __shared__ int sm_last;
     __shared__ int sm_abort;
+    __shared__ int sm_issued;
     __shared__ int sm_old_pos[kConsumerWarps];
     __shared__ int sm_old_slot[kConsumerWarps];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.G;
+    grid_dependency_wait();                               // len / free_slot / slab rows / items come from earlier kernels
     const int4 item = p.items[blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
-    grid_dependency_wait();                               // len / free_slot / slab rows come from earlier kernels
     // Only now may the score kernel's CTAs become resident: they read len / free_slot before their own
     // dependency wait, and this order guarantees that the previous step's bookkeeping is complete by then
     // even when the whole grid is resident at once.
@@ -262,6 +266,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             mbar_init(smem_u32(&bar_empty[s]), kConsumerWarps);
         }
         sm_abort = 0;
+        sm_issued = 0;
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -277,10 +282,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         // ---------------- producer: one lane issues the TMA loads
         if (lane == 0) {
             const uint64_t stream_policy = l2_evict_first_policy();
-            for (int it = 0; it < n_tiles; ++it) {
+            int it = 0;
+            for (; it < n_tiles; ++it) {
                 const int s = it % kStages;
+                // test aid (BAKLAVA_FLAG_TEST_STALL): the first chunk of a head gets its first tile only, so that
+                // the consumers' bounded wait for the second one runs out; nothing is in flight by then
+                if ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0 && it == 1) break;
                 if (it >= kStages) {
-                    if (!mbar_wait(smem_u32(&bar_empty[s]), ((it / kStages) - 1) & 1)) {
+                    if (!mbar_wait(smem_u32(&bar_empty[s]), ((it / kStages) - 1) & 1, p.wait_cycles)) {
                         atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
                         sm_abort = 1;
                         break;
@@ -301,6 +310,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                     }
                 }
             }
+            sm_issued = it;
         }
     } else {
         // ---------------- consumers
@@ -327,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         bool alive = true;
         for (int it = 0; it < n_tiles && alive; ++it) {
             const int s = it % kStages;
-            if (!mbar_wait(smem_u32(&bar_full[s]), (it / kStages) & 1)) {
+            if (!mbar_wait(smem_u32(&bar_full[s]), (it / kStages) & 1, p.wait_cycles)) {
                 if (lane == 0) atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
                 alive = false;
                 break;
@@ -655,8 +665,19 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         if (!alive && lane == 0) sm_abort = 1;
     }
     __syncthreads();
-    if (sm_abort) return;                                   // a bounded wait gave up: status word says so
-
+    const int psz = partial_floats(G, D);                   // o, m, l, and the chunk's oldest evictable row
+    float* part = p.partial + (int64_t)blockIdx.x * psz;
+    const bool aborted = sm_abort != 0;                     // a bounded wait gave up: the status word says so
+    if (aborted) {
+        // The head's step is lost, but the launch stays consistent: no copy into this CTA's shared memory may be
+        // left in flight when it exits (bounded wait for every tile that was requested), and the chunk still
+        // arrives, with a mark, so that the head's counters return to zero and its bookkeeping is skipped.
+        if (tid == 0)
+            for (int t = max(0, sm_issued - kStages); t < sm_issued; ++t)
+                mbar_wait(smem_u32(&bar_full[t % kStages]), (t / kStages) & 1, p.wait_cycles);
+        if (tid < G) part[G * D + tid] = __int_as_float(0x7fc00000);
+    }
+    if (!aborted) {
     // ---- the four warps' states -> one partial for the chunk (the ring is idle now: reuse it)
     float* sm_o = reinterpret_cast<float*>(ring_ptr);       // [kConsumerWarps][G][D]
     if (warp < kConsumerWarps) {
@@ -688,8 +709,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         }
     }
     __syncthreads();
-    const int psz = partial_floats(G, D);                   // o, m, l, and the chunk's oldest evictable row
-    float* part = p.partial + (int64_t)blockIdx.x * psz;
     for (int i = tid; i < G * D; i += kThreads) {
         const int a = i / D, d = i - a * D;
         float mm = -INFINITY;
@@ -712,6 +731,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         part[G * D + 2 * G] = __int_as_float(bp);
         part[G * D + 2 * G + 1] = __int_as_float(bs);
     }
+    }
     __threadfence();
     __syncthreads();
     if (tid == 0) {
@@ -733,10 +753,21 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     for (int i = tid; i < n_ml; i += kThreads) {
         const int c = i / G, a = i - c * G;
         const float* pc = part0 + (int64_t)c * psz + G * D;
-        sm_mc[i] = __ldcg(pc + a);
+        const float mc = __ldcg(pc + a);
+        if (mc != mc) sm_abort = 1;                         // a chunk of this head gave up
+        sm_mc[i] = mc;
         sm_lc[i] = __ldcg(pc + G + a);
     }
     __syncthreads();
+    if (sm_abort) {
+        // lost step: no output, no bookkeeping; the counters go back to zero and the score pieces are told
+        if (tid == 0) {
+            p.stats[(int64_t)unit * 2 * kG] = __int_as_float(0x7fc00000);
+            p.arrive[unit] = 0;
+            if (keep_logits) st_release(p.ready + unit, 1);
+        }
+        return;
+    }
     if (tid < G) {
         float mm = -INFINITY;
         for (int c = 0; c < active; ++c) mm = fmaxf(mm, sm_mc[c * G + tid]);
@@ -872,7 +903,8 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
         Mq[a] = p.stats[(int64_t)unit * 2 * kG + a];
         iL[a] = p.stats[(int64_t)unit * 2 * kG + kG + a];
     }
-    const bool appended = hs.do_append;
+    const bool lost = Mq[0] != Mq[0];                      // the attention kernel gave the head's step up
+    const bool appended = hs.do_append && !lost;
     const int R = C - 1;
     const bool evict = appended && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n_hi > R;
     const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
@@ -881,7 +913,7 @@ __global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const Dec
     unsigned long long best = ~0ull;
     int best_slot = -1;
     // eight consecutive rows per thread: they share one 16-row block, hence one reference maximum per head
-    for (int j0 = begin + 8 * tid; j0 < end; j0 += 8 * kScoreThreads) {
+    for (int j0 = begin + 8 * tid; j0 < (lost ? begin : end); j0 += 8 * kScoreThreads) {
         float fac[G];
 #pragma unroll
         for (int a = 0; a < G; ++a) {
@@ -1064,6 +1096,8 @@ cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CU
 }  // namespace
 
 namespace {
+std::atomic<long long> g_wait_cycles{ptx::kWaitCycles};
+
 int decode_attn_impl(
         const baklava_shape* shape, const baklava_cache* cache,
         const void* q, const void* k_new, const void* v_new, int32_t t_pos, const int32_t* t_pos_seq,
@@ -1073,15 +1107,17 @@ int decode_attn_impl(
     int rc = baklava_check_shape(shape);
     if (rc) return rc;
     if (!cache || !q || !out || !items || !info || !ws) return BAKLAVA_ERR_INVALID_ARG;
-    if (flags & ~(BAKLAVA_FLAG_NO_APPEND | BAKLAVA_FLAG_NO_SCORE | BAKLAVA_FLAG_NO_EVICT)) return BAKLAVA_ERR_INVALID_ARG;
+    if (flags & ~(BAKLAVA_FLAG_NO_APPEND | BAKLAVA_FLAG_NO_SCORE | BAKLAVA_FLAG_NO_EVICT | BAKLAVA_FLAG_TEST_STALL))
+        return BAKLAVA_ERR_INVALID_ARG;
     const bool no_append = flags & BAKLAVA_FLAG_NO_APPEND;
     if (!no_append && (!k_new || !v_new)) return BAKLAVA_ERR_INVALID_ARG;
     if (!cache->k_slab || !cache->v_slab || !cache->pos || !cache->score || !cache->len || !cache->free_slot ||
         !cache->cap || !cache->slab_off || !cache->status || cache->B <= 0 || cache->seq_stride_tokens <= 0)
         return BAKLAVA_ERR_INVALID_ARG;
-    const void* ptrs[] = {q, k_new, v_new, out, cache->k_slab, cache->v_slab, items, ws};
+    const void* ptrs[] = {q, k_new, v_new, out, cache->k_slab, cache->v_slab, cache->pos, cache->score, items, ws};
     for (const void* ptr : ptrs)
         if (ptr && !baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
+    if (cache->seq_stride_tokens % 16 != 0) return BAKLAVA_ERR_INVALID_ARG;   // rows of pos / score go in 16-byte vectors
     if (info->layer_begin < 0 || info->layer_end > shape->L || info->layer_begin >= info->layer_end ||
         info->B != cache->B || info->n_items <= 0 || info->n_score_items <= 0 ||
         info->n_units != (info->layer_end - info->layer_begin) * cache->B * shape->Hkv)
@@ -1145,6 +1181,7 @@ int decode_attn_impl(
     p.best_slot = reinterpret_cast<int32_t*>(base + lay.best_off + 8 * (size_t)info->n_score_items);
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
     p.kv_scale = cache->kv_scale;
+    p.wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
@@ -1200,4 +1237,10 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_attn_varlen
     if (!t_pos) return BAKLAVA_ERR_INVALID_ARG;
     return decode_attn_impl(shape, cache, q, k_new, v_new, 0, t_pos, out, lse, flags, items, info, ws, ws_bytes,
                             stream);
+}
+
+extern "C" __attribute__((visibility("default"))) int baklava_set_wait_limit(int64_t sm_cycles) {
+    if (sm_cycles <= 0) return BAKLAVA_ERR_INVALID_ARG;
+    g_wait_cycles.store(sm_cycles, std::memory_order_relaxed);
+    return BAKLAVA_OK;
 }

@@ -8,6 +8,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+#include <climits>
 #include <cstdint>
 
 #include "baklava.h"
@@ -209,6 +211,171 @@ __global__ void __launch_bounds__(kCopyThreads) evict_copy_kernel(const EvictPar
     }
 }
 
+// ---------------------------------------------------------------- in place (no dense source)
+// The same rule applied to the rows a slab already holds (a budget that shrank, a cache that filled up under
+// NO_EVICT, a freed slot to close).  Eq. 5-6 remove rows and keep the order of the others, so the kept rows move
+// down to slots 0 .. n'-1 in the order they have in the slab; for a slab filled by baklava_evict that is
+// ascending position.  Rows only ever move to lower slots, so one CTA per head can move them block by block
+// (read a block of sources, synchronise, write) without staging a copy of the head.
+//
+// Rows are not in position order here, so ties at the score threshold are settled by a second radix select on
+// the position (earliest positions stay).
+
+// k-th largest 32-bit key among the rows for which key_of(j, &key) is true; returns the key and, in `want`,
+// how many rows with exactly that key belong to the top k.  Whole CTA.
+template <typename KeyOf>
+__device__ __forceinline__ uint32_t radix_select(int n, int k, KeyOf key_of, int* hist, uint32_t* sh_prefix,
+                                                 int* sh_want, int& want) {
+    uint32_t prefix = 0;
+    want = k;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int i = threadIdx.x; i < 256; i += kSelThreads) hist[i] = 0;
+        __syncthreads();
+        const uint32_t mask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
+        for (int j = threadIdx.x; j < n; j += kSelThreads) {
+            uint32_t key;
+            if (key_of(j, key) && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int left = want, bin = 255;
+            for (; bin > 0; --bin) {
+                if (hist[bin] >= left) break;
+                left -= hist[bin];
+            }
+            *sh_prefix = prefix | ((uint32_t)bin << shift);
+            *sh_want = left;
+        }
+        __syncthreads();
+        prefix = *sh_prefix;
+        want = *sh_want;
+        __syncthreads();
+    }
+    return prefix;
+}
+
+template <int kRowBytes>
+__global__ void __launch_bounds__(kSelThreads) evict_inplace_kernel(const EvictParams p) {
+    __shared__ int hist[256];
+    __shared__ int warp_sums[32];
+    __shared__ uint32_t sh_prefix;
+    __shared__ int sh_want;
+    __shared__ int sh_red[32];
+
+    const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const Where w = locate(p, unit);
+    const int C = p.cap[w.head];
+    const int R = C - p.reserve;
+    const int n = p.len[w.st], f = p.free_slot[w.st];
+    int32_t* order = p.kept + (int64_t)unit * p.T;           // source slot of every kept row, in slab order
+    if (R < 1 || C > p.T || n < 0 || n > C || f < 0 || f > n || (f < n && n >= C)) {
+        if (tid == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
+        return;                                              // the head is left as it is
+    }
+    const int span = n + (f < n ? 1 : 0);                    // slots 0 .. span-1 hold the n rows and, maybe, the hole
+    const int32_t* pos = p.pos + w.slab0;
+    float* score = p.score + w.slab0;
+
+    uint32_t thr_key = 0, thr_pos = 0;
+    int t_max = INT32_MIN, quota = 0;
+    const bool cut = n > R;
+    int W = 0;
+    if (cut) {
+        // the latest position present, the sinks and the rows of the recent window
+        for (int j = tid; j < span; j += kSelThreads)
+            if (j != f) t_max = max(t_max, pos[j]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t_max = max(t_max, __shfl_xor_sync(0xffffffffu, t_max, o));
+        if (lane == 0) sh_red[warp] = t_max;
+        __syncthreads();
+        t_max = sh_red[0];
+        for (int i = 1; i < kSelThreads / 32; ++i) t_max = max(t_max, sh_red[i]);
+        __syncthreads();
+        W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
+        int fixed = 0;
+        for (int j = tid; j < span; j += kSelThreads)
+            if (j != f && (pos[j] < p.n_sink || pos[j] > t_max - W)) ++fixed;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) fixed += __shfl_xor_sync(0xffffffffu, fixed, o);
+        if (lane == 0) sh_red[warp] = fixed;
+        __syncthreads();
+        fixed = 0;
+        for (int i = 0; i < kSelThreads / 32; ++i) fixed += sh_red[i];
+        __syncthreads();
+        quota = R - fixed;
+        if (quota < 0 || quota > n - fixed) {
+            if (tid == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
+            return;
+        }
+        if (quota > 0) {
+            const int lo_pos = p.n_sink, hi_pos = t_max - W;
+            auto is_cand = [&](int j) { return j != f && pos[j] >= lo_pos && pos[j] <= hi_pos; };
+            int want = 0;
+            thr_key = radix_select(span, quota, [&](int j, uint32_t& key) {
+                if (!is_cand(j)) return false;
+                key = ordered_bits(score[j]);
+                return true;
+            }, hist, &sh_prefix, &sh_want, want);
+            // of the rows exactly at the threshold the `want` earliest positions stay
+            int unused = 0;
+            const uint32_t inv = radix_select(span, want, [&](int j, uint32_t& key) {
+                if (!is_cand(j) || ordered_bits(score[j]) != thr_key) return false;
+                key = ~(uint32_t)pos[j];
+                return true;
+            }, hist, &sh_prefix, &sh_want, unused);
+            thr_pos = ~inv;                                   // rows at the threshold with pos <= thr_pos stay
+        }
+    }
+    // list the kept rows in slab order
+    int base = 0;
+    for (int j0 = 0; j0 < span; j0 += kSelThreads) {
+        const int j = j0 + tid;
+        bool keep = j < span && j != f;
+        if (keep && cut) {
+            const int ps = pos[j];
+            if (ps >= p.n_sink && ps <= t_max - W) {
+                const uint32_t key = ordered_bits(score[j]);
+                keep = quota > 0 && (key > thr_key || (key == thr_key && (uint32_t)ps <= thr_pos));
+            }
+        }
+        int total;
+        const int rank = base + block_exclusive_scan(keep ? 1 : 0, warp_sums, total);
+        if (keep) order[rank] = j;
+        base += total;
+    }
+    const int n_keep = base;
+    __syncthreads();
+    // move: row order[r] -> slot r, r ascending; order[r] >= r, so a block's writes never reach a later source
+    constexpr int kVec = kRowBytes / 16;                     // 16-byte pieces per row and operand
+    constexpr int kRows = kSelThreads / kVec;                // rows per pass
+    uint8_t* ks = reinterpret_cast<uint8_t*>(p.k_slab) + w.slab0 * kRowBytes;
+    uint8_t* vs = reinterpret_cast<uint8_t*>(p.v_slab) + w.slab0 * kRowBytes;
+    int32_t* pos_w = p.pos + w.slab0;
+    for (int r0 = 0; r0 < n_keep; r0 += kRows) {
+        const int r = r0 + tid / kVec, c = tid % kVec;
+        const bool on = r < n_keep;
+        int src = 0, ps = 0;
+        float sc = 0.0f;
+        uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+        if (on) {
+            src = __ldcg(order + r);
+            if (src != r) {
+                kv = *(reinterpret_cast<const uint4*>(ks + (int64_t)src * kRowBytes) + c);
+                vv = *(reinterpret_cast<const uint4*>(vs + (int64_t)src * kRowBytes) + c);
+                if (c == 0) { ps = pos_w[src]; sc = score[src]; }
+            }
+        }
+        __syncthreads();
+        if (on && src != r) {
+            *(reinterpret_cast<uint4*>(ks + (int64_t)r * kRowBytes) + c) = kv;
+            *(reinterpret_cast<uint4*>(vs + (int64_t)r * kRowBytes) + c) = vv;
+            if (c == 0) { pos_w[r] = ps; score[r] = sc; }
+        }
+        __syncthreads();
+    }
+    if (tid == 0) { p.len[w.st] = n_keep; p.free_slot[w.st] = n_keep; }
+}
+
 }  // namespace
 
 extern "C" __attribute__((visibility("default"))) size_t baklava_evict_workspace_size(const baklava_shape* shape, int32_t B, int32_t layers, int32_t T) {
@@ -223,11 +390,14 @@ int evict_impl(const baklava_shape* shape, const baklava_cache* cache, int32_t l
                const void* k_dense, const void* v_dense, const float* score_dense, int32_t T, const int32_t* seq_len,
                int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve,
                int32_t* kept, void* stream) {
-    if (!k_dense || !v_dense) return BAKLAVA_ERR_UNSUPPORTED;   // in-place compaction of a slab
-    if (T <= 0 || reserve < 1 || stride_layer < 0 || stride_seq < 0 || stride_head < T) return BAKLAVA_ERR_INVALID_ARG;
+    const bool in_place = !k_dense && !v_dense;
+    if (!in_place && (!k_dense || !v_dense)) return BAKLAVA_ERR_INVALID_ARG;
+    if (in_place && (score_dense || seq_len)) return BAKLAVA_ERR_INVALID_ARG;   // the slab's own scores and lengths rule
+    if (T <= 0 || reserve < 1) return BAKLAVA_ERR_INVALID_ARG;
+    if (!in_place && (stride_layer < 0 || stride_seq < 0 || stride_head < T)) return BAKLAVA_ERR_INVALID_ARG;
     const void* ptrs[] = {k_dense, v_dense, cache->k_slab, cache->v_slab};
     for (const void* ptr : ptrs)
-        if (!baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
+        if (ptr && !baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
     const int64_t units = (int64_t)(layer_end - layer_begin) * cache->B * shape->Hkv;
     const int64_t row_blocks = ((int64_t)T + kCopyRows - 1) / kCopyRows;
     if (units > INT32_MAX || row_blocks > 65535) return BAKLAVA_ERR_UNSUPPORTED;
@@ -255,6 +425,12 @@ int evict_impl(const baklava_shape* shape, const baklava_cache* cache, int32_t l
     if (quantised && shape->D != 128) return BAKLAVA_ERR_UNSUPPORTED;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (in_place) {
+        if (quantised) evict_inplace_kernel<128><<<(unsigned)units, kSelThreads, 0, s>>>(p);
+        else if (shape->D == 128) evict_inplace_kernel<256><<<(unsigned)units, kSelThreads, 0, s>>>(p);
+        else evict_inplace_kernel<128><<<(unsigned)units, kSelThreads, 0, s>>>(p);
+        return cudaGetLastError() == cudaSuccess ? BAKLAVA_OK : BAKLAVA_ERR_CUDA;
+    }
     evict_select_kernel<<<(unsigned)units, kSelThreads, 0, s>>>(p);
     if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
     const dim3 grid((unsigned)units, (unsigned)row_blocks);
@@ -313,18 +489,20 @@ constexpr size_t kStaticKeptEntries = BAKLAVA_EVICT_STATIC_MAX_ENTRIES;   // 4 M
 static __device__ __align__(256) int32_t g_static_kept[kStaticKeptEntries];
 
 constexpr int kMaxDevices = 64;
-int32_t* g_static_kept_addr[kMaxDevices] = {};           // device address of the array, per device
+std::atomic<int32_t*> g_static_kept_addr[kMaxDevices];   // device address of the array, per device (zero-initialised)
 
 // The array's name is only a host-side handle; the kernels need its address on the current device.
 int static_kept_address(int32_t** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return BAKLAVA_ERR_CUDA;
-    if (!g_static_kept_addr[dev]) {
+    int32_t* known = g_static_kept_addr[dev].load(std::memory_order_acquire);
+    if (!known) {                                            // threads that race here all look up the same address
         void* addr = nullptr;
         if (cudaGetSymbolAddress(&addr, g_static_kept) != cudaSuccess || !addr) return BAKLAVA_ERR_CUDA;
-        g_static_kept_addr[dev] = static_cast<int32_t*>(addr);
+        known = static_cast<int32_t*>(addr);
+        g_static_kept_addr[dev].store(known, std::memory_order_release);
     }
-    *out = g_static_kept_addr[dev];
+    *out = known;
     return BAKLAVA_OK;
 }
 
@@ -336,7 +514,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_evict_static(
         int64_t stride_layer, int64_t stride_seq, int64_t stride_head, int32_t reserve, void* stream) {
     int rc = check_cache_and_layers(shape, cache, layer_begin, layer_end);
     if (rc) return rc;
-    if (!k_dense || !v_dense || T <= 0) return BAKLAVA_ERR_INVALID_ARG;
+    if (T <= 0) return BAKLAVA_ERR_INVALID_ARG;
     const int64_t units = (int64_t)(layer_end - layer_begin) * cache->B * shape->Hkv;
     if (units * (int64_t)T > (int64_t)kStaticKeptEntries) return BAKLAVA_ERR_WORKSPACE;   // beyond the fixed array
     int32_t* kept = nullptr;

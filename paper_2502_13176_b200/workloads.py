@@ -111,10 +111,14 @@ def kv_scales(w):
 
 
 def kv_fp8_scales(w, scales):
-    """Per-head FP8 scales (K, V) as float32 [L, Hkv, 2]: six standard deviations of the head's widest
-    channel map to the largest finite E4M3 value (448)."""
+    """Per-head FP8 scales as float32 [L, Hkv, 4] = (K scale, 1 / K scale, V scale, 1 / V scale), the layout the
+    library takes: six standard deviations of the head's widest channel map to the largest finite E4M3 value
+    (448); the reciprocals are float32 divisions, rounded once, and are inputs like the scales themselves."""
     widest = torch.stack([scales[0].amax(dim=2), scales[1].amax(dim=2)], dim=2)      # [L, Hkv, 2]
-    return (widest * (6.0 / 448.0)).to(torch.float32).numpy()
+    sc = (widest * (6.0 / 448.0)).to(torch.float32)
+    one = torch.ones((), dtype=torch.float32)
+    four = torch.stack([sc[..., 0], one / sc[..., 0], sc[..., 1], one / sc[..., 1]], dim=2)
+    return four.numpy()
 
 
 def dense_kv(w, l, b, h, scales, device="cpu", T=None):

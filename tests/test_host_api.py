@@ -140,6 +140,27 @@ def test_argument_errors_are_codes_not_crashes():
     assert L.baklava_evict(ctypes.byref(shape), None, 0, 1, None, None, None, 4, 0, 0, 4, 1, None, 0, None) == -1
 
 
+def test_misaligned_state_arrays_and_odd_strides_are_refused_on_the_host():
+    """pos and score are read in 16-byte vectors: a pointer or a sequence stride that breaks that must come
+    back as an argument error before anything touches the device (the addresses here are never dereferenced)."""
+    shape = bk.make_shape(2, 4, 2, 128)
+    info = bk.PlanInfo(4, 4, 4, 256, 0, 2, 1, 1 << 20)
+    base = 0x7f0000000000
+
+    def call(pos_off=0, score_off=0, stride=4096, flags=0):
+        c = bk.CacheStruct(base, base + (1 << 24), base + (2 << 24) + pos_off, base + (3 << 24) + score_off,
+                           base + (4 << 24), base + (5 << 24), base + (6 << 24), base + (7 << 24), stride, 1,
+                           base + (8 << 24), bk.KV_BF16, None)
+        return bk.lib().baklava_decode_attn(ctypes.byref(shape), ctypes.byref(c), base + (9 << 24), base + (10 << 24),
+                                            base + (11 << 24), 5, base + (12 << 24), None, flags, base + (13 << 24),
+                                            ctypes.byref(info), base + (14 << 24), 1 << 30, None)
+    assert call(pos_off=4) == -1
+    assert call(score_off=8) == -1
+    assert call(stride=4104) == -1
+    assert call(flags=1 << 20) == -1
+    assert bk.lib().baklava_set_wait_limit(-5) == -1
+
+
 def test_search_pick_matches_oracle_rule():
     from oracle import search as osearch
     rng = np.random.default_rng(9)

@@ -111,3 +111,35 @@ def test_bulk_evict_compacts_in_position_order():
     for m in sorted(set(range(T)) - set(idx), reverse=True):
         del rows[m]
     assert rows == list(idx)
+
+
+def test_compaction_in_place_is_eq_5_6_one_row_at_a_time():
+    """Rows in arbitrary (slot) order: taking the losers out one by one, each time closing the gap as
+    Eq. 5-6 print it, leaves the survivors in their original relative order; for rows already in
+    position order it coincides with bulk_evict."""
+    rng = np.random.default_rng(13)
+    for trial in range(20):
+        n, D = int(rng.integers(10, 60)), 4
+        R = int(rng.integers(7, n + 3))                                   # sometimes nothing has to go
+        K = rng.standard_normal((n, D)); V = rng.standard_normal((n, D))
+        pos = rng.permutation(n + 5)[:n]; score = np.round(rng.random(n), 1)
+        K2, V2, pos2, score2, idx = oe.compact_in_place(K, V, pos, score, R, 2, 1, 3)
+        keep = set(int(i) for i in oe.select_keep(pos, score, R, 2, 1, 3))
+        Kl, Vl, pl, sl = [list(x) for x in (K, V, pos, score)]
+        alive = list(range(n))
+        while True:
+            losers = [m for m, j in enumerate(alive) if j not in keep]
+            if not losers:
+                break
+            m = losers[0]                                                 # Eq. 5-6: [x_1..x_{m-1}, x_{m+1}..x_n]
+            for lst in (Kl, Vl, pl, sl, alive):
+                del lst[m]
+        assert alive == list(idx)
+        np.testing.assert_array_equal(np.array(Kl), K2); np.testing.assert_array_equal(np.array(Vl), V2)
+        np.testing.assert_array_equal(np.array(pl), pos2); np.testing.assert_array_equal(np.array(sl), score2)
+    T = 50
+    K = rng.standard_normal((T, 4)); V = rng.standard_normal((T, 4)); score = rng.random(T)
+    a = oe.compact_in_place(K, V, np.arange(T), score, 17, 4, 1, 2)
+    b = oe.bulk_evict(K, V, np.arange(T), score, 17, 4, 1, 2)
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)

@@ -36,8 +36,12 @@ def test_static_scratch_matches_workspace_version_twice():
             c.k_slab.zero_(); c.v_slab.zero_()
         ws = torch.empty((bk.baklava_evict_workspace_size(shape, B, L, T),), dtype=torch.uint8, device=dev)
         bk.baklava_evict(shape, ref, 0, L, k, v, sc, T, B * Hkv * T, Hkv * T, T, 1, ws)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         bk.baklava_evict_static(shape, got, 0, L, k, v, sc, T, B * Hkv * T, Hkv * T, T, 1)
         torch.cuda.synchronize()
+        if call > 0:                                     # after the first call's one-time set-up: the call itself
+            assert torch.cuda.mem_get_info()[0] == free_before   # takes no device memory and returns none
         assert int(got.status.item()) == 0 and int(ref.status.item()) == 0
         assert torch.equal(got.len, ref.len) and torch.equal(got.free_slot, ref.free_slot), "call %d" % call
         assert torch.equal(got.pos, ref.pos) and torch.equal(got.score, ref.score), "call %d" % call
