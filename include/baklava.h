@@ -72,6 +72,8 @@ extern "C" {
                                         /*   recent_den), where the oldest row outside both is evicted:  */
                                         /*   the paper's evaluated policy, with no score traffic at all  */
 #define BAKLAVA_FLAG_NO_EVICT      4u   /* never evict; a cache that fills up stays full              */
+#define BAKLAVA_FLAG_OVERLAP_PREV   8u   /* this call may start while the work in front of it on the   */
+                                        /*   stream is still finishing (see baklava_decode_attn)      */
 #define BAKLAVA_FLAG_TEST_STALL  256u   /* test aid, never set it in production: the first chunk of   */
                                         /*   every head is fed its first 64 (FP8: 128) rows only, so    */
                                         /*   that the bounded wait for the next ones runs out and the   */
@@ -149,8 +151,7 @@ typedef struct baklava_alloc_params {
 /* What baklava_decode_plan decided; passed back to baklava_decode_attn unchanged. */
 typedef struct baklava_plan_info {
     int32_t n_items;        /* attention work items (one chunk of one head of one sequence each)    */
-    int32_t n_score_items;  /* coarser pieces of the same heads for the score / eviction pass,      */
-                            /*   listed after the attention items                                   */
+    int32_t n_score_items;  /* always 0 (kept so that the structure's layout is stable)             */
     int32_t n_units;        /* (layer, sequence, KV head) triples in the layer range                */
     int32_t chunk_tokens;   /* target chunk length the plan used                                    */
     int32_t layer_begin, layer_end, B;
@@ -209,7 +210,7 @@ int baklava_allocate(const baklava_shape* shape, const double* kv_importance,
  *   chunk_tokens  target chunk length, 0 = choose from the total work and n_sm
  *   n_sm          streaming multiprocessors of the device (used when chunk_tokens = 0)
  *   items_out     host int32 [4 * items_capacity] or NULL to only fill `info`
- * The caller copies items_out ((info->n_items + info->n_score_items) * 16 bytes) to the device and hands it
+ * The caller copies items_out (info->n_items * 16 bytes) to the device and hands it
  * to baklava_decode_attn together with `info`. */
 int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t B,
                         int32_t layer_begin, int32_t layer_end, int32_t chunk_tokens, int32_t n_sm,
@@ -237,7 +238,24 @@ int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t 
  *            and not shared by steps that overlap in time; the library restores the
  *            parts that must be zero before it returns the stream to the caller, also
  *            after a step that set BAKLAVA_STATUS_TIMEOUT.
- * A head with no valid row gives out = 0 and lse = -inf. */
+ * A head with no valid row gives out = 0 and lse = -inf.
+ *
+ * Ordering on the stream.  A call is one kernel, launched with programmatic stream serialisation: its
+ * blocks may become resident while the work in front of it drains, and they wait for that work to
+ * complete before they read anything.  A model calls attention one layer at a time (Eq. 7 per layer),
+ * and a call for one layer is too short to fill the GPU: most of its time is the start-up and the tail
+ * (merge of the partial results, score update, eviction) of its few heads.  BAKLAVA_FLAG_OVERLAP_PREV
+ * lets a call start streaming its K / V rows at once, beside the tails of the calls in front of it.
+ * A run of calls is an unflagged call followed by flagged ones.  By setting the flag the caller vouches
+ * that nothing this call reads or writes (the cache state of its layer range, q, k_new, v_new, t_pos,
+ * items, out, lse, ws) is written, or has what this call writes read, by any earlier call of the same run
+ * or by anything else enqueued on the stream since the run's first call was enqueued: within a run the
+ * kernels may all be in flight at once.  The calls for the layers of one decode step qualify when each
+ * layer has its own workspace and all their inputs were written before the first of them was enqueued
+ * (the first one unflagged, the rest flagged); a call whose q comes out of the kernel just in front of
+ * it, or the next step of the same layers, does not.  An unflagged call, and any other work enqueued
+ * after a run, starts only when every call of the run has completed (no kernel of the library completes
+ * before the kernel in front of it). */
 int baklava_decode_attn(const baklava_shape* shape, const baklava_cache* cache,
                         const void* q, const void* k_new, const void* v_new, int32_t t_pos,
                         void* out, float* lse, uint32_t flags,

@@ -3,9 +3,9 @@
 //
 // One launch covers every (layer, sequence, KV head) of a layer range.  A head is cut into
 // chunks (the host plan); one CTA reduces one chunk to a partial (o, m, l) and leaves the
-// chunk's logits in the workspace.  The CTA that delivers the last partial of a head merges
-// them in chunk order, writes the output, turns the logits into probabilities with the final
-// normaliser, adds them to the scores and picks the row to evict in the same sweep.
+// chunk's unnormalised probabilities in the workspace.  The CTA that delivers the last partial of a
+// head finishes the head: it merges the partials in chunk order, writes the output, brings the
+// probabilities to the final normaliser, adds them to the scores and picks the row to evict.
 //
 // Inside a chunk: a producer warp streams 64-token K and V tiles with TMA (128-byte swizzle)
 // into a ring of shared-memory stages guarded by full/empty mbarriers; four consumer warps take
@@ -56,7 +56,7 @@ struct DecodeParams {
     const int64_t* slab_off;
     int64_t seq_stride;
     uint32_t* status;
-    int32_t B, L, Hq, Hkv, G, n_sink, recent_num, recent_den;
+    int32_t B, L, Hq, Hkv, G, D, n_sink, recent_num, recent_den;
     int32_t layer_begin, layers;
     const __nv_bfloat16* q;
     const __nv_bfloat16* k_new;
@@ -67,16 +67,11 @@ struct DecodeParams {
     const int32_t* t_pos_seq;      // per-sequence positions [B] (negative: the sequence sits this step out) or NULL
     uint32_t flags;
     int32_t window_evict;          // 1: no scores are kept and the policy is sinks + window: evict by position
-    const int4* items;             // attention items, then score items
+    const int4* items;             // the plan's work items
     int32_t n_items;
-    int32_t n_score_items;
-    int32_t* arrive;
-    int32_t* ready;                // [n_units]: 1 once a head's partials are merged and its statistics are final
+    int32_t* arrive;               // [n_units]: chunks of a head that have delivered their partial
     float* partial;
     float* logit;
-    float* stats;                  // [n_units][2 * kG]
-    unsigned long long* best_key;  // [n_score_items]
-    int32_t* best_slot;            // [n_score_items]
     float scale_log2;   // log2(e) / sqrt(D)
     const float* kv_scale;   // FP8 slabs: [L, Hkv, 4] (K scale, its reciprocal, V scale, its reciprocal)
     long long wait_cycles;   // SM clock cycles after which a wait on a tile gives up
@@ -129,6 +124,16 @@ __device__ __forceinline__ HeadState head_state(const DecodeParams& p, const Uni
 // grid_dependency_wait returns once the previous grid has completed and its writes are visible.
 __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// one arrival on a counter in global memory that also publishes this CTA's earlier writes and acquires the
+// other arrivers' (the thread calling it has been through a CTA barrier with the writers)
+__device__ __forceinline__ int arrive_acq_rel(int32_t* ptr) {
+    int before;
+    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(before) : "l"(ptr) : "memory");
+    return before;
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 __device__ __forceinline__ int ld_acquire(const int32_t* ptr) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
@@ -183,6 +188,291 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// ---------------------------------------------------------------- steps 3-4: scores and the row to evict
+// Run by the CTA that delivered a head's last partial, over the whole head.  Every row's stored probabilities
+// are brought to the head's final normaliser and added to its score; rows that may be evicted compete on the
+// 64-bit key (score bits, inverted position): the smallest key is the lowest score and, among equal scores,
+// the latest token.  Eight consecutive rows per thread and group (they share one 16-row block, hence one
+// reference maximum per query head), two groups in flight.  Each warp leaves its best candidate in shared
+// memory.
+template <int G>
+struct SweepGroup {
+    uint4 pr[G];
+    float fac[G];
+    float4 s0, s1;
+    int4 p0, p1;
+};
+
+template <int G>
+__device__ __forceinline__ void sweep_head(const float* logit_h, float* score, const int32_t* pos, int n_sink, int C,
+                                           int n_hi, int hole, bool evict, int newest_candidate, const float* sm_M,
+                                           const float* sm_invL, unsigned long long* sm_key, int* sm_slot) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const __half* prob_h = reinterpret_cast<const __half*>(logit_h);
+    const float* mref_h = reinterpret_cast<const float*>(prob_h + (int64_t)G * C);
+    float Mq[G], iL[G];
+#pragma unroll
+    for (int a = 0; a < G; ++a) { Mq[a] = sm_M[a]; iL[a] = sm_invL[a]; }
+    unsigned long long best = ~0ull;
+    int best_slot = -1;
+
+    auto load = [&](SweepGroup<G>& g, int j0) {              // a full group: rows j0 .. j0 + 7 all inside the head
+#pragma unroll
+        for (int a = 0; a < G; ++a) {
+            g.fac[a] = __ldcg(mref_h + a * (C >> 4) + (j0 >> 4));
+            g.pr[a] = __ldcg(reinterpret_cast<const uint4*>(prob_h + (int64_t)a * C + j0));
+        }
+        g.s0 = *reinterpret_cast<const float4*>(score + j0);
+        g.s1 = *reinterpret_cast<const float4*>(score + j0 + 4);
+        if (evict) {
+            g.p0 = *reinterpret_cast<const int4*>(pos + j0);
+            g.p1 = *reinterpret_cast<const int4*>(pos + j0 + 4);
+        }
+    };
+    auto finish = [&](SweepGroup<G>& g, int j0) {
+        float inc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) inc[e] = 0.0f;
+#pragma unroll
+        for (int a = 0; a < G; ++a) {
+            const float f = (g.fac[a] == -INFINITY) ? 0.0f : exp2f(g.fac[a] - Mq[a]) * iL[a];
+            const uint32_t w[4] = {g.pr[a].x, g.pr[a].y, g.pr[a].z, g.pr[a].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 pe = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
+                inc[2 * k] = fmaf(pe.x, f, inc[2 * k]);
+                inc[2 * k + 1] = fmaf(pe.y, f, inc[2 * k + 1]);
+            }
+        }
+        const float old[8] = {g.s0.x, g.s0.y, g.s0.z, g.s0.w, g.s1.x, g.s1.y, g.s1.z, g.s1.w};
+        float sc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sc[e] = (j0 + e == hole) ? old[e] : old[e] + inc[e];   // the freed slot is not a row
+        *reinterpret_cast<float4*>(score + j0) = make_float4(sc[0], sc[1], sc[2], sc[3]);
+        *reinterpret_cast<float4*>(score + j0 + 4) = make_float4(sc[4], sc[5], sc[6], sc[7]);
+        if (evict) {
+            const int ps[8] = {g.p0.x, g.p0.y, g.p0.z, g.p0.w, g.p1.x, g.p1.y, g.p1.z, g.p1.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                if (j0 + e != hole && ps[e] >= n_sink && ps[e] <= newest_candidate) {
+                    const unsigned long long key =
+                        ((unsigned long long)__float_as_uint(sc[e]) << 32) | (uint32_t)(~(uint32_t)ps[e]);
+                    if (key < best) { best = key; best_slot = j0 + e; }
+                }
+            }
+        }
+    };
+
+    constexpr int kStride = 8 * kThreads;
+    const int n_full = n_hi & ~7;                          // rows covered by full groups
+    int j0 = 8 * tid;
+    for (; j0 + kStride < n_full; j0 += 2 * kStride) {     // two full groups of this thread in flight
+        SweepGroup<G> g0, g1;
+        load(g0, j0);
+        load(g1, j0 + kStride);
+        finish(g0, j0);
+        finish(g1, j0 + kStride);
+    }
+    if (j0 < n_full) {
+        SweepGroup<G> g0;
+        load(g0, j0);
+        finish(g0, j0);
+    }
+    // the ragged end of the head: fewer than eight rows, one thread
+    if (tid == ((n_full >> 3) % kThreads) && n_full < n_hi) {
+        float f[G];
+#pragma unroll
+        for (int a = 0; a < G; ++a) {
+            const float mr = __ldcg(mref_h + a * (C >> 4) + (n_full >> 4));
+            f[a] = (mr == -INFINITY) ? 0.0f : exp2f(mr - Mq[a]) * iL[a];
+        }
+        for (int j = n_full; j < n_hi; ++j) {
+            if (j == hole) continue;
+            float inc = 0.0f;
+#pragma unroll
+            for (int a = 0; a < G; ++a) inc = fmaf(__half2float(__ldcg(prob_h + (int64_t)a * C + j)), f[a], inc);
+            const float sc = score[j] + inc;
+            score[j] = sc;
+            if (evict) {
+                const int ps = pos[j];
+                if (ps >= n_sink && ps <= newest_candidate) {
+                    const unsigned long long key = ((unsigned long long)__float_as_uint(sc) << 32) | (uint32_t)(~(uint32_t)ps);
+                    if (key < best) { best = key; best_slot = j; }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, off);
+        const int os = __shfl_xor_sync(0xffffffffu, best_slot, off);
+        if (ok < best) { best = ok; best_slot = os; }
+    }
+    if (lane == 0) { sm_key[warp] = best; sm_slot[warp] = best_slot; }
+}
+
+// ---------------------------------------------------------------- the end of a head
+// Run by the CTA that delivered a head's last partial: final (max, 1 / sum) of every query head, the merged
+// output (chunks in order: the result does not depend on which CTA comes last), then the score update over the
+// whole head, the row to evict and the bookkeeping.  Other heads' CTAs keep streaming meanwhile; the plan puts
+// the largest heads first, so the long tails fall into the middle of a launch.  Not inlined: its registers are
+// its own and do not weigh on the streaming loop.
+struct TailArgs {
+    const float* part0;            // the head's first partial
+    float* scratch;                // idle shared memory, 2 * max_merge_entries(D) floats
+    int32_t* arrive;               // the head's arrival counter
+    float* lse;                    // the group's entries of lse, or NULL
+    __nv_bfloat16* out;            // the group's rows of out
+    const float* logit_h;          // the head's probability scratch
+    float* score;                  // the head's rows of score / pos
+    const int32_t* pos;
+    int32_t* len;
+    int32_t* free_slot;
+    uint32_t* status;
+    int active, G, C, n, n_hi, hole, n_sink, newest_candidate;
+    bool keep_logits, do_append, may_evict, pos_evict, overlap;
+};
+
+template <int D, bool kByPosition>
+__device__ __noinline__ void finish_head(const TailArgs t) {
+    constexpr int kG = BAKLAVA_MAX_GROUP;
+    __shared__ float sm_M[kG];
+    __shared__ float sm_invL[kG];
+    __shared__ int sm_gave_up;
+    __shared__ unsigned long long sm_key[kThreads / 32];   // each warp's eviction candidate
+    __shared__ int sm_slot[kThreads / 32];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = t.G, active = t.active;
+    const int psz = partial_floats(G, D);
+    const float* part0 = t.part0;
+    // every chunk's (max, sum) into shared memory with one round of loads (the plan keeps chunks x group
+    // within max_merge_entries(D))
+    float* sm_mc = t.scratch;
+    float* sm_lc = sm_mc + max_merge_entries(D);
+    const int n_ml = active * G;
+    if (tid == 0) sm_gave_up = 0;
+    __syncthreads();
+    for (int i = tid; i < n_ml; i += kThreads) {
+        const int c = i / G, a = i - c * G;
+        const float* pc = part0 + (int64_t)c * psz + G * D;
+        const float mc = __ldcg(pc + a);
+        if (mc != mc) sm_gave_up = 1;                       // a chunk of this head ran out of time
+        sm_mc[i] = mc;
+        sm_lc[i] = __ldcg(pc + G + a);
+    }
+    __syncthreads();
+    if (sm_gave_up) {
+        // lost step: no output, no score update, no bookkeeping; the counter goes back to zero
+        if (tid == 0) {
+            *t.arrive = 0;
+            if (t.overlap) grid_dependency_wait();
+        }
+        return;
+    }
+    for (int a = warp; a < G; a += kThreads / 32) {         // one warp per query head, lanes over the chunks
+        float mm = -INFINITY;
+        for (int c = lane; c < active; c += 32) mm = fmaxf(mm, sm_mc[c * G + a]);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, off));
+        float ll = 0.0f;
+        for (int c = lane; c < active; c += 32) {
+            const float mc = sm_mc[c * G + a];
+            if (mc != -INFINITY) ll = fmaf(sm_lc[c * G + a], exp2f(mc - mm), ll);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) ll += __shfl_xor_sync(0xffffffffu, ll, off);
+        if (lane == 0) {
+            sm_M[a] = mm;
+            sm_invL[a] = ll > 0.0f ? 1.0f / ll : 0.0f;
+            if (t.lse) t.lse[a] = ll > 0.0f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < n_ml; i += kThreads) {            // each chunk's weight in the merged output
+        const int a = i % G;
+        const float mc = sm_mc[i];
+        sm_lc[i] = (mc == -INFINITY) ? 0.0f : exp2f(mc - sm_M[a]);
+    }
+    __syncthreads();
+    for (int grp = tid; grp < G * D / 4; grp += kThreads) { // four output elements per thread, chunks in order
+        const int a = (grp * 4) / D;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int c = 0;
+        for (; c + 8 <= active; c += 8) {                   // eight chunks' loads in flight
+            float4 oc[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                oc[k] = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)(c + k) * psz) + grp);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const float wgt = sm_lc[(c + k) * G + a];
+                acc.x = fmaf(oc[k].x, wgt, acc.x); acc.y = fmaf(oc[k].y, wgt, acc.y);
+                acc.z = fmaf(oc[k].z, wgt, acc.z); acc.w = fmaf(oc[k].w, wgt, acc.w);
+            }
+        }
+        for (; c < active; ++c) {
+            const float4 oc = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)c * psz) + grp);
+            const float wgt = sm_lc[c * G + a];
+            acc.x = fmaf(oc.x, wgt, acc.x); acc.y = fmaf(oc.y, wgt, acc.y);
+            acc.z = fmaf(oc.z, wgt, acc.z); acc.w = fmaf(oc.w, wgt, acc.w);
+        }
+        const float inv = sm_invL[a];
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        uint2 packed;
+        packed.x = *reinterpret_cast<const uint32_t*>(&lo);
+        packed.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(t.out + grp * 4) = packed;
+    }
+
+    // ---- steps 3-4
+    const bool evict = !kByPosition && t.keep_logits && t.may_evict;
+    if (!kByPosition && t.keep_logits) {
+        switch (G) {
+            case 1: sweep_head<1>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 2: sweep_head<2>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 3: sweep_head<3>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 4: sweep_head<4>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 5: sweep_head<5>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 6: sweep_head<6>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 7: sweep_head<7>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            default: sweep_head<8>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+        }
+    }
+    __syncthreads();                                        // output, scores and the warps' candidates are written
+    if (tid == 0) {
+        *t.arrive = 0;
+        if (t.do_append) {
+            int victim = -1;
+            bool wanted = false;                            // a row has to go
+            if (kByPosition && t.pos_evict) {
+                wanted = true;
+                int bp = INT32_MAX;
+                for (int c = 0; c < active; ++c) {
+                    const float* pc = part0 + (int64_t)c * psz + G * D + 2 * G;
+                    const int cp = __float_as_int(__ldcg(pc));
+                    if (cp < bp) { bp = cp; victim = __float_as_int(__ldcg(pc + 1)); }
+                }
+            } else if (evict) {
+                wanted = true;
+                unsigned long long bk = ~0ull;
+                for (int w = 0; w < kThreads / 32; ++w)
+                    if (sm_key[w] < bk) { bk = sm_key[w]; victim = sm_slot[w]; }
+            }
+            if (wanted && victim < 0) atomicOr(t.status, BAKLAVA_STATUS_BAD_STATE);   // nothing outside sinks + window
+            if (victim >= 0) {
+                *t.free_slot = victim;                      // len stays n: one row in, one row out (Eq. 5-6)
+            } else {
+                *t.len = t.n + 1;
+                *t.free_slot = t.n + 1;
+            }
+        }
+        // an overlapping call has not looked behind yet: a grid of this library never completes before the grid
+        // in front of it, which keeps "complete" transitive along the stream
+        if (t.overlap) grid_dependency_wait();
+    }
+}
+
 // ---------------------------------------------------------------- steps 2-4
 // kByPosition: the score-free sinks + window policy (a second instantiation, so that the default
 // path carries none of its registers or branches).
@@ -212,8 +502,6 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     __shared__ __align__(8) uint64_t bar_empty[kStages];
     __shared__ float sm_m[kConsumerWarps][kG];
     __shared__ float sm_l[kConsumerWarps][kG];
-    __shared__ float sm_M[kG];
-    __shared__ float sm_invL[kG];
     __shared__ int sm_last;
     __shared__ int sm_abort;
     __shared__ int sm_issued;
@@ -222,25 +510,44 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.G;
-    grid_dependency_wait();                               // len / free_slot / slab rows / items come from earlier kernels
+    // BAKLAVA_FLAG_OVERLAP_PREV: the caller vouches that nothing still in flight on the stream touches this call's
+    // data, so the chunk starts streaming at once and releases what follows at once.  The dependency wait is still
+    // made, at the very end, by the CTAs that finish a head (and by thread 0 of a CTA with nothing to do): a grid
+    // of this library never completes before the grid in front of it, so an unflagged call, whose CTAs all wait
+    // before they read anything, finds everything before it complete.
+    const bool overlap = (p.flags & BAKLAVA_FLAG_OVERLAP_PREV) != 0;
+    // what needs no memory of an earlier kernel comes first: the barriers and the tensor maps (kernel parameters)
+    if (tid == kConsumerWarps * 32) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), kConsumerWarps);
+        }
+        sm_abort = 0;
+        sm_issued = 0;
+        ptx::fence_mbar_init();
+        prefetch_tensormap(&k_map);
+        prefetch_tensormap(&v_map);
+    }
+    if (!overlap) grid_dependency_wait();                 // len / free_slot / slab rows / items come from earlier kernels
+    else launch_dependents();
     const int4 item = p.items[blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
     // Only now may the score kernel's CTAs become resident: they read len / free_slot before their own
     // dependency wait, and this order guarantees that the previous step's bookkeeping is complete by then
     // even when the whole grid is resident at once.
-    launch_dependents();
+    if (!overlap) launch_dependents();
     const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
-    if (t_pos < 0) return;                                // idle sequence: nothing of it is read or written
-    const HeadState hs = head_state(p, u);
-    if (hs.bad) {
-        if (tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
+    const HeadState hs = head_state(p, u);                // (its loads go out together with the one above)
+    const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
+    const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
+    // idle sequence (none of its rows, outputs or bookkeeping is touched), inconsistent head, chunk past the rows
+    if (t_pos < 0 || hs.bad || piece >= active) {
+        if (t_pos >= 0 && hs.bad && tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
+        if (overlap && tid == 0) grid_dependency_wait();
         return;
     }
     if (hs.overflow && tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_OVERFLOW);
-    const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
-    const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
-    if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
     const int n_tiles = end > begin ? (end - begin + kTT - 1) / kTT : 0;
     const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
@@ -260,16 +567,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
 
-    if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), kConsumerWarps);
-        }
-        sm_abort = 0;
-        sm_issued = 0;
-        ptx::fence_mbar_init();
-    }
-    __syncthreads();
+    __syncthreads();                                      // the barriers are initialised
 
     // per-warp online-softmax state; row q of the group lives in the quad of lanes with lane / 4 == q
     const int qrow = lane >> 2, qcol = (lane & 3) * 2;
@@ -732,303 +1030,32 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         part[G * D + 2 * G + 1] = __int_as_float(bs);
     }
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int before = atomicAdd(p.arrive + unit, 1);
-        sm_last = (before == active - 1);
-    }
+    __syncthreads();                                        // the whole partial is written ...
+    if (tid == 0) sm_last = (arrive_acq_rel(p.arrive + unit) == active - 1);   // ... and published with the arrival
     __syncthreads();
     if (!sm_last) return;
-    __threadfence();
 
-    // ---- this CTA delivered the head's last partial: merge them in chunk order, write the output
-    // and leave the final (max, 1 / sum) of every query head for the score kernel
-    const float* part0 = p.partial + (int64_t)(blockIdx.x - piece) * psz;
-    // every chunk's (max, sum) into shared memory with one round of loads (the ring is idle now; the plan
-    // keeps chunks x group within max_merge_entries(D))
-    float* sm_mc = reinterpret_cast<float*>(ring_ptr);
-    float* sm_lc = sm_mc + max_merge_entries(D);
-    const int n_ml = active * G;
-    for (int i = tid; i < n_ml; i += kThreads) {
-        const int c = i / G, a = i - c * G;
-        const float* pc = part0 + (int64_t)c * psz + G * D;
-        const float mc = __ldcg(pc + a);
-        if (mc != mc) sm_abort = 1;                         // a chunk of this head gave up
-        sm_mc[i] = mc;
-        sm_lc[i] = __ldcg(pc + G + a);
-    }
-    __syncthreads();
-    if (sm_abort) {
-        // lost step: no output, no bookkeeping; the counters go back to zero and the score pieces are told
-        if (tid == 0) {
-            p.stats[(int64_t)unit * 2 * kG] = __int_as_float(0x7fc00000);
-            p.arrive[unit] = 0;
-            if (keep_logits) st_release(p.ready + unit, 1);
-        }
-        return;
-    }
-    if (tid < G) {
-        float mm = -INFINITY;
-        for (int c = 0; c < active; ++c) mm = fmaxf(mm, sm_mc[c * G + tid]);
-        float ll = 0.0f;
-        for (int c = 0; c < active; ++c) {
-            const float mc = sm_mc[c * G + tid];
-            if (mc != -INFINITY) ll = fmaf(sm_lc[c * G + tid], exp2f(mc - mm), ll);
-        }
-        const float inv = ll > 0.0f ? 1.0f / ll : 0.0f;
-        sm_M[tid] = mm;
-        sm_invL[tid] = inv;
-        p.stats[(int64_t)unit * 2 * kG + tid] = mm;
-        p.stats[(int64_t)unit * 2 * kG + kG + tid] = inv;
-        if (p.lse)
-            p.lse[(int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + tid] = ll > 0.0f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
-    }
-    __syncthreads();
-    for (int i = tid; i < n_ml; i += kThreads) {            // each chunk's weight in the merged output
-        const int a = i % G;
-        const float mc = sm_mc[i];
-        sm_lc[i] = (mc == -INFINITY) ? 0.0f : exp2f(mc - sm_M[a]);
-    }
-    __syncthreads();
-    __nv_bfloat16* orow = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
-    for (int grp = tid; grp < G * D / 4; grp += kThreads) { // four output elements per thread, chunks in order
-        const int a = (grp * 4) / D;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        int c = 0;
-        for (; c + 8 <= active; c += 8) {                   // eight chunks' loads in flight
-            float4 oc[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-                oc[k] = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)(c + k) * psz) + grp);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const float wgt = sm_lc[(c + k) * G + a];
-                acc.x = fmaf(oc[k].x, wgt, acc.x); acc.y = fmaf(oc[k].y, wgt, acc.y);
-                acc.z = fmaf(oc[k].z, wgt, acc.z); acc.w = fmaf(oc[k].w, wgt, acc.w);
-            }
-        }
-        for (; c < active; ++c) {
-            const float4 oc = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)c * psz) + grp);
-            const float wgt = sm_lc[c * G + a];
-            acc.x = fmaf(oc.x, wgt, acc.x); acc.y = fmaf(oc.y, wgt, acc.y);
-            acc.z = fmaf(oc.z, wgt, acc.z); acc.w = fmaf(oc.w, wgt, acc.w);
-        }
-        const float inv = sm_invL[a];
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-        const __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-        uint2 packed;
-        packed.x = *reinterpret_cast<const uint32_t*>(&lo);
-        packed.y = *reinterpret_cast<const uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(orow + grp * 4) = packed;
-    }
-    __syncthreads();                                        // every thread's share of the output is written
-    if (tid == 0) {
-        p.arrive[unit] = 0;                                 // the score kernel counts arrivals again
-        // the head is final: its score pieces may start although other heads are still being attended
-        if (keep_logits) st_release(p.ready + unit, 1);
-        if (!keep_logits && hs.do_append) {                 // no score pass follows: finish the bookkeeping here
-            int victim = -1;
-            if (kByPosition && pos_evict) {
-                int bp = INT32_MAX;
-                for (int c = 0; c < active; ++c) {
-                    const float* pc = part0 + (int64_t)c * psz + G * D + 2 * G;
-                    const int cp = __float_as_int(__ldcg(pc));
-                    if (cp < bp) { bp = cp; victim = __float_as_int(__ldcg(pc + 1)); }
-                }
-                if (victim < 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);   // nothing outside sinks + window
-            }
-            if (victim >= 0) {
-                p.free_slot[u.st] = victim;                 // len stays n: one row in, one row out (Eq. 5-6)
-            } else {
-                p.len[u.st] = n + 1;
-                p.free_slot[u.st] = n + 1;
-            }
-        }
-    }
-}
-
-// ---------------------------------------------------------------- steps 3-4: scores and eviction
-// One CTA per chunk again.  Every row's logits become probabilities with the head's final
-// normaliser and are added to its score; rows that may be evicted compete on the 64-bit key
-// (score bits, inverted position): the smallest key is the lowest score and, among equal scores,
-// the latest token.  The CTA that finishes a head last picks the head's victim among the chunks'
-// candidates and updates len / free_slot.
-constexpr int kScoreThreads = 128;                       // eight rows per thread and sweep
-constexpr int kReadyPolls = 1 << 14;                     // polls of a head's ready flag before falling back
-
-template <int G>
-__global__ void __launch_bounds__(kScoreThreads, 8) score_evict_kernel(const DecodeParams p) {
-    constexpr int kG = BAKLAVA_MAX_GROUP;
-    __shared__ unsigned long long sm_key[kScoreThreads / 32];
-    __shared__ int sm_slot[kScoreThreads / 32];
-    __shared__ int sm_last;
-    __shared__ int sm_ready;
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int4 item = p.items[p.n_items + blockIdx.x];
-    const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
-    const Unit u = decode_unit(p, unit);
-    launch_dependents();
-    // len and free_slot are not touched by the attention kernel when a score pass follows (this kernel does
-    // the bookkeeping), so the head's state can be read while that kernel is still draining
-    const HeadState hs = head_state(p, u);
-    const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
-    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
-    if (hs.bad || t_pos < 0) return;                       // reported by the attention kernel / idle sequence
-    const int C = hs.C, n = hs.n, hole = hs.hole, n_hi = hs.n_att;
-    const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
-    if (piece >= active) return;
-    const int end = min(begin + chunk_len, n_hi);
-    // This kernel's CTAs become resident while the last attention CTAs are still running.  A piece needs
-    // only its own head: it watches the head's ready flag (set with release semantics by the CTA that merged
-    // the head) instead of waiting for the whole attention grid.  The watch is bounded; if it runs out, the
-    // grid-wide dependency wait below is always sufficient.
-    if (tid == 0) {
-        int ok = 0;
-        for (int i = 0; i < kReadyPolls && !ok; ++i) {
-            ok = ld_acquire(p.ready + unit) != 0;
-            if (!ok) __nanosleep(64);
-        }
-        sm_ready = ok;
-    }
-    __syncthreads();
-    if (!sm_ready) grid_dependency_wait();                // the attention kernel's scratch and statistics
-
-    const __half* prob_h = reinterpret_cast<const __half*>(p.logit + row0 * G);
-    const float* mref_h = reinterpret_cast<const float*>(prob_h + (int64_t)G * C);
-    float Mq[G], iL[G];
-#pragma unroll
-    for (int a = 0; a < G; ++a) {
-        Mq[a] = p.stats[(int64_t)unit * 2 * kG + a];
-        iL[a] = p.stats[(int64_t)unit * 2 * kG + kG + a];
-    }
-    const bool lost = Mq[0] != Mq[0];                      // the attention kernel gave the head's step up
-    const bool appended = hs.do_append && !lost;
-    const int R = C - 1;
-    const bool evict = appended && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n_hi > R;
-    const int W = max(0, (int)(((int64_t)(R - p.n_sink) * p.recent_num) / p.recent_den));
-    const int newest_candidate = t_pos - W;              // rows with pos > this are in the recent window
-
-    unsigned long long best = ~0ull;
-    int best_slot = -1;
-    // eight consecutive rows per thread: they share one 16-row block, hence one reference maximum per head
-    for (int j0 = begin + 8 * tid; j0 < (lost ? begin : end); j0 += 8 * kScoreThreads) {
-        float fac[G];
-#pragma unroll
-        for (int a = 0; a < G; ++a) {
-            const float mr = __ldcg(mref_h + a * (C >> 4) + (j0 >> 4));
-            fac[a] = (mr == -INFINITY) ? 0.0f : exp2f(mr - Mq[a]) * iL[a];
-        }
-        float inc[8], sc[8];
-        int ps[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) { inc[e] = 0.0f; ps[e] = 0; }
-        if (j0 + 8 <= end) {
-            uint4 pr[G];
-#pragma unroll
-            for (int a = 0; a < G; ++a)
-                pr[a] = __ldcg(reinterpret_cast<const uint4*>(prob_h + (int64_t)a * C + j0));
-            const float4 s0 = *reinterpret_cast<const float4*>(p.score + row0 + j0);
-            const float4 s1 = *reinterpret_cast<const float4*>(p.score + row0 + j0 + 4);
-            if (evict) {
-                const int4 p0 = *reinterpret_cast<const int4*>(p.pos + row0 + j0);
-                const int4 p1 = *reinterpret_cast<const int4*>(p.pos + row0 + j0 + 4);
-                ps[0] = p0.x; ps[1] = p0.y; ps[2] = p0.z; ps[3] = p0.w;
-                ps[4] = p1.x; ps[5] = p1.y; ps[6] = p1.z; ps[7] = p1.w;
-            }
-#pragma unroll
-            for (int a = 0; a < G; ++a) {
-                const uint32_t w[4] = {pr[a].x, pr[a].y, pr[a].z, pr[a].w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float2 pe = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
-                    inc[2 * k] = fmaf(pe.x, fac[a], inc[2 * k]);
-                    inc[2 * k + 1] = fmaf(pe.y, fac[a], inc[2 * k + 1]);
-                }
-            }
-            const float old[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-#pragma unroll
-            for (int e = 0; e < 8; ++e) sc[e] = (j0 + e == hole) ? old[e] : old[e] + inc[e];   // the freed slot is not a row
-            *reinterpret_cast<float4*>(p.score + row0 + j0) = make_float4(sc[0], sc[1], sc[2], sc[3]);
-            *reinterpret_cast<float4*>(p.score + row0 + j0 + 4) = make_float4(sc[4], sc[5], sc[6], sc[7]);
-        } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int j = j0 + e;
-                sc[e] = 0.0f;
-                if (j < end && j != hole) {
-#pragma unroll
-                    for (int a = 0; a < G; ++a)
-                        inc[e] = fmaf(__half2float(__ldcg(prob_h + (int64_t)a * C + j)), fac[a], inc[e]);
-                    sc[e] = p.score[row0 + j] + inc[e];
-                    p.score[row0 + j] = sc[e];
-                    if (evict) ps[e] = p.pos[row0 + j];
-                }
-            }
-        }
-        if (evict) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int j = j0 + e;
-                if (j < end && j != hole && ps[e] >= p.n_sink && ps[e] <= newest_candidate) {
-                    const unsigned long long key =
-                        ((unsigned long long)__float_as_uint(sc[e]) << 32) | (uint32_t)(~(uint32_t)ps[e]);
-                    if (key < best) { best = key; best_slot = j; }
-                }
-            }
-        }
-    }
-    if (evict) {
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, off);
-            const int os = __shfl_xor_sync(0xffffffffu, best_slot, off);
-            if (ok < best) { best = ok; best_slot = os; }
-        }
-        if (lane == 0) { sm_key[warp] = best; sm_slot[warp] = best_slot; }
-        __syncthreads();
-        if (tid == 0) {
-            for (int w = 0; w < kScoreThreads / 32; ++w)
-                if (sm_key[w] < best) { best = sm_key[w]; best_slot = sm_slot[w]; }
-            p.best_key[blockIdx.x] = best;
-            p.best_slot[blockIdx.x] = best_slot;
-        }
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const int before = atomicAdd(p.arrive + unit, 1);
-        sm_last = (before == active - 1);
-    }
-    __syncthreads();
-    if (!sm_last) return;
-    __threadfence();
-    if (tid == 0) {
-        if (appended) {
-            if (evict) {
-                const int64_t first = (int64_t)blockIdx.x - piece;
-                unsigned long long bk = ~0ull;
-                int bs = -1;
-                for (int c = 0; c < active; ++c) {
-                    const unsigned long long kc = __ldcg(p.best_key + first + c);
-                    if (kc < bk) { bk = kc; bs = __ldcg(p.best_slot + first + c); }
-                }
-                if (bs >= 0) {
-                    p.free_slot[u.st] = bs;                 // len stays n: one row in, one row out
-                } else {
-                    atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);   // capacity too small for sinks + window
-                    p.len[u.st] = n + 1;
-                    p.free_slot[u.st] = n + 1;
-                }
-            } else {
-                p.len[u.st] = n + 1;
-                p.free_slot[u.st] = n + 1;
-            }
-        }
-        p.arrive[unit] = 0;
-        p.ready[unit] = 0;                                  // every piece of the head is past its watch
-    }
+    // ---- this CTA delivered the head's last partial and finishes the head
+    TailArgs t;
+    t.part0 = p.partial + (int64_t)(blockIdx.x - piece) * psz;
+    t.scratch = reinterpret_cast<float*>(ring_ptr);         // the ring is idle now
+    t.arrive = p.arrive + unit;
+    t.lse = p.lse ? p.lse + (int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G : nullptr;
+    t.out = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
+    t.logit_h = p.logit + row0 * G;
+    t.score = p.score + row0;
+    t.pos = p.pos + row0;
+    t.len = p.len + u.st;
+    t.free_slot = p.free_slot + u.st;
+    t.status = p.status;
+    t.active = active; t.G = G; t.C = C; t.n = n; t.n_hi = n_hi; t.hole = hole; t.n_sink = p.n_sink;
+    t.newest_candidate = window_from;                       // rows with a later position are in the recent window
+    t.keep_logits = keep_logits;
+    t.do_append = hs.do_append;
+    t.may_evict = hs.do_append && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n_hi > C - 1;
+    t.pos_evict = pos_evict;
+    t.overlap = overlap;
+    finish_head<D, kByPosition>(t);
 }
 
 // ---------------------------------------------------------------- host side
@@ -1107,7 +1134,8 @@ int decode_attn_impl(
     int rc = baklava_check_shape(shape);
     if (rc) return rc;
     if (!cache || !q || !out || !items || !info || !ws) return BAKLAVA_ERR_INVALID_ARG;
-    if (flags & ~(BAKLAVA_FLAG_NO_APPEND | BAKLAVA_FLAG_NO_SCORE | BAKLAVA_FLAG_NO_EVICT | BAKLAVA_FLAG_TEST_STALL))
+    if (flags & ~(BAKLAVA_FLAG_NO_APPEND | BAKLAVA_FLAG_NO_SCORE | BAKLAVA_FLAG_NO_EVICT | BAKLAVA_FLAG_OVERLAP_PREV |
+                  BAKLAVA_FLAG_TEST_STALL))
         return BAKLAVA_ERR_INVALID_ARG;
     const bool no_append = flags & BAKLAVA_FLAG_NO_APPEND;
     if (!no_append && (!k_new || !v_new)) return BAKLAVA_ERR_INVALID_ARG;
@@ -1119,13 +1147,13 @@ int decode_attn_impl(
         if (ptr && !baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
     if (cache->seq_stride_tokens % 16 != 0) return BAKLAVA_ERR_INVALID_ARG;   // rows of pos / score go in 16-byte vectors
     if (info->layer_begin < 0 || info->layer_end > shape->L || info->layer_begin >= info->layer_end ||
-        info->B != cache->B || info->n_items <= 0 || info->n_score_items <= 0 ||
+        info->B != cache->B || info->n_items <= 0 || info->n_score_items != 0 ||
         info->n_units != (info->layer_end - info->layer_begin) * cache->B * shape->Hkv)
         return BAKLAVA_ERR_INVALID_ARG;
     const int64_t rows = (int64_t)cache->B * cache->seq_stride_tokens;
     if (rows > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     DecodeWorkspace lay;
-    const size_t need = baklava_decode_ws_bytes(shape, info->n_items, info->n_score_items, info->n_units, cache->B,
+    const size_t need = baklava_decode_ws_bytes(shape, info->n_items, info->n_units, cache->B,
                                                 cache->seq_stride_tokens, &lay);
     if (ws_bytes < need) return BAKLAVA_ERR_WORKSPACE;
 
@@ -1154,6 +1182,7 @@ int decode_attn_impl(
     p.status = cache->status;
     p.B = cache->B;
     p.L = shape->L; p.Hq = shape->Hq; p.Hkv = shape->Hkv; p.G = shape->Hq / shape->Hkv;
+    p.D = shape->D;
     p.n_sink = shape->n_sink; p.recent_num = shape->recent_num; p.recent_den = shape->recent_den;
     p.layer_begin = info->layer_begin;
     p.layers = info->layer_end - info->layer_begin;
@@ -1170,15 +1199,10 @@ int decode_attn_impl(
     p.flags = ((flags & BAKLAVA_FLAG_NO_SCORE) && !p.window_evict) ? (flags | BAKLAVA_FLAG_NO_EVICT) : flags;
     p.items = reinterpret_cast<const int4*>(items);
     p.n_items = info->n_items;
-    p.n_score_items = info->n_score_items;
     char* base = static_cast<char*>(ws);
     p.arrive = reinterpret_cast<int32_t*>(base + lay.arrive_off);
-    p.ready = p.arrive + info->n_units;
     p.partial = reinterpret_cast<float*>(base + lay.partial_off);
     p.logit = reinterpret_cast<float*>(base + lay.logit_off);
-    p.stats = reinterpret_cast<float*>(base + lay.stats_off);
-    p.best_key = reinterpret_cast<unsigned long long*>(base + lay.best_off);
-    p.best_slot = reinterpret_cast<int32_t*>(base + lay.best_off + 8 * (size_t)info->n_score_items);
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
     p.kv_scale = cache->kv_scale;
     p.wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
@@ -1189,30 +1213,7 @@ int decode_attn_impl(
     else if (p.window_evict) err = shape->D == 128 ? launch_chunks<128, true>(p, k_map, v_map, s) : launch_chunks<64, true>(p, k_map, v_map, s);
     else err = shape->D == 128 ? launch_chunks<128, false>(p, k_map, v_map, s) : launch_chunks<64, false>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
-    if (!(p.flags & BAKLAVA_FLAG_NO_SCORE)) {
-        void (*score_fn)(const DecodeParams) = nullptr;
-        switch (p.G) {
-            case 1: score_fn = score_evict_kernel<1>; break;
-            case 2: score_fn = score_evict_kernel<2>; break;
-            case 3: score_fn = score_evict_kernel<3>; break;
-            case 4: score_fn = score_evict_kernel<4>; break;
-            case 5: score_fn = score_evict_kernel<5>; break;
-            case 6: score_fn = score_evict_kernel<6>; break;
-            case 7: score_fn = score_evict_kernel<7>; break;
-            default: score_fn = score_evict_kernel<8>; break;
-        }
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)p.n_score_items);
-        cfg.blockDim = dim3(kScoreThreads);
-        cfg.stream = s;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, score_fn, p) != cudaSuccess) return BAKLAVA_ERR_CUDA;
-        if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
-    }
+    if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
     return BAKLAVA_OK;
 }
 }  // namespace

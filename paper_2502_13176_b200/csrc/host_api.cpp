@@ -160,16 +160,14 @@ extern "C" __attribute__((visibility("default"))) int baklava_allocate(const bak
 }
 
 // ---------------------------------------------------------------- decode work plan
-size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_score_items, int64_t n_units, int32_t B,
+size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_units, int32_t B,
                                int64_t seq_stride_tokens, DecodeWorkspace* lay) {
     const int g = s->Hq / s->Hkv;
     DecodeWorkspace w;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 255) / 256 * 256; return at; };
     w.control_off = take(sizeof(int32_t) * 64);
-    w.arrive_off = take(sizeof(int32_t) * 2 * (size_t)n_units);
-    w.stats_off = take(sizeof(float) * (size_t)n_units * 2 * BAKLAVA_MAX_GROUP);
-    w.best_off = take(16 * (size_t)n_score_items);
+    w.arrive_off = take(sizeof(int32_t) * (size_t)n_units);
     w.partial_off = take(sizeof(float) * (size_t)n_items * partial_floats(g, s->D));
     w.logit_off = take(sizeof(float) * (size_t)B * (size_t)seq_stride_tokens * g);
     w.total = off;
@@ -204,12 +202,27 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
     // Chunk length.  A fixed request is used as given.  Otherwise the launch is self-balancing: CTAs are
     // dispatched in item order, so the list starts with long chunks (about half of a CTA slot's share of
     // the tokens: little per-chunk overhead) and ends with short ones (a short tail).
-    const bool guided = chunk_tokens == 0;
+    bool guided = chunk_tokens == 0;
     int64_t target = chunk_tokens;
     if (guided) {
         const int64_t slots = (int64_t)n_sm * kCtasPerSm;
         target = (tokens / (2 * slots) + kTile - 1) / kTile * kTile;
         target = std::max<int64_t>(kMinChunk, std::min<int64_t>(target, 4096));
+        if (target == kMinChunk) {
+            // A short launch (one layer of a model): nothing balances a second, partly filled wave, so all chunks
+            // get the same length, the shortest (from the minimum up) with which every chunk is resident at once.
+            guided = false;
+            for (; target < 4096; target += kTile) {
+                int64_t count = 0;
+                for (int i : heads) {
+                    const int64_t c = cap[(size_t)layer_begin * Hkv + i];
+                    const int64_t pieces = (c + target - 1) / target;
+                    const int64_t len = ((c + pieces - 1) / pieces + kTile - 1) / kTile * kTile;
+                    count += (c + len - 1) / len * B;
+                }
+                if (count <= slots) break;
+            }
+        }
     }
     target = std::max<int64_t>(kTile, (target + kTile - 1) / kTile * kTile);
 
@@ -248,21 +261,18 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
         }
         return BAKLAVA_OK;
     };
-    int64_t n_items = 0, n_score = 0;
-    rc = emit(target, guided, &n_items);         // attention chunks
+    int64_t n_items = 0;
+    rc = emit(target, guided, &n_items);
     if (rc) return rc;
-    rc = emit(kScoreChunk, false, &n_score);     // coarser pieces for the score / eviction pass
-    if (rc) return rc;
-    if (n_score > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     if (n_items > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     info->n_items = (int32_t)n_items;
-    info->n_score_items = (int32_t)n_score;
+    info->n_score_items = 0;
     info->n_units = layers * B * Hkv;
     info->chunk_tokens = (int32_t)target;
     info->layer_begin = layer_begin;
     info->layer_end = layer_end;
     info->B = B;
-    info->ws_bytes = (int64_t)baklava_decode_ws_bytes(shape, n_items, n_score, info->n_units, B, seq_stride_tokens, nullptr);
+    info->ws_bytes = (int64_t)baklava_decode_ws_bytes(shape, n_items, info->n_units, B, seq_stride_tokens, nullptr);
     return BAKLAVA_OK;
 }
 

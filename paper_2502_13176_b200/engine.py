@@ -78,12 +78,16 @@ class DecodeSession:
             plan = bk.baklava_decode_plan(self.shape, self.cap, self.w.B, l, l + 1, self.stride, n_sm=n_sm).to(self.device)
             self.layer_plans.append((plan, bk.decode_workspace(plan, self.device)))
 
-    def step_layers(self, q, k_new, v_new, t_pos, flags=0):
+    def step_layers(self, q, k_new, v_new, t_pos, flags=0, overlap=True):
         """One decode step as one call per layer; t_pos: device int32 [B] (so that the sequence of calls can be
-        captured in a CUDA graph and replayed with the positions advanced on the device)."""
+        captured in a CUDA graph and replayed with the positions advanced on the device).  q / k_new / v_new of
+        every layer must be complete before the first call is enqueued when `overlap` is set."""
         for i, (plan, ws) in enumerate(self.layer_plans):
+            # every layer has its own heads, inputs and workspace, and all inputs are complete before the first
+            # call: from the second layer on a call may start beside the previous layer's tail
+            fl = flags | (bk.FLAG_OVERLAP_PREV if overlap and i > 0 else 0)
             bk.baklava_decode_attn_varlen(self.shape, self.cache, q[i:i + 1], k_new[i:i + 1], v_new[i:i + 1], t_pos,
-                                          self.out[i:i + 1], self.lse[i:i + 1], flags, plan, ws)
+                                          self.out[i:i + 1], self.lse[i:i + 1], fl, plan, ws)
         return self.out
 
     def retained_kv_bytes(self):

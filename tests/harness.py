@@ -39,7 +39,9 @@ class Session:
     """One workload on the device (library) with oracle twins for the heads in `heads`."""
 
     def __init__(self, w, heads=None, chunk_tokens=0, layers=None, prefill=True, device="cuda", caps=None,
-                 kv_dtype=bk.KV_BF16):
+                 kv_dtype=bk.KV_BF16, per_layer=False):
+        """`per_layer`: every step is issued as one call per layer, each with its own plan and workspace and, from
+        the second layer on, BAKLAVA_FLAG_OVERLAP_PREV (the form a model's layer loop uses)."""
         self.w, self.device = w, device
         self.kv_dtype = kv_dtype
         self.shape = shape_of(w)
@@ -67,6 +69,13 @@ class Session:
                                            chunk_tokens=chunk_tokens,
                                            n_sm=torch.cuda.get_device_properties(0).multi_processor_count).to(device)
         self.ws = bk.decode_workspace(self.plan, device)
+        self.layer_plans = None
+        if per_layer:
+            self.layer_plans = []
+            for l in range(self.lb, self.le):
+                plan = bk.baklava_decode_plan(self.shape, self.cap, w.B, l, l + 1, self.stride, chunk_tokens=chunk_tokens,
+                                              n_sm=torch.cuda.get_device_properties(0).multi_processor_count).to(device)
+                self.layer_plans.append((plan, bk.decode_workspace(plan, device)))
         nl = self.le - self.lb
         self.out = torch.zeros((nl, w.B, w.Hq, w.D), dtype=torch.bfloat16, device=device)
         self.lse = torch.zeros((nl, w.B, w.Hq), dtype=torch.float32, device=device)
@@ -160,7 +169,14 @@ class Session:
         w = self.w
         q, kn, vn = wl.decode_inputs(w, step_index, self.scales, self.device, layers=(self.lb, self.le))
         t_pos = self.t
-        bk.baklava_decode_attn(self.shape, self.cache, q, kn, vn, t_pos, self.out, self.lse, flags, self.plan, self.ws)
+        if self.layer_plans is None:
+            bk.baklava_decode_attn(self.shape, self.cache, q, kn, vn, t_pos, self.out, self.lse, flags, self.plan, self.ws)
+        else:
+            torch.cuda.synchronize()                        # the inputs of every layer are complete before the first call
+            for i, (plan, ws) in enumerate(self.layer_plans):
+                bk.baklava_decode_attn(self.shape, self.cache, q[i:i + 1], kn[i:i + 1], vn[i:i + 1], t_pos,
+                                       self.out[i:i + 1], self.lse[i:i + 1],
+                                       flags | (bk.FLAG_OVERLAP_PREV if i > 0 else 0), plan, ws)
         torch.cuda.synchronize()
         if not (flags & bk.FLAG_NO_APPEND):
             self.t += 1

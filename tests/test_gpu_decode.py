@@ -48,6 +48,35 @@ def test_layer_range_launch():
     assert int(s.cache.len[0, 0].sum()) == 0                         # layer 0 was never touched
 
 
+@pytest.mark.parametrize("chunk", [64, 0])
+def test_one_call_per_layer_overlapping_the_previous_layers_tail(chunk):
+    """The layer loop of a model: one call per layer with its own plan and workspace, every call after the first
+    flagged as independent of the one before it.  Same results as the oracle, step after step."""
+    w = wl.scaled(wl.LLAMA3_8B_32K, L=5, T=2000, steps=6)
+    s = Session(w, chunk_tokens=chunk, per_layer=True)
+    for i in range(w.steps):
+        s.step(i)
+    w = wl.scaled(wl.QWEN25_7B_8K_B16, L=3, B=3, T=1500, steps=4)
+    s = Session(w, chunk_tokens=chunk, per_layer=True)
+    for i in range(w.steps):
+        s.step(i)
+
+
+def test_one_call_per_layer_leaves_the_same_cache_as_one_call_for_all_layers():
+    # same chunks either way, so scores, victims and rows agree bit for bit; the outputs are summed over the chunks
+    # in an order that depends on how the launch is cut into score pieces, so they may differ in the last place
+    w = wl.scaled(wl.LLAMA3_8B_32K, L=4, T=3000, steps=3)
+    outs = []
+    for per_layer in (False, True):
+        s = Session(w, heads=[], chunk_tokens=128, per_layer=per_layer)
+        for i in range(w.steps):
+            s.step(i, check=False)
+        outs.append((s.cache.score.clone(), s.cache.free_slot.clone(), s.cache.pos.clone(), s.cache.k_slab.clone(),
+                     s.out.float().clone()))
+    assert all(torch.equal(a, b) for a, b in zip(outs[0][:4], outs[1][:4]))
+    assert torch.allclose(outs[0][4], outs[1][4], rtol=2 ** -7, atol=1e-4)
+
+
 def test_filling_from_empty_then_steady_state():
     w = wl.scaled(wl.TINY, T=64, budget=0.5, steps=80)               # capacities of 16 .. 48 tokens
     s = Session(w, prefill=False, chunk_tokens=64)

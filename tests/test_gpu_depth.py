@@ -80,6 +80,20 @@ def test_qwen_8k_batch16_all_128_steps():
     np.testing.assert_array_equal(s.cache.len.cpu().numpy(), np.broadcast_to(expect, (w.B, w.L, w.Hkv)))
 
 
+def test_llama_32k_one_call_per_layer():
+    """The full-size Llama workload issued layer by layer (32 calls per step, each after the first overlapping the
+    tail of the one before it), all heads checked at the first and the last step."""
+    w = wl.scaled(wl.LLAMA3_8B_32K, steps=12)
+    cap = _caps_of(w)
+    teacher = _sample(w, cap, 12)
+    s = Session(w, heads=teacher[:2], per_layer=True)
+    everyone = [(0, l, h) for l in range(w.L) for h in range(w.Hkv)]
+    for i in range(w.steps):
+        s.step(i, teacher=everyone if i in (0, w.steps - 1) else teacher, hold=set(teacher))
+    s.check_held_rows()
+    _report(s, "llama 32K, one call per layer")
+
+
 def test_heads_of_a_131072_token_context():
     # two layers of the sweep's longest point: 90 % of a 128K context, heads of 59K .. 177K rows, tens of chunks each
     w = wl.scaled(wl.sweep_point(1, 131072, 0.9), L=2, steps=4)
