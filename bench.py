@@ -436,7 +436,7 @@ def main():
         sess.prefill_synthetic()
     if args.per_layer != "off":
         # layer by layer, as a model calls attention; positions live on the device and advance there
-        sess.per_layer_plans()
+        sess.per_layer_plans(args.chunk)
         t_dev = torch.full((w.B,), w.T, dtype=torch.int32, device=dev)
         sq, sk, sv = (torch.empty_like(t) for t in wl.decode_inputs(w, 0, sess.scales, dev))
 

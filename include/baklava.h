@@ -151,7 +151,8 @@ typedef struct baklava_alloc_params {
 /* What baklava_decode_plan decided; passed back to baklava_decode_attn unchanged. */
 typedef struct baklava_plan_info {
     int32_t n_items;        /* attention work items (one chunk of one head of one sequence each)    */
-    int32_t n_score_items;  /* always 0 (kept so that the structure's layout is stable)             */
+    int32_t n_score_items;  /* short launches only (all chunks resident at once): pieces of the heads  */
+                            /*   for a score / eviction pass of its own, listed after the items; else 0 */
     int32_t n_units;        /* (layer, sequence, KV head) triples in the layer range                */
     int32_t chunk_tokens;   /* target chunk length the plan used                                    */
     int32_t layer_begin, layer_end, B;
@@ -210,7 +211,7 @@ int baklava_allocate(const baklava_shape* shape, const double* kv_importance,
  *   chunk_tokens  target chunk length, 0 = choose from the total work and n_sm
  *   n_sm          streaming multiprocessors of the device (used when chunk_tokens = 0)
  *   items_out     host int32 [4 * items_capacity] or NULL to only fill `info`
- * The caller copies items_out (info->n_items * 16 bytes) to the device and hands it
+ * The caller copies items_out ((info->n_items + info->n_score_items) * 16 bytes) to the device and hands it
  * to baklava_decode_attn together with `info`. */
 int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t B,
                         int32_t layer_begin, int32_t layer_end, int32_t chunk_tokens, int32_t n_sm,
@@ -240,7 +241,8 @@ int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t 
  *            after a step that set BAKLAVA_STATUS_TIMEOUT.
  * A head with no valid row gives out = 0 and lse = -inf.
  *
- * Ordering on the stream.  A call is one kernel, launched with programmatic stream serialisation: its
+ * Ordering on the stream.  A call is one kernel (two for an unflagged short launch: the score update of
+ * its few long heads is then spread over a second one), launched with programmatic stream serialisation: its
  * blocks may become resident while the work in front of it drains, and they wait for that work to
  * complete before they read anything.  A model calls attention one layer at a time (Eq. 7 per layer),
  * and a call for one layer is too short to fill the GPU: most of its time is the start-up and the tail

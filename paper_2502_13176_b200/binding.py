@@ -154,7 +154,7 @@ def baklava_allocate(shape, kv_importance, t, r_num, r_den, total_tokens, min_to
 
 
 class Plan:
-    """The decode work plan: `items` (int32 [n_items, 4], host) and `info`; `items_dev` after `.to(device)`."""
+    """The decode work plan: `items` (int32 [n_items + n_score_items, 4], host) and `info`; `items_dev` after `.to(device)`."""
 
     def __init__(self, items, info):
         self.items, self.info, self.items_dev = items, info, None
@@ -170,7 +170,7 @@ def baklava_decode_plan(shape, cap, B, layer_begin, layer_end, seq_stride_tokens
     capp = cap.ctypes.data_as(POINTER(c_int32))
     _check(lib().baklava_decode_plan(ctypes.byref(shape), capp, B, layer_begin, layer_end, chunk_tokens, n_sm,
                                      int(seq_stride_tokens), None, 0, ctypes.byref(info)), "baklava_decode_plan")
-    total = info.n_items
+    total = info.n_items + info.n_score_items
     items = np.empty((total, 4), dtype=np.int32)
     _check(lib().baklava_decode_plan(ctypes.byref(shape), capp, B, layer_begin, layer_end, chunk_tokens, n_sm,
                                      int(seq_stride_tokens), items.ctypes.data_as(POINTER(c_int32)), total,

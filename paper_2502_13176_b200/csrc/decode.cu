@@ -69,9 +69,13 @@ struct DecodeParams {
     int32_t window_evict;          // 1: no scores are kept and the policy is sinks + window: evict by position
     const int4* items;             // the plan's work items
     int32_t n_items;
+    int32_t split_tail;            // 1: the score update and the eviction run as a second kernel (short launches)
     int32_t* arrive;               // [n_units]: chunks of a head that have delivered their partial
     float* partial;
     float* logit;
+    float* stats;                  // [n_units][2 * kG]: final (max, 1 / sum) of every query head (split tail only)
+    unsigned long long* best_key;  // [n_score_items]: each piece's eviction candidate (split tail only)
+    int32_t* best_slot;            // [n_score_items]
     float scale_log2;   // log2(e) / sqrt(D)
     const float* kv_scale;   // FP8 slabs: [L, Hkv, 4] (K scale, its reciprocal, V scale, its reciprocal)
     long long wait_cycles;   // SM clock cycles after which a wait on a tile gives up
@@ -134,6 +138,9 @@ __device__ __forceinline__ int arrive_acq_rel(int32_t* ptr) {
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* ptr) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
 __device__ __forceinline__ int ld_acquire(const int32_t* ptr) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
@@ -179,6 +186,30 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a2,
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(zero), "r"(a2), "r"(zero), "r"(b0), "r"(b1));
 }
+// D (16x8, fp32) += A (16x16, row) * B (16x8, col), all four A registers in use
+__device__ __forceinline__ void mma_bf16_full(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                              uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16_full(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// transpose of an 8 x 8 matrix of 16-bit elements held one row per quad of lanes (lane / 4 = row, two
+// consecutive elements per lane): afterwards lane (g, t) holds elements (2 t, g) and (2 t + 1, g)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     const __half2 v = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
@@ -189,11 +220,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // ---------------------------------------------------------------- steps 3-4: scores and the row to evict
-// Run by the CTA that delivered a head's last partial, over the whole head.  Every row's stored probabilities
+// Run over the whole head by the CTA that delivered its last partial, or over a piece of it by a CTA of the
+// second kernel of a short launch.  Every row's stored probabilities
 // are brought to the head's final normaliser and added to its score; rows that may be evicted compete on the
 // 64-bit key (score bits, inverted position): the smallest key is the lowest score and, among equal scores,
 // the latest token.  Eight consecutive rows per thread and group (they share one 16-row block, hence one
-// reference maximum per query head), two groups in flight.  Each warp leaves its best candidate in shared
+// reference maximum per query head), two or three groups in flight.  Each warp leaves its best candidate in shared
 // memory.
 template <int G>
 struct SweepGroup {
@@ -205,8 +237,9 @@ struct SweepGroup {
 
 template <int G>
 __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, const int32_t* pos, int n_sink, int C,
-                                           int n_hi, int hole, bool evict, int newest_candidate, const float* sm_M,
-                                           const float* sm_invL, unsigned long long* sm_key, int* sm_slot) {
+                                           int j_begin, int n_hi, int hole, bool evict, int newest_candidate,
+                                           const float* sm_M, const float* sm_invL, unsigned long long* sm_key,
+                                           int* sm_slot) {                // rows j_begin (a multiple of 64) .. n_hi - 1
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const __half* prob_h = reinterpret_cast<const __half*>(logit_h);
     const float* mref_h = reinterpret_cast<const float*>(prob_h + (int64_t)G * C);
@@ -265,7 +298,18 @@ __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, c
 
     constexpr int kStride = 8 * kThreads;
     const int n_full = n_hi & ~7;                          // rows covered by full groups
-    int j0 = 8 * tid;
+    int j0 = j_begin + 8 * tid;
+    if (G <= 4) {
+        for (; j0 + 2 * kStride < n_full; j0 += 3 * kStride) {   // three full groups of this thread in flight
+            SweepGroup<G> g0, g1, g2;
+            load(g0, j0);
+            load(g1, j0 + kStride);
+            load(g2, j0 + 2 * kStride);
+            finish(g0, j0);
+            finish(g1, j0 + kStride);
+            finish(g2, j0 + 2 * kStride);
+        }
+    }
     for (; j0 + kStride < n_full; j0 += 2 * kStride) {     // two full groups of this thread in flight
         SweepGroup<G> g0, g1;
         load(g0, j0);
@@ -279,7 +323,7 @@ __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, c
         finish(g0, j0);
     }
     // the ragged end of the head: fewer than eight rows, one thread
-    if (tid == ((n_full >> 3) % kThreads) && n_full < n_hi) {
+    if (tid == (((n_full - j_begin) >> 3) % kThreads) && n_full < n_hi) {
         float f[G];
 #pragma unroll
         for (int a = 0; a < G; ++a) {
@@ -329,12 +373,41 @@ struct TailArgs {
     int32_t* len;
     int32_t* free_slot;
     uint32_t* status;
+    float* stats;                  // the head's final (max, 1 / sum), for a score pass that runs as a second kernel
     int active, G, C, n, n_hi, hole, n_sink, newest_candidate;
-    bool keep_logits, do_append, may_evict, pos_evict, overlap;
+    bool keep_logits, do_append, may_evict, pos_evict, overlap, split;
 };
 
 template <int D, bool kByPosition>
-__device__ __noinline__ void finish_head(const TailArgs t) {
+__device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch, int unit, int piece, int active) {
+    // everything about the head is derived again from the parameters, so that the call passes five values
+    const DecodeParams& p = *pp;
+    const Unit u = decode_unit(p, unit);
+    const HeadState hs = head_state(p, u);
+    const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
+    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    TailArgs t;
+    t.part0 = p.partial + (int64_t)((int)blockIdx.x - piece) * partial_floats(p.G, D);
+    t.scratch = scratch;
+    t.arrive = p.arrive + unit;
+    t.lse = p.lse ? p.lse + (int64_t)(u.li * p.B + u.b) * p.Hq + u.h * p.G : nullptr;
+    t.out = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * p.G) * D;
+    t.logit_h = p.logit + row0 * p.G;
+    t.score = p.score + row0;
+    t.pos = p.pos + row0;
+    t.len = p.len + u.st;
+    t.free_slot = p.free_slot + u.st;
+    t.status = p.status;
+    t.stats = p.stats + (int64_t)unit * 2 * BAKLAVA_MAX_GROUP;
+    t.active = active; t.G = p.G; t.C = hs.C; t.n = hs.n; t.n_hi = hs.n_att; t.hole = hs.hole; t.n_sink = p.n_sink;
+    // rows with a later position are in the recent window
+    t.newest_candidate = t_pos - max(0, (int)(((int64_t)(hs.C - 1 - p.n_sink) * p.recent_num) / p.recent_den));
+    t.keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
+    t.do_append = hs.do_append;
+    t.may_evict = hs.do_append && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && hs.n_att > hs.C - 1;
+    t.pos_evict = kByPosition && hs.do_append && hs.n_att > hs.C - 1;
+    t.overlap = (p.flags & BAKLAVA_FLAG_OVERLAP_PREV) != 0;
+    t.split = !kByPosition && t.keep_logits && p.split_tail != 0;
     constexpr int kG = BAKLAVA_MAX_GROUP;
     __shared__ float sm_M[kG];
     __shared__ float sm_invL[kG];
@@ -342,7 +415,7 @@ __device__ __noinline__ void finish_head(const TailArgs t) {
     __shared__ unsigned long long sm_key[kThreads / 32];   // each warp's eviction candidate
     __shared__ int sm_slot[kThreads / 32];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = t.G, active = t.active;
+    const int G = t.G;
     const int psz = partial_floats(G, D);
     const float* part0 = t.part0;
     // every chunk's (max, sum) into shared memory with one round of loads (the plan keeps chunks x group
@@ -365,6 +438,7 @@ __device__ __noinline__ void finish_head(const TailArgs t) {
         // lost step: no output, no score update, no bookkeeping; the counter goes back to zero
         if (tid == 0) {
             *t.arrive = 0;
+            if (t.split) t.stats[0] = __int_as_float(0x7fc00000);   // the second kernel is told
             if (t.overlap) grid_dependency_wait();
         }
         return;
@@ -384,6 +458,7 @@ __device__ __noinline__ void finish_head(const TailArgs t) {
         if (lane == 0) {
             sm_M[a] = mm;
             sm_invL[a] = ll > 0.0f ? 1.0f / ll : 0.0f;
+            if (t.split) { t.stats[a] = mm; t.stats[kG + a] = sm_invL[a]; }
             if (t.lse) t.lse[a] = ll > 0.0f ? (mm + log2f(ll)) * kLn2 : -INFINITY;
         }
     }
@@ -398,13 +473,25 @@ __device__ __noinline__ void finish_head(const TailArgs t) {
         const int a = (grp * 4) / D;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         int c = 0;
-        for (; c + 8 <= active; c += 8) {                   // eight chunks' loads in flight
-            float4 oc[8];
+        for (; c + 16 <= active; c += 16) {                 // sixteen chunks' loads in flight
+            float4 oc[16];
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
+            for (int k = 0; k < 16; ++k)
                 oc[k] = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)(c + k) * psz) + grp);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < 16; ++k) {
+                const float wgt = sm_lc[(c + k) * G + a];
+                acc.x = fmaf(oc[k].x, wgt, acc.x); acc.y = fmaf(oc[k].y, wgt, acc.y);
+                acc.z = fmaf(oc[k].z, wgt, acc.z); acc.w = fmaf(oc[k].w, wgt, acc.w);
+            }
+        }
+        for (; c + 4 <= active; c += 4) {
+            float4 oc[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                oc[k] = __ldcg(reinterpret_cast<const float4*>(part0 + (int64_t)(c + k) * psz) + grp);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
                 const float wgt = sm_lc[(c + k) * G + a];
                 acc.x = fmaf(oc[k].x, wgt, acc.x); acc.y = fmaf(oc[k].y, wgt, acc.y);
                 acc.z = fmaf(oc[k].z, wgt, acc.z); acc.w = fmaf(oc[k].w, wgt, acc.w);
@@ -425,18 +512,24 @@ __device__ __noinline__ void finish_head(const TailArgs t) {
         *reinterpret_cast<uint2*>(t.out + grp * 4) = packed;
     }
 
+    if (t.split) {                                          // steps 3-4 follow as a kernel of their own
+        __syncthreads();
+        if (tid == 0) *t.arrive = 0;
+        return;
+    }
+
     // ---- steps 3-4
     const bool evict = !kByPosition && t.keep_logits && t.may_evict;
     if (!kByPosition && t.keep_logits) {
         switch (G) {
-            case 1: sweep_head<1>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 2: sweep_head<2>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 3: sweep_head<3>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 4: sweep_head<4>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 5: sweep_head<5>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 6: sweep_head<6>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 7: sweep_head<7>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            default: sweep_head<8>(t.logit_h, t.score, t.pos, t.n_sink, t.C, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 1: sweep_head<1>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 2: sweep_head<2>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 3: sweep_head<3>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 4: sweep_head<4>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 5: sweep_head<5>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 6: sweep_head<6>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 7: sweep_head<7>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            default: sweep_head<8>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
         }
     }
     __syncthreads();                                        // output, scores and the warps' candidates are written
@@ -484,7 +577,7 @@ __device__ __noinline__ void finish_head(const TailArgs t) {
 // and become two fp16 pairs; V comes through ldmatrix.trans as two tokens x two adjacent channels per
 // register, which a byte permute splits into an even-channel and an odd-channel operand.
 template <int D, bool kByPosition, bool kFp8>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(const DecodeParams p,
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(const __grid_constant__ DecodeParams p,
                                                                 const __grid_constant__ CUtensorMap k_map,
                                                                 const __grid_constant__ CUtensorMap v_map) {
     constexpr int kKSteps = D / 16;                    // MMA k-steps over the head dimension
@@ -567,14 +660,26 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
 
+    // The head's tail reads and rewrites the score (and reads the position) of every row; those lines were last
+    // touched a whole step ago.  Each chunk asks for its own share now, so that the tail finds them in L2.
+    if (!kByPosition && keep_logits) {
+        for (int r = begin + 32 * tid; r < end; r += 32 * kThreads) {
+            prefetch_l2(p.score + row0 + r);
+            prefetch_l2(p.pos + row0 + r);
+        }
+    }
     __syncthreads();                                      // the barriers are initialised
 
-    // per-warp online-softmax state; row q of the group lives in the quad of lanes with lane / 4 == q
-    const int qrow = lane >> 2, qcol = (lane & 3) * 2;
-    float m_run = -INFINITY, l_run = 0.0f;
-    float o[kNTiles][4];
+    // Tokens sit on the M side of both contractions (S^T = K Q^T and O^T = V^T P^T): a 16-token block costs
+    // D / 16 MMAs each, with every accumulator row in use.  Lane (g, t) = (lane / 4, lane % 4) of a consumer warp
+    // holds, of S^T, tokens g and g + 8 of the block for the query heads 2 t and 2 t + 1, and, of O^T, two
+    // channels of every 16-channel group for the same two heads; its online-softmax state is that of those two
+    // heads (the maximum shared by the warp, the sum its own rows' share, added up at the end of the chunk).
+    const int g8 = lane >> 2, t4 = lane & 3;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
+    float o[D / 16][4];
 #pragma unroll
-    for (int j = 0; j < kNTiles; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f; }
+    for (int j = 0; j < D / 16; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f; }
 
     if (warp == kConsumerWarps) {
         // ---------------- producer: one lane issues the TMA loads
@@ -612,26 +717,28 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         }
     } else {
         // ---------------- consumers
-        // query fragments (A operand): rows >= G are zero; a0 covers k 0..7 of a k-step, a2 k 8..15
-        uint32_t qa0[kKSteps], qa2[kKSteps];
+        // query fragments (B operand of S^T): head g of the group (zero from G on), per 16-channel step the
+        // channels 2 t, 2 t + 1 (q0) and 8 + 2 t, 9 + 2 t (q1); for FP8 slabs the channels 4 t .. 4 t + 3, the order
+        // in which the four bytes of a K register arrive (the contraction index may be permuted at will)
+        uint32_t q0[kKSteps], q1[kKSteps];
         {
-            const __nv_bfloat16* qrow_ptr = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + qrow) * D;
+            const __nv_bfloat16* q_ptr = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + g8) * D;
 #pragma unroll
             for (int ks = 0; ks < kKSteps; ++ks) {
                 if (kFp8) {
-                    // channels 16 ks + 4 (lane % 4) + {0, 1} and + {2, 3}: the order the K bytes arrive in
-                    const uint2 raw = qrow < G ? *reinterpret_cast<const uint2*>(qrow_ptr + ks * 16 + 2 * qcol) : make_uint2(0u, 0u);
+                    const uint2 raw = g8 < G ? *reinterpret_cast<const uint2*>(q_ptr + ks * 16 + 4 * t4) : make_uint2(0u, 0u);
                     const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
                     const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                    qa0[ks] = pack_f16(f0.x, f0.y);
-                    qa2[ks] = pack_f16(f1.x, f1.y);
+                    q0[ks] = pack_f16(f0.x, f0.y);
+                    q1[ks] = pack_f16(f1.x, f1.y);
                 } else {
-                    qa0[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + qcol) : 0u;
-                    qa2[ks] = qrow < G ? *reinterpret_cast<const uint32_t*>(qrow_ptr + ks * 16 + 8 + qcol) : 0u;
+                    q0[ks] = g8 < G ? *reinterpret_cast<const uint32_t*>(q_ptr + ks * 16 + 2 * t4) : 0u;
+                    q1[ks] = g8 < G ? *reinterpret_cast<const uint32_t*>(q_ptr + ks * 16 + 8 + 2 * t4) : 0u;
                 }
             }
         }
         const int lm = lane >> 3, li8 = lane & 7;          // ldmatrix: matrix index and row inside it
+        const int w0 = warp * kBlocks * kWarpTokens;       // this warp's rows inside a tile
         bool alive = true;
         for (int it = 0; it < n_tiles && alive; ++it) {
             const int s = it % kStages;
@@ -642,162 +749,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             }
             const uint32_t k_tile = ring + s * kStageBytes;
             const uint32_t v_tile = k_tile + kTileBytes;
-            if constexpr (kBlocks == 1) {
-            // one 16-token block per warp and stage
-#pragma unroll
-            for (int blk = 0; blk < kBlocks; ++blk) {
-            const int r0 = (warp * kBlocks + blk) * kWarpTokens;     // this block's rows inside the tile
-            const int tok0 = begin + it * kTT + r0;                  // first token of the block
-            const int valid = min(kWarpTokens, end - tok0);          // rows of the block inside the chunk
-            if (valid > 0) {
-                if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + kWarpTokens) {
-                    // step 1 (Eq. 4): the new token's row replaces whatever the tile holds at the free slot,
-                    // in shared memory for this pass and in the slab for the steps to come
-                    constexpr int kVec = D / 8;
-                    const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
-                    const int64_t row = row0 + hs.f;
-                    uint8_t* k_ptr = ring_ptr + s * kStageBytes;
-                    if (kFp8) {                              // quantise the row: eight elements per lane and operand
-                        for (int i = lane; i < 2 * kVec; i += 32) {
-                            const bool is_v = i >= kVec;
-                            const int c = is_v ? i - kVec : i;
-                            const uint4 raw = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
-                            const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + (is_v ? 3 : 1)]);
-                            *reinterpret_cast<uint2*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c >> 1) +
-                                                      (c & 1) * 8) = val;
-                            uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
-                            *(reinterpret_cast<uint2*>(slab + row * D) + c) = val;
-                        }
-                    } else {
-                    for (int i = lane; i < 2 * kVec; i += 32) {
-                        const bool is_v = i >= kVec;
-                        const int c = is_v ? i - kVec : i;
-                        const uint4 val = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
-                        *reinterpret_cast<uint4*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c)) = val;
-                        *(reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c) = val;
-                    }
-                    }
-                    if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
-                    __syncwarp();
-                }
-                if (kByPosition && pos_evict && lane < valid && tok0 + lane != hs.f) {
-                    const int ps = p.pos[row0 + tok0 + lane];
-                    if (ps >= p.n_sink && ps <= window_from && ps < old_pos) { old_pos = ps; old_slot = tok0 + lane; }
-                }
-                // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
-                if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
-                    uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
-                    constexpr int kPieces = kRowBytes / 16;     // 16-byte pieces of a row
-                    for (int i = lane; i < kWarpTokens * kPieces; i += 32) {
-                        const int r = i / kPieces, c = i % kPieces;
-                        if (r >= valid || tok0 + r == hole)
-                            *reinterpret_cast<uint4*>(v_ptr + tile_offset(r0 + r, c)) = make_uint4(0, 0, 0, 0);
-                    }
-                    __syncwarp();
-                }
-                // S = Q K^T for 16 tokens: two 8-token column blocks
-                float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                if (kFp8) {
-#pragma unroll
-                    for (int kk = 0; kk < D / 32; ++kk) {     // 32 channels per load: two k-steps for both token blocks
-                        uint32_t kb[4];
-                        ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * kk + (lm & 1)), kb);
-#pragma unroll
-                        for (int c = 0; c < 2; ++c) {
-                            const int ks = 2 * kk + c;
-                            mma_f16(sacc[0], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[c]), fp8::f16x2_from_e4m3x2(kb[c] >> 16));
-                            mma_f16(sacc[1], qa0[ks], qa2[ks], fp8::f16x2_from_e4m3x2(kb[2 + c]),
-                                    fp8::f16x2_from_e4m3x2(kb[2 + c] >> 16));
-                        }
-                    }
-                } else {
-#pragma unroll
-                for (int ks = 0; ks < kKSteps; ++ks) {
-                    uint32_t kb[4];
-                    ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kb);
-                    mma_bf16(sacc[0], qa0[ks], qa2[ks], kb[0], kb[1]);
-                    mma_bf16(sacc[1], qa0[ks], qa2[ks], kb[2], kb[3]);
-                }
-                }
-                // this thread: row qrow, tokens tok0 + 8 t + qcol + {0, 1}
-                float sv[4];
-                bool ok[4];
-#pragma unroll
-                for (int t = 0; t < 2; ++t)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int tok = tok0 + 8 * t + qcol + e;
-                        sv[2 * t + e] = sacc[t][e] * scale_k;
-                        ok[2 * t + e] = tok < end && tok != hole;
-                    }
-                float mx = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) mx = fmaxf(mx, ok[i] ? sv[i] : -INFINITY);
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run, mx);
-                const float corr = (m_new == -INFINITY) ? 1.0f : exp2f(m_run - m_new);
-                float pv[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) pv[i] = ok[i] ? exp2f(sv[i] - m_new) : 0.0f;
-                l_run = l_run * corr + (pv[0] + pv[1]) + (pv[2] + pv[3]);
-                m_run = m_new;
-                if (keep_logits && qrow < G) {
-#pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        const int tok = tok0 + 8 * t + qcol;
-                        __half* dst = prob_h + (int64_t)qrow * C + tok;
-                        if (tok + 1 < end) *reinterpret_cast<__half2*>(dst) = __floats2half2_rn(pv[2 * t], pv[2 * t + 1]);
-                        else if (tok < end) dst[0] = __float2half_rn(pv[2 * t]);
-                    }
-                    if ((lane & 3) == 0) mref_h[qrow * (C >> 4) + (tok0 >> 4)] = m_new;
-                }
-                if (__any_sync(0xffffffffu, corr != 1.0f)) {
-#pragma unroll
-                    for (int j = 0; j < kNTiles; ++j) { o[j][0] *= corr; o[j][1] *= corr; }
-                }
-                if (kFp8) {
-                    const uint32_t pa0 = pack_f16(pv[0], pv[1]), pa2 = pack_f16(pv[2], pv[3]);
-                    // a register of the transposed load = two tokens x two adjacent channels; the permute puts the
-                    // even channel's token pair in the low half and the odd channel's in the high half.
-                    // o[2 c] collects channels 16 c + 0, 2, .., 14 and o[2 c + 1] channels 16 c + 1, 3, .., 15.
-#pragma unroll
-                    for (int c2 = 0; c2 < D / 32; ++c2) {
-                        uint32_t vb[4];
-                        ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * c2 + (lm >> 1)), vb);
-#pragma unroll
-                        for (int h2 = 0; h2 < 2; ++h2) {
-                            const uint32_t lo = __byte_perm(vb[2 * h2], 0u, 0x3120), hi = __byte_perm(vb[2 * h2 + 1], 0u, 0x3120);
-                            const int c = 2 * c2 + h2;
-                            mma_f16(o[2 * c], pa0, pa2, fp8::f16x2_from_e4m3x2(lo), fp8::f16x2_from_e4m3x2(hi));
-                            mma_f16(o[2 * c + 1], pa0, pa2, fp8::f16x2_from_e4m3x2(lo >> 16), fp8::f16x2_from_e4m3x2(hi >> 16));
-                        }
-                    }
-                } else {
-                const uint32_t pa0 = pack_bf16(pv[0], pv[1]), pa2 = pack_bf16(pv[2], pv[3]);
-                // O += P V: V^T fragments through ldmatrix.trans, two 8-wide column blocks per load
-#pragma unroll
-                for (int j2 = 0; j2 < kNTiles / 2; ++j2) {
-                    uint32_t vb[4];
-                    ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * j2 + (lm >> 1)), vb);
-                    mma_bf16(o[2 * j2], pa0, pa2, vb[0], vb[1]);
-                    mma_bf16(o[2 * j2 + 1], pa0, pa2, vb[2], vb[3]);
-                }
-                }
-            }
-            }
-            } else {
-            // several 16-token blocks per warp and stage (FP8 rows): one softmax update over all of them,
-            // which halves the serial part per token and gives the MMAs of the blocks to the scheduler together
-            const int w0 = warp * kBlocks * kWarpTokens;             // this warp's rows inside the tile
-            const int wtok0 = begin + it * kTT + w0;                 // their first token
+            const int wtok0 = begin + it * kTT + w0;                 // first token of this warp's share of the stage
             if (wtok0 < end) {
 #pragma unroll
                 for (int blk = 0; blk < kBlocks; ++blk) {            // per 16-token block: patch the tile where needed
                     const int r0 = w0 + blk * kWarpTokens;
                     const int tok0 = wtok0 + blk * kWarpTokens;
-                    const int valid = kBlocks == 1 ? min(kWarpTokens, end - tok0)
-                                                   : max(0, min(kWarpTokens, end - tok0));   // rows of the block inside the chunk
+                    const int valid = max(0, min(kWarpTokens, end - tok0));   // rows of the block inside the chunk
                     if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
                         // step 1 (Eq. 4): the new token's row replaces whatever the tile holds at the free slot,
                         // in shared memory for this pass and in the slab for the steps to come
@@ -844,118 +802,133 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
                         __syncwarp();
                     }
                 }
-                // S = Q K^T for the warp's 16 * kBlocks tokens: 8-token column blocks, all under one softmax update
-                constexpr int kCols = 2 * kBlocks;
-                float sacc[kCols][4];
+                // S^T = K Q^T for the warp's 16 * kBlocks tokens: st[blk] = (token g: heads 2 t, 2 t + 1; token g + 8: same)
+                float st[kBlocks][4];
 #pragma unroll
-                for (int t = 0; t < kCols; ++t) { sacc[t][0] = sacc[t][1] = sacc[t][2] = sacc[t][3] = 0.0f; }
-#pragma unroll
-                for (int sb = 0; sb < kBlocks; ++sb) {
-                    const int r0 = w0 + sb * kWarpTokens;
+                for (int blk = 0; blk < kBlocks; ++blk) {
+                    st[blk][0] = st[blk][1] = st[blk][2] = st[blk][3] = 0.0f;
+                    const int r0 = w0 + blk * kWarpTokens;
                     if (kFp8) {
 #pragma unroll
-                        for (int kk = 0; kk < D / 32; ++kk) {     // 32 channels per load: two k-steps for both token blocks
-                            uint32_t kb[4];
+                        for (int kk = 0; kk < D / 32; ++kk) {     // 32 channels per load: two steps of 16
+                            uint32_t kb[4];      // (tokens 0-7 | 8-15) x (channels 0-15 | 16-31), four bytes per lane
                             ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * kk + (lm & 1)), kb);
 #pragma unroll
                             for (int c = 0; c < 2; ++c) {
-                                const int ks = 2 * kk + c;
-                                uint32_t b0, b1;
-                                fp8::f16x4_from_e4m3x4(kb[c], b0, b1);
-                                mma_f16(sacc[2 * sb], qa0[ks], qa2[ks], b0, b1);
-                                fp8::f16x4_from_e4m3x4(kb[2 + c], b0, b1);
-                                mma_f16(sacc[2 * sb + 1], qa0[ks], qa2[ks], b0, b1);
+                                uint32_t a0, a2, a1, a3;
+                                fp8::f16x4_from_e4m3x4(kb[c], a0, a2);
+                                fp8::f16x4_from_e4m3x4(kb[2 + c], a1, a3);
+                                mma_f16_full(st[blk], a0, a1, a2, a3, q0[2 * kk + c], q1[2 * kk + c]);
                             }
                         }
                     } else {
 #pragma unroll
                         for (int ks = 0; ks < kKSteps; ++ks) {
-                            uint32_t kb[4];
+                            uint32_t kb[4];      // (tokens 0-7 | 8-15) x (channels 0-7 | 8-15) of the step
                             ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kb);
-                            mma_bf16(sacc[2 * sb], qa0[ks], qa2[ks], kb[0], kb[1]);
-                            mma_bf16(sacc[2 * sb + 1], qa0[ks], qa2[ks], kb[2], kb[3]);
+                            mma_bf16_full(st[blk], kb[0], kb[2], kb[1], kb[3], q0[ks], q1[ks]);
                         }
                     }
                 }
-                // this thread: row qrow, tokens wtok0 + 8 t + qcol + {0, 1}
-                float sv[2 * kCols];
-                bool ok[2 * kCols];
+                // online softmax for the two heads of this lane over the warp's tokens of the stage
+                float mx[2] = {-INFINITY, -INFINITY};
+                bool ok[kBlocks][2];
 #pragma unroll
-                for (int t = 0; t < kCols; ++t)
+                for (int blk = 0; blk < kBlocks; ++blk)
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int tok = wtok0 + 8 * t + qcol + e;
-                        sv[2 * t + e] = sacc[t][e] * scale_k;
-                        ok[2 * t + e] = tok < end && tok != hole;
+                    for (int r = 0; r < 2; ++r) {
+                        const int tok = wtok0 + blk * kWarpTokens + g8 + 8 * r;
+                        ok[blk][r] = tok < end && tok != hole;
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            st[blk][2 * r + e] *= scale_k;
+                            if (ok[blk][r]) mx[e] = fmaxf(mx[e], st[blk][2 * r + e]);
+                        }
                     }
-                float mx = -INFINITY;
+                float corr[2];
 #pragma unroll
-                for (int i = 0; i < 2 * kCols; ++i) mx = fmaxf(mx, ok[i] ? sv[i] : -INFINITY);
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run, mx);
-                const float corr = (m_new == -INFINITY) ? 1.0f : exp2f(m_run - m_new);
-                float pv[2 * kCols];
+                for (int e = 0; e < 2; ++e) {
+                    mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 4));
+                    mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 8));
+                    mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 16));
+                    const float m_new = fmaxf(m_run[e], mx[e]);
+                    corr[e] = (m_new == -INFINITY) ? 1.0f : exp2f(m_run[e] - m_new);
+                    m_run[e] = m_new;
+                }
+                float psum[2] = {0.0f, 0.0f};
 #pragma unroll
-                for (int i = 0; i < 2 * kCols; ++i) pv[i] = ok[i] ? exp2f(sv[i] - m_new) : 0.0f;
-                float psum = (pv[0] + pv[1]) + (pv[2] + pv[3]);
+                for (int blk = 0; blk < kBlocks; ++blk)
 #pragma unroll
-                for (int sb = 1; sb < kBlocks; ++sb) psum += (pv[4 * sb] + pv[4 * sb + 1]) + (pv[4 * sb + 2] + pv[4 * sb + 3]);
-                l_run = l_run * corr + psum;
-                m_run = m_new;
-                if (keep_logits && qrow < G) {
+                    for (int r = 0; r < 2; ++r)
 #pragma unroll
-                    for (int t = 0; t < kCols; ++t) {
-                        const int tok = wtok0 + 8 * t + qcol;
-                        __half* dst = prob_h + (int64_t)qrow * C + tok;
-                        if (tok + 1 < end) *reinterpret_cast<__half2*>(dst) = __floats2half2_rn(pv[2 * t], pv[2 * t + 1]);
-                        else if (tok < end) dst[0] = __float2half_rn(pv[2 * t]);
+                        for (int e = 0; e < 2; ++e) {
+                            const float pv = ok[blk][r] ? exp2f(st[blk][2 * r + e] - m_run[e]) : 0.0f;
+                            st[blk][2 * r + e] = pv;
+                            psum[e] += pv;
+                        }
+                l_run[0] = l_run[0] * corr[0] + psum[0];
+                l_run[1] = l_run[1] * corr[1] + psum[1];
+                if (__any_sync(0xffffffffu, corr[0] != 1.0f || corr[1] != 1.0f)) {
+#pragma unroll
+                    for (int j = 0; j < D / 16; ++j) { o[j][0] *= corr[0]; o[j][1] *= corr[1]; o[j][2] *= corr[0]; o[j][3] *= corr[1]; }
+                }
+                // P^T as the B operand of O^T += V^T P^T: the 8 x 8 blocks (tokens x heads) this warp holds one
+                // row per quad are transposed, so that lane (g, t) gets head g, tokens 2 t, 2 t + 1 (and + 8)
+                uint32_t pb[kBlocks][2];
+#pragma unroll
+                for (int blk = 0; blk < kBlocks; ++blk) {
+                    const int tok0 = wtok0 + blk * kWarpTokens;
+                    const uint32_t h0 = movmatrix_trans(pack_f16(st[blk][0], st[blk][1]));
+                    const uint32_t h1 = movmatrix_trans(pack_f16(st[blk][2], st[blk][3]));
+                    if (kFp8) {
+                        pb[blk][0] = h0; pb[blk][1] = h1;
+                    } else {
+                        pb[blk][0] = movmatrix_trans(pack_bf16(st[blk][0], st[blk][1]));
+                        pb[blk][1] = movmatrix_trans(pack_bf16(st[blk][2], st[blk][3]));
                     }
-                    if ((lane & 3) == 0) {
-#pragma unroll
-                        for (int sb = 0; sb < kBlocks; ++sb)      // the reference maximum of every 16-token block written
-                            if (wtok0 + sb * kWarpTokens < end) mref_h[qrow * (C >> 4) + (wtok0 >> 4) + sb] = m_new;
+                    if (keep_logits && g8 < G && tok0 < end) {
+                        // the unnormalised probabilities of head g, in fp16, and the maximum they were taken under
+                        __half* dst = prob_h + (int64_t)g8 * C + tok0 + 2 * t4;
+                        if (tok0 + 2 * t4 + 1 < end) *reinterpret_cast<uint32_t*>(dst) = h0;
+                        else if (tok0 + 2 * t4 < end) dst[0] = __ushort_as_half((unsigned short)(h0 & 0xffffu));
+                        if (tok0 + 8 + 2 * t4 + 1 < end) *reinterpret_cast<uint32_t*>(dst + 8) = h1;
+                        else if (tok0 + 8 + 2 * t4 < end) dst[8] = __ushort_as_half((unsigned short)(h1 & 0xffffu));
+                    }
+                    if (keep_logits && g8 == 0 && tok0 < end) {
+                        if (2 * t4 < G) mref_h[(2 * t4) * (C >> 4) + (tok0 >> 4)] = m_run[0];
+                        if (2 * t4 + 1 < G) mref_h[(2 * t4 + 1) * (C >> 4) + (tok0 >> 4)] = m_run[1];
                     }
                 }
-                if (__any_sync(0xffffffffu, corr != 1.0f)) {
+                // O^T += V^T P^T: V^T fragments through ldmatrix.trans
 #pragma unroll
-                    for (int j = 0; j < kNTiles; ++j) { o[j][0] *= corr; o[j][1] *= corr; }
-                }
-                if (kFp8) {
-                    // a register of the transposed load = two tokens x two adjacent channels; the permute puts the
-                    // even channel's token pair in the low half and the odd channel's in the high half.
-                    // o[2 c] collects channels 16 c + 0, 2, .., 14 and o[2 c + 1] channels 16 c + 1, 3, .., 15.
+                for (int blk = 0; blk < kBlocks; ++blk) {
+                    const int r0 = w0 + blk * kWarpTokens;
+                    if (kFp8) {
+                        // a register of the transposed load = two tokens x two adjacent channels; the permute puts the
+                        // even channel's token pair in the low half and the odd channel's in the high half.  Row g of
+                        // the MMA is channel 2 g of the 16-channel group, row g + 8 channel 2 g + 1.
 #pragma unroll
-                    for (int c2 = 0; c2 < D / 32; ++c2) {
-#pragma unroll
-                        for (int sb = 0; sb < kBlocks; ++sb) {
-                            const uint32_t pa0 = pack_f16(pv[4 * sb], pv[4 * sb + 1]), pa2 = pack_f16(pv[4 * sb + 2], pv[4 * sb + 3]);
-                            uint32_t vb[4];
-                            ldmatrix_x4_trans(v_tile + tile_offset(w0 + sb * kWarpTokens + (lm & 1) * 8 + li8, 2 * c2 + (lm >> 1)), vb);
+                        for (int c2 = 0; c2 < D / 32; ++c2) {
+                            uint32_t vb[4];      // (tokens 0-7 | 8-15) x (channels 0-15 | 16-31)
+                            ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * c2 + (lm >> 1)), vb);
 #pragma unroll
                             for (int h2 = 0; h2 < 2; ++h2) {
                                 const uint32_t lo = __byte_perm(vb[2 * h2], 0u, 0x3120), hi = __byte_perm(vb[2 * h2 + 1], 0u, 0x3120);
-                                const int c = 2 * c2 + h2;
                                 uint32_t even0, odd0, even1, odd1;               // tokens 0-7 and 8-15 of the block
                                 fp8::f16x4_from_e4m3x4(lo, even0, odd0);
                                 fp8::f16x4_from_e4m3x4(hi, even1, odd1);
-                                mma_f16(o[2 * c], pa0, pa2, even0, even1);
-                                mma_f16(o[2 * c + 1], pa0, pa2, odd0, odd1);
+                                mma_f16_full(o[2 * c2 + h2], even0, odd0, even1, odd1, pb[blk][0], pb[blk][1]);
                             }
                         }
-                    }
-                } else {
-                    // O += P V: V^T fragments through ldmatrix.trans, two 8-wide column blocks per load
-                    const uint32_t pa0 = pack_bf16(pv[0], pv[1]), pa2 = pack_bf16(pv[2], pv[3]);
+                    } else {
 #pragma unroll
-                    for (int j2 = 0; j2 < kNTiles / 2; ++j2) {
-                        uint32_t vb[4];
-                        ldmatrix_x4_trans(v_tile + tile_offset(w0 + (lm & 1) * 8 + li8, 2 * j2 + (lm >> 1)), vb);
-                        mma_bf16(o[2 * j2], pa0, pa2, vb[0], vb[1]);
-                        mma_bf16(o[2 * j2 + 1], pa0, pa2, vb[2], vb[3]);
+                        for (int c = 0; c < D / 16; ++c) {
+                            uint32_t vb[4];      // (tokens 0-7 | 8-15) x (channels 0-7 | 8-15) of the group
+                            ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * c + (lm >> 1)), vb);
+                            mma_bf16_full(o[c], vb[0], vb[2], vb[1], vb[3], pb[blk][0], pb[blk][1]);
+                        }
                     }
                 }
-            }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
@@ -988,22 +961,30 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             }
             if (lane == 0) { sm_old_pos[warp] = old_pos; sm_old_slot[warp] = old_slot; }
         }
-        float lq = l_run;
-        lq += __shfl_xor_sync(0xffffffffu, lq, 1);
-        lq += __shfl_xor_sync(0xffffffffu, lq, 2);
-        if (qrow < G) {
-            if (kFp8) {                                         // four consecutive channels per thread and 16-channel group
-                const float sv_ = p.kv_scale[u.head * 4 + 2];
+        // the sums were kept per lane (its own token rows): add them up over the eight row groups
 #pragma unroll
-                for (int c = 0; c < D / 16; ++c)
-                    *reinterpret_cast<float4*>(sm_o + ((warp * G + qrow) * D + 16 * c + 2 * qcol)) =
-                        make_float4(o[2 * c][0] * sv_, o[2 * c + 1][0] * sv_, o[2 * c][1] * sv_, o[2 * c + 1][1] * sv_);
-            } else {
+        for (int e = 0; e < 2; ++e) {
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 4);
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 8);
+            l_run[e] += __shfl_xor_sync(0xffffffffu, l_run[e], 16);
+        }
+        const float sv_ = kFp8 ? p.kv_scale[u.head * 4 + 2] : 1.0f;
 #pragma unroll
-            for (int j = 0; j < kNTiles; ++j)
-                *reinterpret_cast<float2*>(sm_o + ((warp * G + qrow) * D + 8 * j + qcol)) = make_float2(o[j][0], o[j][1]);
+        for (int e = 0; e < 2; ++e) {
+            const int head = 2 * t4 + e;
+            if (head < G) {
+                float* dst = sm_o + (warp * G + head) * D;
+#pragma unroll
+                for (int c = 0; c < D / 16; ++c) {
+                    if (kFp8) {                             // rows g and g + 8 of the MMA are channels 2 g and 2 g + 1
+                        *reinterpret_cast<float2*>(dst + 16 * c + 2 * g8) = make_float2(o[c][e] * sv_, o[c][2 + e] * sv_);
+                    } else {
+                        dst[16 * c + g8] = o[c][e];
+                        dst[16 * c + 8 + g8] = o[c][2 + e];
+                    }
+                }
+                if (g8 == 0) { sm_m[warp][head] = m_run[e]; sm_l[warp][head] = l_run[e]; }
             }
-            if ((lane & 3) == 0) { sm_m[warp][qrow] = m_run; sm_l[warp][qrow] = lq; }
         }
     }
     __syncthreads();
@@ -1036,26 +1017,104 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     if (!sm_last) return;
 
     // ---- this CTA delivered the head's last partial and finishes the head
-    TailArgs t;
-    t.part0 = p.partial + (int64_t)(blockIdx.x - piece) * psz;
-    t.scratch = reinterpret_cast<float*>(ring_ptr);         // the ring is idle now
-    t.arrive = p.arrive + unit;
-    t.lse = p.lse ? p.lse + (int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G : nullptr;
-    t.out = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
-    t.logit_h = p.logit + row0 * G;
-    t.score = p.score + row0;
-    t.pos = p.pos + row0;
-    t.len = p.len + u.st;
-    t.free_slot = p.free_slot + u.st;
-    t.status = p.status;
-    t.active = active; t.G = G; t.C = C; t.n = n; t.n_hi = n_hi; t.hole = hole; t.n_sink = p.n_sink;
-    t.newest_candidate = window_from;                       // rows with a later position are in the recent window
-    t.keep_logits = keep_logits;
-    t.do_append = hs.do_append;
-    t.may_evict = hs.do_append && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n_hi > C - 1;
-    t.pos_evict = pos_evict;
-    t.overlap = overlap;
-    finish_head<D, kByPosition>(t);
+    finish_head<D, kByPosition>(&p, reinterpret_cast<float*>(ring_ptr), unit, piece, active);   // the ring is idle now
+}
+
+// ---------------------------------------------------------------- steps 3-4 as a kernel of their own
+// A short launch (one layer of one sequence) ends with a few long heads, and one CTA sweeping a long head would
+// be most of the call's time.  There the attention kernel stops after the merged output and this kernel follows:
+// one CTA per piece of a head does the score update of its rows; the CTA that finishes a head last picks the
+// head's victim among the pieces' candidates and does the bookkeeping.
+__global__ void __launch_bounds__(kThreads) sweep_kernel(const DecodeParams p) {
+    constexpr int kG = BAKLAVA_MAX_GROUP;
+    __shared__ float sm_M[kG];
+    __shared__ float sm_invL[kG];
+    __shared__ unsigned long long sm_key[kThreads / 32];
+    __shared__ int sm_slot[kThreads / 32];
+    __shared__ int sm_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = p.G;
+    launch_dependents();                                  // what follows waits for this grid by itself
+    grid_dependency_wait();                               // the attention kernel: statistics, scratch, appended rows
+    const int4 item = p.items[p.n_items + blockIdx.x];
+    const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
+    const Unit u = decode_unit(p, unit);
+    const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
+    const HeadState hs = head_state(p, u);                // unchanged so far: this kernel does the bookkeeping
+    if (hs.bad || t_pos < 0) return;                      // reported by the attention kernel / idle sequence
+    const int C = hs.C, n = hs.n, n_hi = hs.n_att;
+    const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
+    if (piece >= active) return;
+    const int end = min(begin + chunk_len, n_hi);
+    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    if (tid < G) {
+        sm_M[tid] = p.stats[(int64_t)unit * 2 * kG + tid];
+        sm_invL[tid] = p.stats[(int64_t)unit * 2 * kG + kG + tid];
+    }
+    __syncthreads();
+    const bool lost = sm_M[0] != sm_M[0];                  // the attention kernel gave the head's step up
+    const bool appended = hs.do_append && !lost;
+    const bool evict = appended && (p.flags & BAKLAVA_FLAG_NO_EVICT) == 0 && n_hi > C - 1;
+    const int newest_candidate = t_pos - max(0, (int)(((int64_t)(C - 1 - p.n_sink) * p.recent_num) / p.recent_den));
+    if (!lost && begin < end) {
+        const float* logit_h = p.logit + row0 * G;
+        float* score = p.score + row0;
+        const int32_t* pos = p.pos + row0;
+        switch (G) {
+            case 1: sweep_head<1>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 2: sweep_head<2>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 3: sweep_head<3>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 4: sweep_head<4>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 5: sweep_head<5>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 6: sweep_head<6>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 7: sweep_head<7>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            default: sweep_head<8>(logit_h, score, pos, p.n_sink, C, begin, end, hs.hole, evict, newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+        }
+    } else if (lane == 0) {
+        sm_key[warp] = ~0ull;
+        sm_slot[warp] = -1;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long bk = ~0ull;
+        int bs = -1;
+        for (int w = 0; w < kThreads / 32; ++w)
+            if (sm_key[w] < bk) { bk = sm_key[w]; bs = sm_slot[w]; }
+        p.best_key[blockIdx.x] = bk;
+        p.best_slot[blockIdx.x] = bs;
+        sm_last = (arrive_acq_rel(p.arrive + unit) == active - 1);
+    }
+    __syncthreads();
+    if (!sm_last || warp != 0) return;
+    // the head's victim among the pieces' candidates: lanes take every 32nd piece, then the warp reduces
+    unsigned long long bk = ~0ull;
+    int bs = -1;
+    if (evict) {
+        const int64_t first = (int64_t)blockIdx.x - piece;
+        for (int c = lane; c < active; c += 32) {
+            const unsigned long long kc = __ldcg(p.best_key + first + c);
+            const int sc = __ldcg(p.best_slot + first + c);
+            if (kc < bk) { bk = kc; bs = sc; }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const unsigned long long ok = __shfl_xor_sync(0xffffffffu, bk, off);
+            const int os = __shfl_xor_sync(0xffffffffu, bs, off);
+            if (ok < bk) { bk = ok; bs = os; }
+        }
+    }
+    if (lane == 0) {
+        if (appended) {
+            if (evict && bs >= 0) {
+                p.free_slot[u.st] = bs;                     // len stays n: one row in, one row out (Eq. 5-6)
+            } else {
+                if (evict) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);   // capacity too small for sinks + window
+                p.len[u.st] = n + 1;
+                p.free_slot[u.st] = n + 1;
+            }
+        }
+        p.arrive[unit] = 0;
+    }
 }
 
 // ---------------------------------------------------------------- host side
@@ -1147,13 +1206,13 @@ int decode_attn_impl(
         if (ptr && !baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
     if (cache->seq_stride_tokens % 16 != 0) return BAKLAVA_ERR_INVALID_ARG;   // rows of pos / score go in 16-byte vectors
     if (info->layer_begin < 0 || info->layer_end > shape->L || info->layer_begin >= info->layer_end ||
-        info->B != cache->B || info->n_items <= 0 || info->n_score_items != 0 ||
+        info->B != cache->B || info->n_items <= 0 || info->n_score_items < 0 ||
         info->n_units != (info->layer_end - info->layer_begin) * cache->B * shape->Hkv)
         return BAKLAVA_ERR_INVALID_ARG;
     const int64_t rows = (int64_t)cache->B * cache->seq_stride_tokens;
     if (rows > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
     DecodeWorkspace lay;
-    const size_t need = baklava_decode_ws_bytes(shape, info->n_items, info->n_units, cache->B,
+    const size_t need = baklava_decode_ws_bytes(shape, info->n_items, info->n_score_items, info->n_units, cache->B,
                                                 cache->seq_stride_tokens, &lay);
     if (ws_bytes < need) return BAKLAVA_ERR_WORKSPACE;
 
@@ -1203,6 +1262,12 @@ int decode_attn_impl(
     p.arrive = reinterpret_cast<int32_t*>(base + lay.arrive_off);
     p.partial = reinterpret_cast<float*>(base + lay.partial_off);
     p.logit = reinterpret_cast<float*>(base + lay.logit_off);
+    p.stats = reinterpret_cast<float*>(base + lay.stats_off);
+    p.best_key = reinterpret_cast<unsigned long long*>(base + lay.best_off);
+    p.best_slot = reinterpret_cast<int32_t*>(base + lay.best_off + 8 * (size_t)info->n_score_items);
+    // A short launch that may not overlap what follows it ends in a kernel of its own for the score update
+    // (the plan lists its pieces); otherwise the CTA that finishes a head does it all.
+    p.split_tail = info->n_score_items > 0 && !(p.flags & (BAKLAVA_FLAG_NO_SCORE | BAKLAVA_FLAG_OVERLAP_PREV));
     p.scale_log2 = kLog2e / sqrtf((float)shape->D);
     p.kv_scale = cache->kv_scale;
     p.wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
@@ -1213,6 +1278,18 @@ int decode_attn_impl(
     else if (p.window_evict) err = shape->D == 128 ? launch_chunks<128, true>(p, k_map, v_map, s) : launch_chunks<64, true>(p, k_map, v_map, s);
     else err = shape->D == 128 ? launch_chunks<128, false>(p, k_map, v_map, s) : launch_chunks<64, false>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    if (p.split_tail) {
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)info->n_score_items);
+        cfg.blockDim = dim3(kThreads);
+        cfg.stream = s;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, sweep_kernel, p) != cudaSuccess) return BAKLAVA_ERR_CUDA;
+    }
     if (cudaGetLastError() != cudaSuccess) return BAKLAVA_ERR_CUDA;
     return BAKLAVA_OK;
 }

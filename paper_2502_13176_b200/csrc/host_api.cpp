@@ -160,7 +160,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_allocate(const bak
 }
 
 // ---------------------------------------------------------------- decode work plan
-size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_units, int32_t B,
+size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t n_score_items, int64_t n_units, int32_t B,
                                int64_t seq_stride_tokens, DecodeWorkspace* lay) {
     const int g = s->Hq / s->Hkv;
     DecodeWorkspace w;
@@ -168,6 +168,8 @@ size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t 
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 255) / 256 * 256; return at; };
     w.control_off = take(sizeof(int32_t) * 64);
     w.arrive_off = take(sizeof(int32_t) * (size_t)n_units);
+    w.stats_off = take(sizeof(float) * (size_t)n_units * 2 * BAKLAVA_MAX_GROUP);
+    w.best_off = take(16 * (size_t)n_score_items);
     w.partial_off = take(sizeof(float) * (size_t)n_items * partial_floats(g, s->D));
     w.logit_off = take(sizeof(float) * (size_t)B * (size_t)seq_stride_tokens * g);
     w.total = off;
@@ -261,18 +263,26 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
         }
         return BAKLAVA_OK;
     };
-    int64_t n_items = 0;
+    int64_t n_items = 0, n_score = 0;
     rc = emit(target, guided, &n_items);
     if (rc) return rc;
     if (n_items > INT32_MAX) return BAKLAVA_ERR_UNSUPPORTED;
+    // A launch whose chunks are all resident at once ends with its few longest heads; the plan then also lists
+    // pieces of the heads for a score / eviction pass that runs as a kernel of its own (about two per SM).
+    const bool short_launch = n_sm > 0 && n_items <= (int64_t)n_sm * kCtasPerSm;
+    if (short_launch) {
+        const int64_t len = std::min<int64_t>(kScoreChunk, std::max<int64_t>(kMinChunk, (tokens / (2 * (int64_t)n_sm) + kTile - 1) / kTile * kTile));
+        rc = emit(len, false, &n_score);
+        if (rc) return rc;
+    }
     info->n_items = (int32_t)n_items;
-    info->n_score_items = 0;
+    info->n_score_items = (int32_t)n_score;
     info->n_units = layers * B * Hkv;
     info->chunk_tokens = (int32_t)target;
     info->layer_begin = layer_begin;
     info->layer_end = layer_end;
     info->B = B;
-    info->ws_bytes = (int64_t)baklava_decode_ws_bytes(shape, n_items, info->n_units, B, seq_stride_tokens, nullptr);
+    info->ws_bytes = (int64_t)baklava_decode_ws_bytes(shape, n_items, n_score, info->n_units, B, seq_stride_tokens, nullptr);
     return BAKLAVA_OK;
 }
 

@@ -70,12 +70,13 @@ class DecodeSession:
                                       self.plan, self.ws)
         return self.out
 
-    def per_layer_plans(self):
+    def per_layer_plans(self, chunk_tokens=0):
         """One plan and workspace per layer, for callers that run attention layer by layer (as a model does)."""
         n_sm = torch.cuda.get_device_properties(self.device).multi_processor_count
         self.layer_plans = []
         for l in range(self.lb, self.le):
-            plan = bk.baklava_decode_plan(self.shape, self.cap, self.w.B, l, l + 1, self.stride, n_sm=n_sm).to(self.device)
+            plan = bk.baklava_decode_plan(self.shape, self.cap, self.w.B, l, l + 1, self.stride, chunk_tokens=chunk_tokens,
+                                          n_sm=n_sm).to(self.device)
             self.layer_plans.append((plan, bk.decode_workspace(plan, self.device)))
 
     def step_layers(self, q, k_new, v_new, t_pos, flags=0, overlap=True):
