@@ -328,19 +328,35 @@ def run_prefill_scores(args):
     k = synth.normal_bf16(w.seed, wl.T_PROFILE_K, (B, w.Hkv, T, w.D), dev)
     score = torch.empty((B, w.Hkv, T), dtype=torch.float32, device=dev)
     ws = torch.empty((bk.baklava_prefill_workspace_size(shape, B, T),), dtype=torch.uint8, device=dev)
-    ms, clocks = timed_calls(dev, lambda: bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws),
+    lse = None
+    if args.lse_given:
+        # the rows' natural-log normaliser as a prefill attention kernel would leave it (set-up, not timed):
+        # plain torch, a block of query rows at a time
+        lse = torch.empty((B, w.Hq, T), dtype=torch.float32, device=dev)
+        cols = torch.arange(T, device=dev)
+        for b in range(B):
+            for h in range(w.Hq):
+                for r0 in range(0, T, 4096):
+                    sc = (q[b, h, r0:r0 + 4096].float() @ k[b, h // w.g].float().T) / w.D ** 0.5
+                    sc.masked_fill_(cols[None, :] > torch.arange(r0, min(T, r0 + 4096), device=dev)[:, None], float("-inf"))
+                    lse[b, h, r0:r0 + 4096] = torch.logsumexp(sc, dim=1)
+        del sc
+    ms, clocks = timed_calls(dev, lambda: bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws, lse=lse),
                              args.steps, args.warmup)
     assert bk.workspace_error(ws) == 0
-    flop = 2 * B * w.Hq * 1.0 * T * T * w.D           # Q K^T under the causal mask, twice
+    passes = 1 if args.lse_given else 2
+    flop = passes * B * w.Hq * 1.0 * T * T * w.D      # Q K^T under the causal mask, once per pass
     line = tensor_line("prompt-score seeding TFLOP/s (one layer)", "prefill-scores-llama3-8b",
-                       {"batch": B, "prompt_tokens": T}, "qk_pass_kernel", flop, ms, clocks, args, 2)
+                       {"batch": B, "prompt_tokens": T, "passes": passes,
+                        "lse": "given by the caller" if args.lse_given else "computed by the first pass"},
+                       "qk_pass_kernel", flop, ms, clocks, args, passes)
     host = [t.cpu().pin_memory() for t in (q, k)]
     back = torch.empty(score.shape, dtype=score.dtype).pin_memory()
 
     def e2e():
         for d, h in zip((q, k), host):
             d.copy_(h, non_blocking=True)
-        bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws)
+        bk.baklava_prefill_scores(shape, q, k, None, B, T, score, ws, lse=lse)
         back.copy_(score, non_blocking=True)
     e2e_ms, _ = timed_calls(dev, e2e, max(1, args.steps // 4), 1)
     line["e2e"] = {"value": flop / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
@@ -380,6 +396,8 @@ def main():
     ap.add_argument("--per-layer", default="off", choices=["off", "calls", "graph"],
                     help="one baklava_decode_attn_varlen call per layer instead of one call over all layers: "
                          "issued one by one (calls) or captured once in a CUDA graph and replayed (graph)")
+    ap.add_argument("--lse-given", action="store_true",
+                    help="prefill workload: hand the rows' log-sum-exp to baklava_prefill_scores (one pass instead of two)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="with --per-layer: do not let a layer's call start beside the previous layer's tail")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -328,10 +328,14 @@ int baklava_evict_varlen(const baklava_shape* shape, const baklava_cache* cache,
  *   q           device bf16 [B, Hq, T, D]
  *   k           device bf16 [B, Hkv, T, D]
  *   prompt_len  device int32 [B] (rows and keys at or past len count for nothing) or NULL for len = T
+ *   lse         device fp32 [B, Hq, T] or NULL: the natural-log normaliser of every causal row i,
+ *               log sum_{j <= i} exp(q_i . k_j / sqrt(D)), as the attention kernel that processed the
+ *               prompt leaves it (rows at or past prompt_len are not read).  With it the call makes one
+ *               pass over Q K^T instead of two; the result is the same up to the rounding of lse.
  *   score       device fp32 [B, Hkv, T], overwritten
  *   ws          device workspace >= baklava_prefill_workspace_size() bytes */
 int baklava_prefill_scores(const baklava_shape* shape, const void* q, const void* k,
-                           const int32_t* prompt_len, int32_t B, int32_t T,
+                           const int32_t* prompt_len, const float* lse, int32_t B, int32_t T,
                            float* score, void* ws, size_t ws_bytes, void* stream);
 size_t baklava_prefill_workspace_size(const baklava_shape* shape, int32_t B, int32_t T);
 

@@ -88,7 +88,7 @@ def lib():
                                            c_void_p, c_int32, c_int64, c_int64, c_int64, c_int32, c_void_p]
         L.baklava_profile_heads.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                             c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
-        L.baklava_prefill_scores.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_int32, c_int32,
+        L.baklava_prefill_scores.argtypes = [POINTER(Shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
                                              c_void_p, c_void_p, c_size_t, c_void_p]
         L.baklava_prefill_workspace_size.restype = c_size_t
         L.baklava_prefill_workspace_size.argtypes = [POINTER(Shape), c_int32, c_int32]
@@ -305,8 +305,8 @@ def baklava_prefill_workspace_size(shape, B, T):
     return int(lib().baklava_prefill_workspace_size(ctypes.byref(shape), B, T))
 
 
-def baklava_prefill_scores(shape, q, k, prompt_len, B, T, score, ws, stream=None):
-    _check(lib().baklava_prefill_scores(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(prompt_len), B, T, _ptr(score),
+def baklava_prefill_scores(shape, q, k, prompt_len, B, T, score, ws, stream=None, lse=None):
+    _check(lib().baklava_prefill_scores(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(prompt_len), _ptr(lse), B, T, _ptr(score),
                                         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
            "baklava_prefill_scores")
 

@@ -2,7 +2,8 @@
 // processed, i.e. the column sums of the causal attention matrix of Eq. 1, added over the g query heads
 // that share a KV head.
 //
-// Two passes over Q K^T (V is not needed), both on the 5th-generation tensor cores.  A CTA keeps one
+// Two passes over Q K^T (V is not needed; one pass when the caller brings the rows' log-sum-exp), both on the
+// 5th-generation tensor cores.  A CTA keeps one
 // 128-row operand tile resident in shared memory and streams the other operand's tiles through a
 // two-stage TMA ring; one thread issues tcgen05.mma into a double-buffered 128 x 128 fp32 accumulator in
 // tensor memory; eight epilogue warps read it back with tcgen05.ld, one accumulator row per pair of threads.
@@ -38,6 +39,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 struct PrefillParams {
     const int32_t* prompt_len;   // [B] or null
     float* lse2;                 // [B, Hq, T] log2-domain log-sum-exp of every query row (+inf past the prompt)
+    const float* lse_nat;        // caller's natural-log log-sum-exp [B, Hq, T] (then lse2 is not used), or null
     float* score;                // [B, Hkv, T]
     uint32_t* error;
     int32_t B, T, Hq, Hkv, n_blk;
@@ -168,6 +170,8 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
         float m_run = -INFINITY, l_run = 0.0f, colsum = 0.0f;
         auto fetch_lse = [&](int it) -> float {              // the log-sum-exp of streamed query row e of tile it
             const int t = stream_blk(it) * kTileRows + e;
+            if (p.lse_nat)                                   // the caller's own (natural logarithm; rows past the prompt: none)
+                return t < len ? p.lse_nat[(int64_t)stream_head(it) * p.T + t] * kLog2e : INFINITY;
             return t < p.T ? p.lse2[(int64_t)stream_head(it) * p.T + t] : INFINITY;
         };
         if (PASS == kPassColumnSums) {
@@ -332,8 +336,10 @@ cudaError_t launch_pass(const PrefillParams& p, const CUtensorMap& qm, const CUt
 
 template <int D>
 cudaError_t launch_prefill(const PrefillParams& p, const CUtensorMap& qm, const CUtensorMap& km, cudaStream_t s) {
-    cudaError_t e = launch_pass<D, kPassLse>(p, qm, km, dim3(p.n_blk, p.Hq, p.B), s);
-    if (e != cudaSuccess) return e;
+    if (!p.lse_nat) {                                       // the rows' log-sum-exp first, unless the caller has it
+        cudaError_t e = launch_pass<D, kPassLse>(p, qm, km, dim3(p.n_blk, p.Hq, p.B), s);
+        if (e != cudaSuccess) return e;
+    }
     return launch_pass<D, kPassColumnSums>(p, qm, km, dim3(p.n_blk, p.Hkv, p.B), s);
 }
 
@@ -349,6 +355,7 @@ int baklava_launch_row_max(const baklava_shape* shape, const void* q, const void
     p.prompt_len = prompt_len;
     p.error = error;
     p.lse2 = lse2;
+    p.lse_nat = nullptr;
     p.score = nullptr;
     p.B = B; p.T = T; p.Hq = shape->Hq; p.Hkv = shape->Hkv;
     p.n_blk = (T + kTileRows - 1) / kTileRows;
@@ -377,14 +384,15 @@ extern "C" __attribute__((visibility("default"))) size_t baklava_prefill_workspa
 }
 
 extern "C" __attribute__((visibility("default"))) int baklava_prefill_scores(
-        const baklava_shape* shape, const void* q, const void* k, const int32_t* prompt_len, int32_t B, int32_t T,
-        float* score, void* ws, size_t ws_bytes, void* stream) {
+        const baklava_shape* shape, const void* q, const void* k, const int32_t* prompt_len, const float* lse,
+        int32_t B, int32_t T, float* score, void* ws, size_t ws_bytes, void* stream) {
     int rc = baklava_check_shape(shape);
     if (rc) return rc;
     if (!q || !k || !score || !ws || B <= 0 || T <= 0) return BAKLAVA_ERR_INVALID_ARG;
     const void* ptrs[] = {q, k, ws};
     for (const void* ptr : ptrs)
         if (!baklava_aligned16(ptr)) return BAKLAVA_ERR_INVALID_ARG;
+    if (lse && (reinterpret_cast<uintptr_t>(lse) & 3u)) return BAKLAVA_ERR_INVALID_ARG;
     if (B > 65535 || shape->Hq > 65535) return BAKLAVA_ERR_UNSUPPORTED;
     if (ws_bytes < baklava_prefill_workspace_size(shape, B, T)) return BAKLAVA_ERR_WORKSPACE;
 
@@ -392,6 +400,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_prefill_scores(
     p.prompt_len = prompt_len;
     p.error = static_cast<uint32_t*>(ws);
     p.lse2 = reinterpret_cast<float*>(static_cast<char*>(ws) + 256);
+    p.lse_nat = lse;
     p.score = score;
     p.B = B; p.T = T; p.Hq = shape->Hq; p.Hkv = shape->Hkv;
     p.n_blk = (T + kTileRows - 1) / kTileRows;

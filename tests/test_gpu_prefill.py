@@ -55,6 +55,40 @@ def test_group_of_seven():
     _run(B=1, Hq=7, Hkv=1, T=150, D=128)
 
 
+def test_with_the_rows_normaliser_supplied_one_pass_gives_the_same_scores():
+    """The caller's log-sum-exp (here the oracle's own, rounded to fp32) replaces the first pass."""
+    from oracle.attention import log_sum_exp
+    dev = "cuda"
+    B, Hq, Hkv, T, D = 2, 8, 2, 333, 128
+    lens = [333, 140]
+    shape = bk.make_shape(1, Hq, Hkv, D)
+    g = Hq // Hkv
+    q = synth.normal_bf16(11, 1, (B, Hq, T, D), dev, torch.tensor(2.0))
+    k = synth.normal_bf16(11, 2, (B, Hkv, T, D), dev)
+    Q, K = f64(q), f64(k)
+    lse = np.full((B, Hq, T), np.nan, dtype=np.float32)            # rows past the prompt must never be read
+    for b in range(B):
+        for h in range(Hq):
+            for i in range(lens[b]):
+                lse[b, h, i] = log_sum_exp(Q[b, h, i:i + 1], K[b, h // g, :i + 1])[0]
+    plen = torch.tensor(lens, dtype=torch.int32, device=dev)
+    ws = torch.empty((bk.baklava_prefill_workspace_size(shape, B, T),), dtype=torch.uint8, device=dev)
+    got = []
+    for given in (torch.from_numpy(lse).to(dev), None):
+        score = torch.full((B, Hkv, T), -1.0, dtype=torch.float32, device=dev)
+        bk.baklava_prefill_scores(shape, q, k, plen, B, T, score, ws, lse=given)
+        torch.cuda.synchronize()
+        assert bk.workspace_error(ws) == 0
+        got.append(score.cpu().numpy())
+    for b in range(B):
+        n = lens[b]
+        for c in range(Hkv):
+            ref = prefill_scores(Q[b, c * g:(c + 1) * g, :n], K[b, c, :n])
+            assert_close(got[0][b, c, :n], ref, "one pass, scores b%d kv%d" % (b, c))
+            assert np.all(got[0][b, c, n:] == 0.0)
+    np.testing.assert_allclose(got[0], got[1], rtol=2e-3, atol=1e-5)
+
+
 def test_seeds_a_bulk_eviction_like_the_oracle():
     dev = "cuda"
     B, Hq, Hkv, T, D = 1, 4, 2, 400, 64
