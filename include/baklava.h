@@ -75,7 +75,7 @@ extern "C" {
 #define BAKLAVA_FLAG_OVERLAP_PREV   8u   /* this call may start while the work in front of it on the   */
                                         /*   stream is still finishing (see baklava_decode_attn)      */
 #define BAKLAVA_FLAG_TEST_STALL  256u   /* test aid, never set it in production: the first chunk of   */
-                                        /*   every head is fed its first 64 (FP8: 128) rows only, so    */
+                                        /*   every head is fed its first 64 rows only, so               */
                                         /*   that the bounded wait for the next ones runs out and the   */
                                         /*   time-out path runs (use with a short baklava_set_wait_limit) */
 

@@ -13,13 +13,14 @@ constexpr int kScoreChunk = 2048;   // longest piece of the score / eviction pas
 #ifdef __CUDACC__
 __host__ __device__
 #endif
-constexpr int max_merge_entries(int D) { return 64 * D; }
+constexpr int max_merge_entries(int D) { return 48 * D; }
 
 // Byte offsets of the regions of the decode workspace.
 struct DecodeWorkspace {
     size_t control_off;    // 64 int32: launch-wide counters
     size_t arrive_off;     // int32 [n_units]: chunks of a head that have delivered their partial result
-    size_t stats_off;      // fp32 [n_units][2 * 8]: final (max, 1 / sum) of each query head, log2 domain (split tail)
+    size_t stats_off;      // fp32 [n_units][2 * 8 + 4]: final (max, 1 / sum) of each query head, log2 domain, and where the
+                           //   head's partials are (split tail)
     size_t best_off;       // uint64 [n_score_items] + int32 [n_score_items]: each score piece's eviction candidate
     size_t partial_off;    // fp32 [n_items][g * D + 2 * g + 2]: per-chunk (o, m, l) and its oldest evictable row (pos, slot)
     size_t logit_off;      // per head: fp16 [g][C] unnormalised probabilities of this step and fp32 [g][C / 16] reference

@@ -40,9 +40,16 @@ constexpr int kConsumerWarps = 4;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;     // + one producer warp
 constexpr int kTileTokens = kTile;                      // 64 tokens per stage
 constexpr int kWarpTokens = kTileTokens / kConsumerWarps;
-constexpr int kStages = 2;                              // 64 KB per CTA, three CTAs per SM
+constexpr int kStages = 2;                              // bf16 slabs: two 32 KB stages, 64 KB per CTA, three CTAs per SM
+// FP8 slabs: 128-token stages of the same 32 KB (64-token stages, three of them and four CTAs per SM were
+// measured slower: 151 us against 137 us per step on the Llama-shaped workload)
+constexpr int kFp8StageTokens = 128;
+constexpr int kFp8Stages = 2;
+constexpr int kFp8CtasPerSm = 3;
+constexpr int kMaxStages = 4;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kStatsStride = 2 * BAKLAVA_MAX_GROUP + 4;   // per head: final max [8], 1 / sum [8], first item, chunks
 static_assert(kWarpTokens == 16, "a consumer warp owns one 16-token MMA block of each tile");
 
 struct DecodeParams {
@@ -73,7 +80,8 @@ struct DecodeParams {
     int32_t* arrive;               // [n_units]: chunks of a head that have delivered their partial
     float* partial;
     float* logit;
-    float* stats;                  // [n_units][2 * kG]: final (max, 1 / sum) of every query head (split tail only)
+    float* stats;                  // [n_units][kStatsStride]: final (max, 1 / sum) of every query head, the head's first
+                                   //   item and its number of chunks (split tail only)
     unsigned long long* best_key;  // [n_score_items]: each piece's eviction candidate (split tail only)
     int32_t* best_slot;            // [n_score_items]
     float scale_log2;   // log2(e) / sqrt(D)
@@ -398,7 +406,7 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
     t.len = p.len + u.st;
     t.free_slot = p.free_slot + u.st;
     t.status = p.status;
-    t.stats = p.stats + (int64_t)unit * 2 * BAKLAVA_MAX_GROUP;
+    t.stats = p.stats + (int64_t)unit * kStatsStride;
     t.active = active; t.G = p.G; t.C = hs.C; t.n = hs.n; t.n_hi = hs.n_att; t.hole = hs.hole; t.n_sink = p.n_sink;
     // rows with a later position are in the recent window
     t.newest_candidate = t_pos - max(0, (int)(((int64_t)(hs.C - 1 - p.n_sink) * p.recent_num) / p.recent_den));
@@ -463,6 +471,16 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
         }
     }
     __syncthreads();
+    if (t.split) {
+        // steps 3-4 follow as a kernel of their own, whose pieces also merge the partial outputs (a share of the
+        // output columns each): it is told where the head's partials are
+        if (tid == 0) {
+            reinterpret_cast<int32_t*>(t.stats)[2 * kG] = (int32_t)(part0 - pp->partial) / psz;
+            reinterpret_cast<int32_t*>(t.stats)[2 * kG + 1] = t.active;
+            *t.arrive = 0;
+        }
+        return;
+    }
     for (int i = tid; i < n_ml; i += kThreads) {            // each chunk's weight in the merged output
         const int a = i % G;
         const float mc = sm_mc[i];
@@ -510,12 +528,6 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
         packed.x = *reinterpret_cast<const uint32_t*>(&lo);
         packed.y = *reinterpret_cast<const uint32_t*>(&hi);
         *reinterpret_cast<uint2*>(t.out + grp * 4) = packed;
-    }
-
-    if (t.split) {                                          // steps 3-4 follow as a kernel of their own
-        __syncthreads();
-        if (tid == 0) *t.arrive = 0;
-        return;
     }
 
     // ---- steps 3-4
@@ -577,22 +589,23 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
 // and become two fp16 pairs; V comes through ldmatrix.trans as two tokens x two adjacent channels per
 // register, which a byte permute splits into an even-channel and an odd-channel operand.
 template <int D, bool kByPosition, bool kFp8>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(const __grid_constant__ DecodeParams p,
+__global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) decode_chunk_kernel(const __grid_constant__ DecodeParams p,
                                                                 const __grid_constant__ CUtensorMap k_map,
                                                                 const __grid_constant__ CUtensorMap v_map) {
     constexpr int kKSteps = D / 16;                    // MMA k-steps over the head dimension
     constexpr int kNTiles = D / 8;                     // 8-wide output column blocks
-    constexpr int kTT = kFp8 ? 2 * kTileTokens : kTileTokens;       // tokens per stage
+    constexpr int kTT = kFp8 ? kFp8StageTokens : kTileTokens;       // tokens per stage
+    constexpr int kNS = kFp8 ? kFp8Stages : kStages;            // stages of the ring
     constexpr int kBlocks = kTT / (kConsumerWarps * kWarpTokens);    // 16-token blocks per warp and stage
-    static_assert(kFp8 || kBlocks == 1, "bf16 stages hold one 16-token block per warp");
+    static_assert(kBlocks >= 1 && kNS <= kMaxStages, "a stage holds at least one 16-token block per warp");
     constexpr int kRowBytes = kFp8 ? D : 2 * D;
     constexpr int kTileBytes = kTT * kRowBytes;        // one K (or V) tile
     constexpr int kStageBytes = 2 * kTileBytes;
     constexpr int kG = BAKLAVA_MAX_GROUP;
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_full[kStages];
-    __shared__ __align__(8) uint64_t bar_empty[kStages];
+    __shared__ __align__(8) uint64_t bar_full[kMaxStages];
+    __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
     __shared__ float sm_m[kConsumerWarps][kG];
     __shared__ float sm_l[kConsumerWarps][kG];
     __shared__ int sm_last;
@@ -611,7 +624,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
     const bool overlap = (p.flags & BAKLAVA_FLAG_OVERLAP_PREV) != 0;
     // what needs no memory of an earlier kernel comes first: the barriers and the tensor maps (kernel parameters)
     if (tid == kConsumerWarps * 32) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kNS; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_empty[s]), kConsumerWarps);
         }
@@ -687,12 +700,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
             const uint64_t stream_policy = l2_evict_first_policy();
             int it = 0;
             for (; it < n_tiles; ++it) {
-                const int s = it % kStages;
+                const int s = it % kNS;
                 // test aid (BAKLAVA_FLAG_TEST_STALL): the first chunk of a head gets its first tile only, so that
                 // the consumers' bounded wait for the second one runs out; nothing is in flight by then
                 if ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0 && it == 1) break;
-                if (it >= kStages) {
-                    if (!mbar_wait(smem_u32(&bar_empty[s]), ((it / kStages) - 1) & 1, p.wait_cycles)) {
+                if (it >= kNS) {
+                    if (!mbar_wait(smem_u32(&bar_empty[s]), ((it / kNS) - 1) & 1, p.wait_cycles)) {
                         atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
                         sm_abort = 1;
                         break;
@@ -741,8 +754,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         const int w0 = warp * kBlocks * kWarpTokens;       // this warp's rows inside a tile
         bool alive = true;
         for (int it = 0; it < n_tiles && alive; ++it) {
-            const int s = it % kStages;
-            if (!mbar_wait(smem_u32(&bar_full[s]), (it / kStages) & 1, p.wait_cycles)) {
+            const int s = it % kNS;
+            if (!mbar_wait(smem_u32(&bar_full[s]), (it / kNS) & 1, p.wait_cycles)) {
                 if (lane == 0) atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
                 alive = false;
                 break;
@@ -944,8 +957,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
         // left in flight when it exits (bounded wait for every tile that was requested), and the chunk still
         // arrives, with a mark, so that the head's counters return to zero and its bookkeeping is skipped.
         if (tid == 0)
-            for (int t = max(0, sm_issued - kStages); t < sm_issued; ++t)
-                mbar_wait(smem_u32(&bar_full[t % kStages]), (t / kStages) & 1, p.wait_cycles);
+            for (int t = max(0, sm_issued - kNS); t < sm_issued; ++t)
+                mbar_wait(smem_u32(&bar_full[t % kNS]), (t / kNS) & 1, p.wait_cycles);
         if (tid < G) part[G * D + tid] = __int_as_float(0x7fc00000);
     }
     if (!aborted) {
@@ -1022,9 +1035,10 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_chunk_kernel(cons
 
 // ---------------------------------------------------------------- steps 3-4 as a kernel of their own
 // A short launch (one layer of one sequence) ends with a few long heads, and one CTA sweeping a long head would
-// be most of the call's time.  There the attention kernel stops after the merged output and this kernel follows:
-// one CTA per piece of a head does the score update of its rows; the CTA that finishes a head last picks the
-// head's victim among the pieces' candidates and does the bookkeeping.
+// be most of the call's time.  There the attention kernel stops after the heads' final statistics and this
+// kernel follows: one CTA per piece of a head does the score update of its rows and merges its share of the
+// output columns; the CTA that finishes a head last picks the head's victim among the pieces' candidates and
+// does the bookkeeping.
 __global__ void __launch_bounds__(kThreads) sweep_kernel(const DecodeParams p) {
     constexpr int kG = BAKLAVA_MAX_GROUP;
     __shared__ float sm_M[kG];
@@ -1047,10 +1061,15 @@ __global__ void __launch_bounds__(kThreads) sweep_kernel(const DecodeParams p) {
     if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    const float* stats = p.stats + (int64_t)unit * kStatsStride;
     if (tid < G) {
-        sm_M[tid] = p.stats[(int64_t)unit * 2 * kG + tid];
-        sm_invL[tid] = p.stats[(int64_t)unit * 2 * kG + kG + tid];
+        sm_M[tid] = stats[tid];
+        sm_invL[tid] = stats[kG + tid];
     }
+    const int D = p.D;
+    const int psz = partial_floats(G, D);
+    const float* part0 = p.partial + (int64_t)reinterpret_cast<const int32_t*>(stats)[2 * kG] * psz;
+    const int n_chunks = reinterpret_cast<const int32_t*>(stats)[2 * kG + 1];
     __syncthreads();
     const bool lost = sm_M[0] != sm_M[0];                  // the attention kernel gave the head's step up
     const bool appended = hs.do_append && !lost;
@@ -1073,6 +1092,53 @@ __global__ void __launch_bounds__(kThreads) sweep_kernel(const DecodeParams p) {
     } else if (lane == 0) {
         sm_key[warp] = ~0ull;
         sm_slot[warp] = -1;
+    }
+    // ---- this piece's share of the output: column groups [lo, hi) of the g * D / 4 four-element groups, summed
+    // over the chunks.  Up to kMergeSplit threads share a group (each takes every P-th chunk, in ascending
+    // order) and the group's first thread adds their sums in thread order: the result does not depend on timing.
+    if (!lost) {
+        constexpr int kMergeSplit = 16;
+        __shared__ float4 sm_acc[kThreads];
+        const int n_grp = G * D / 4;
+        const int lo = (int)(((int64_t)piece * n_grp) / active), hi = (int)(((int64_t)(piece + 1) * n_grp) / active);
+        __nv_bfloat16* orow = p.out + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G) * D;
+        for (int g0 = lo; g0 < hi; g0 += kThreads) {
+            const int n_here = min(kThreads, hi - g0);
+            const int P = max(1, min(min(kMergeSplit, kThreads / n_here), n_chunks));
+            const int gl = tid / P, r = tid - gl * P;
+            const bool on = gl < n_here;
+            const int grp = g0 + gl;
+            const int a = on ? (grp * 4) / D : 0;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (on) {
+                const float Ma = sm_M[a];
+#pragma unroll 4
+                for (int c = r; c < n_chunks; c += P) {
+                    const float* pc = part0 + (int64_t)c * psz;
+                    const float mc = __ldcg(pc + G * D + a);
+                    const float4 oc = __ldcg(reinterpret_cast<const float4*>(pc) + grp);
+                    const float wgt = (mc == -INFINITY) ? 0.0f : exp2f(mc - Ma);
+                    acc.x = fmaf(oc.x, wgt, acc.x); acc.y = fmaf(oc.y, wgt, acc.y);
+                    acc.z = fmaf(oc.z, wgt, acc.z); acc.w = fmaf(oc.w, wgt, acc.w);
+                }
+            }
+            sm_acc[tid] = acc;
+            __syncthreads();
+            if (on && r == 0) {
+                for (int k = 1; k < P; ++k) {
+                    const float4 o2 = sm_acc[tid + k];
+                    acc.x += o2.x; acc.y += o2.y; acc.z += o2.z; acc.w += o2.w;
+                }
+                const float inv = sm_invL[a];
+                const __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+                const __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+                uint2 packed;
+                packed.x = *reinterpret_cast<const uint32_t*>(&lo2);
+                packed.y = *reinterpret_cast<const uint32_t*>(&hi2);
+                *reinterpret_cast<uint2*>(orow + grp * 4) = packed;
+            }
+            __syncthreads();
+        }
     }
     __syncthreads();
     if (tid == 0) {
@@ -1148,13 +1214,13 @@ bool make_slab_map(CUtensorMap* map, void* base, int64_t rows, int D) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// FP8 slabs: one byte per element, boxes of 128 rows x 128 bytes (the whole row), 128-byte swizzle
+// FP8 slabs: one byte per element, boxes of one stage's rows x 128 bytes (the whole row), 128-byte swizzle
 bool make_slab_map_fp8(CUtensorMap* map, void* base, int64_t rows, int D) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)D};
-    const cuuint32_t box[2] = {128, (cuuint32_t)(2 * kTileTokens)};
+    const cuuint32_t box[2] = {128, (cuuint32_t)kFp8StageTokens};
     const cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1163,7 +1229,7 @@ bool make_slab_map_fp8(CUtensorMap* map, void* base, int64_t rows, int D) {
 
 template <int D, bool kByPosition, bool kFp8 = false>
 cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
-    constexpr int kSmem = kStages * 2 * kTileTokens * D * 2 + 1024;      // the same 32 KB stages for both formats
+    constexpr int kSmem = (kFp8 ? kFp8Stages * 2 * kFp8StageTokens * D : kStages * 2 * kTileTokens * D * 2) + 1024;
     cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D, kByPosition, kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     cudaLaunchAttribute attr[1];

@@ -168,7 +168,7 @@ size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t 
     auto take = [&](size_t bytes) { size_t at = off; off += (bytes + 255) / 256 * 256; return at; };
     w.control_off = take(sizeof(int32_t) * 64);
     w.arrive_off = take(sizeof(int32_t) * (size_t)n_units);
-    w.stats_off = take(sizeof(float) * (size_t)n_units * 2 * BAKLAVA_MAX_GROUP);
+    w.stats_off = take(sizeof(float) * (size_t)n_units * (2 * BAKLAVA_MAX_GROUP + 4));
     w.best_off = take(16 * (size_t)n_score_items);
     w.partial_off = take(sizeof(float) * (size_t)n_items * partial_floats(g, s->D));
     w.logit_off = take(sizeof(float) * (size_t)B * (size_t)seq_stride_tokens * g);
