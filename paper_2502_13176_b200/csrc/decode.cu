@@ -20,6 +20,7 @@
 #include <climits>
 #include <cmath>
 #include <cstdint>
+#include <type_traits>
 
 #include "baklava.h"
 #include "common.h"
@@ -217,6 +218,12 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     uint32_t d;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
+}
+// 2^x on the special-function unit (one instruction; -inf gives 0, results below 2^-126 flush to 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     const __half2 v = __floats2half2_rn(lo, hi);
@@ -752,6 +759,14 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
         }
         const int lm = lane >> 3, li8 = lane & 7;          // ldmatrix: matrix index and row inside it
         const int w0 = warp * kBlocks * kWarpTokens;       // this warp's rows inside a tile
+        // This lane's row address inside a 16-token block for the two kinds of ldmatrix.  A tile is stored with
+        // the 128-byte swizzle (16-byte piece c of row r at position c ^ (r % 8)); with the piece index
+        // 2 c + b (b = one bit of the matrix index) that is a constant exclusive-or on a per-lane address:
+        //   offset(r, 2 c + b) = (c / 4) * 8192 + ((r * 128 + ((b ^ r % 8) << 4)) ^ ((2 c % 8) << 4))
+        const uint32_t k_lane = (uint32_t)(((lm >> 1) * 8 + li8) * 128 + ((li8 ^ (lm & 1)) << 4));   // K: rows (lm / 2) * 8 + .., b = lm % 2
+        const uint32_t v_lane = (uint32_t)(((lm & 1) * 8 + li8) * 128 + ((li8 ^ (lm >> 1)) << 4));   // V: rows (lm % 2) * 8 + .., b = lm / 2
+        // where this lane leaves the probabilities of head g8 (tokens 2 t4, 2 t4 + 1 of a block) for the score pass
+        __half* const prob_lane = prob_h + (int64_t)g8 * C + 2 * t4;
         bool alive = true;
         for (int it = 0; it < n_tiles && alive; ++it) {
             const int s = it % kNS;
@@ -763,69 +778,72 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
             const uint32_t k_tile = ring + s * kStageBytes;
             const uint32_t v_tile = k_tile + kTileBytes;
             const int wtok0 = begin + it * kTT + w0;                 // first token of this warp's share of the stage
-            if (wtok0 < end) {
+            constexpr int kWarpSpan = kBlocks * kWarpTokens;
+            // One body for the warp's tokens of the stage, compiled twice: the plain form for a span that lies
+            // inside the chunk and holds neither the slot to append to nor a freed slot (nearly always), and the
+            // careful form that patches the tile and masks rows.
+            auto stage_body = [&](auto careful_tag) {
+                constexpr bool kCareful = decltype(careful_tag)::value;
+                if (kCareful) {
 #pragma unroll
-                for (int blk = 0; blk < kBlocks; ++blk) {            // per 16-token block: patch the tile where needed
-                    const int r0 = w0 + blk * kWarpTokens;
-                    const int tok0 = wtok0 + blk * kWarpTokens;
-                    const int valid = max(0, min(kWarpTokens, end - tok0));   // rows of the block inside the chunk
-                    if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
-                        // step 1 (Eq. 4): the new token's row replaces whatever the tile holds at the free slot,
-                        // in shared memory for this pass and in the slab for the steps to come
-                        constexpr int kVec = D / 8;
-                        const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
-                        const int64_t row = row0 + hs.f;
-                        uint8_t* k_ptr = ring_ptr + s * kStageBytes;
-                        if (kFp8) {                          // quantise the row: eight elements per lane and operand
-                            for (int i = lane; i < 2 * kVec; i += 32) {
-                                const bool is_v = i >= kVec;
-                                const int c = is_v ? i - kVec : i;
-                                const uint4 raw = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
-                                const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + (is_v ? 3 : 1)]);
-                                *reinterpret_cast<uint2*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c >> 1) +
-                                                          (c & 1) * 8) = val;
-                                uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
-                                *(reinterpret_cast<uint2*>(slab + row * D) + c) = val;
+                    for (int blk = 0; blk < kBlocks; ++blk) {        // per 16-token block: patch the tile where needed
+                        const int r0 = w0 + blk * kWarpTokens;
+                        const int tok0 = wtok0 + blk * kWarpTokens;
+                        const int valid = max(0, min(kWarpTokens, end - tok0));   // rows of the block inside the chunk
+                        if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
+                            // step 1 (Eq. 4): the new token's row replaces whatever the tile holds at the free slot,
+                            // in shared memory for this pass and in the slab for the steps to come
+                            constexpr int kVec = D / 8;
+                            const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
+                            const int64_t row = row0 + hs.f;
+                            uint8_t* k_ptr = ring_ptr + s * kStageBytes;
+                            if (kFp8) {                      // quantise the row: eight elements per lane and operand
+                                for (int i = lane; i < 2 * kVec; i += 32) {
+                                    const bool is_v = i >= kVec;
+                                    const int c = is_v ? i - kVec : i;
+                                    const uint4 raw = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
+                                    const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + (is_v ? 3 : 1)]);
+                                    *reinterpret_cast<uint2*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c >> 1) +
+                                                              (c & 1) * 8) = val;
+                                    uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
+                                    *(reinterpret_cast<uint2*>(slab + row * D) + c) = val;
+                                }
+                            } else {
+                                for (int i = lane; i < 2 * kVec; i += 32) {
+                                    const bool is_v = i >= kVec;
+                                    const int c = is_v ? i - kVec : i;
+                                    const uint4 val = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
+                                    *reinterpret_cast<uint4*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c)) = val;
+                                    *(reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c) = val;
+                                }
                             }
-                        } else {
-                            for (int i = lane; i < 2 * kVec; i += 32) {
-                                const bool is_v = i >= kVec;
-                                const int c = is_v ? i - kVec : i;
-                                const uint4 val = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
-                                *reinterpret_cast<uint4*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(r0 + (hs.f - tok0), c)) = val;
-                                *(reinterpret_cast<uint4*>((is_v ? p.v_slab : p.k_slab) + row * D) + c) = val;
+                            if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
+                            __syncwarp();
+                        }
+                        // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
+                        if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
+                            uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
+                            constexpr int kPieces = kRowBytes / 16;     // 16-byte pieces of a row
+                            for (int i = lane; i < kWarpTokens * kPieces; i += 32) {
+                                const int r = i / kPieces, c = i % kPieces;
+                                if (r >= valid || tok0 + r == hole)
+                                    *reinterpret_cast<uint4*>(v_ptr + tile_offset(r0 + r, c)) = make_uint4(0, 0, 0, 0);
                             }
+                            __syncwarp();
                         }
-                        if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
-                        __syncwarp();
-                    }
-                    if (kByPosition && pos_evict && lane < valid && tok0 + lane != hs.f) {
-                        const int ps = p.pos[row0 + tok0 + lane];
-                        if (ps >= p.n_sink && ps <= window_from && ps < old_pos) { old_pos = ps; old_slot = tok0 + lane; }
-                    }
-                    // rows past the end of the head (or the freed slot) may hold anything: keep them out of P.V
-                    if (valid < kWarpTokens || (hole >= tok0 && hole < tok0 + kWarpTokens)) {
-                        uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
-                        constexpr int kPieces = kRowBytes / 16;     // 16-byte pieces of a row
-                        for (int i = lane; i < kWarpTokens * kPieces; i += 32) {
-                            const int r = i / kPieces, c = i % kPieces;
-                            if (r >= valid || tok0 + r == hole)
-                                *reinterpret_cast<uint4*>(v_ptr + tile_offset(r0 + r, c)) = make_uint4(0, 0, 0, 0);
-                        }
-                        __syncwarp();
                     }
                 }
-                // S^T = K Q^T for the warp's 16 * kBlocks tokens: st[blk] = (token g: heads 2 t, 2 t + 1; token g + 8: same)
+                // S^T = K Q^T for the warp's tokens: st[blk] = (token g: heads 2 t, 2 t + 1; token g + 8: the same)
                 float st[kBlocks][4];
 #pragma unroll
                 for (int blk = 0; blk < kBlocks; ++blk) {
                     st[blk][0] = st[blk][1] = st[blk][2] = st[blk][3] = 0.0f;
-                    const int r0 = w0 + blk * kWarpTokens;
+                    const uint32_t k_row = k_tile + (uint32_t)((w0 + blk * kWarpTokens) * 128) + k_lane;
                     if (kFp8) {
 #pragma unroll
                         for (int kk = 0; kk < D / 32; ++kk) {     // 32 channels per load: two steps of 16
                             uint32_t kb[4];      // (tokens 0-7 | 8-15) x (channels 0-15 | 16-31), four bytes per lane
-                            ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * kk + (lm & 1)), kb);
+                            ldmatrix_x4((k_row ^ (uint32_t)(((2 * kk) & 7) << 4)) + (kk >> 2) * 8192, kb);
 #pragma unroll
                             for (int c = 0; c < 2; ++c) {
                                 uint32_t a0, a2, a1, a3;
@@ -838,7 +856,7 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
 #pragma unroll
                         for (int ks = 0; ks < kKSteps; ++ks) {
                             uint32_t kb[4];      // (tokens 0-7 | 8-15) x (channels 0-7 | 8-15) of the step
-                            ldmatrix_x4(k_tile + tile_offset(r0 + (lm >> 1) * 8 + li8, 2 * ks + (lm & 1)), kb);
+                            ldmatrix_x4((k_row ^ (uint32_t)(((2 * ks) & 7) << 4)) + (ks >> 2) * 8192, kb);
                             mma_bf16_full(st[blk], kb[0], kb[2], kb[1], kb[3], q0[ks], q1[ks]);
                         }
                     }
@@ -851,7 +869,7 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
 #pragma unroll
                     for (int r = 0; r < 2; ++r) {
                         const int tok = wtok0 + blk * kWarpTokens + g8 + 8 * r;
-                        ok[blk][r] = tok < end && tok != hole;
+                        ok[blk][r] = !kCareful || (tok < end && tok != hole);
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             st[blk][2 * r + e] *= scale_k;
@@ -865,7 +883,7 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
                     mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 8));
                     mx[e] = fmaxf(mx[e], __shfl_xor_sync(0xffffffffu, mx[e], 16));
                     const float m_new = fmaxf(m_run[e], mx[e]);
-                    corr[e] = (m_new == -INFINITY) ? 1.0f : exp2f(m_run[e] - m_new);
+                    corr[e] = (m_new == -INFINITY) ? 1.0f : fast_exp2(m_run[e] - m_new);
                     m_run[e] = m_new;
                 }
                 float psum[2] = {0.0f, 0.0f};
@@ -875,7 +893,7 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
                     for (int r = 0; r < 2; ++r)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const float pv = ok[blk][r] ? exp2f(st[blk][2 * r + e] - m_run[e]) : 0.0f;
+                            const float pv = ok[blk][r] ? fast_exp2(st[blk][2 * r + e] - m_run[e]) : 0.0f;
                             st[blk][2 * r + e] = pv;
                             psum[e] += pv;
                         }
@@ -899,23 +917,30 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
                         pb[blk][0] = movmatrix_trans(pack_bf16(st[blk][0], st[blk][1]));
                         pb[blk][1] = movmatrix_trans(pack_bf16(st[blk][2], st[blk][3]));
                     }
-                    if (keep_logits && g8 < G && tok0 < end) {
+                    if (keep_logits) {
                         // the unnormalised probabilities of head g, in fp16, and the maximum they were taken under
-                        __half* dst = prob_h + (int64_t)g8 * C + tok0 + 2 * t4;
-                        if (tok0 + 2 * t4 + 1 < end) *reinterpret_cast<uint32_t*>(dst) = h0;
-                        else if (tok0 + 2 * t4 < end) dst[0] = __ushort_as_half((unsigned short)(h0 & 0xffffu));
-                        if (tok0 + 8 + 2 * t4 + 1 < end) *reinterpret_cast<uint32_t*>(dst + 8) = h1;
-                        else if (tok0 + 8 + 2 * t4 < end) dst[8] = __ushort_as_half((unsigned short)(h1 & 0xffffu));
-                    }
-                    if (keep_logits && g8 == 0 && tok0 < end) {
-                        if (2 * t4 < G) mref_h[(2 * t4) * (C >> 4) + (tok0 >> 4)] = m_run[0];
-                        if (2 * t4 + 1 < G) mref_h[(2 * t4 + 1) * (C >> 4) + (tok0 >> 4)] = m_run[1];
+                        __half* dst = prob_lane + tok0;
+                        if (!kCareful) {
+                            if (g8 < G) {
+                                *reinterpret_cast<uint32_t*>(dst) = h0;
+                                *reinterpret_cast<uint32_t*>(dst + 8) = h1;
+                            }
+                        } else if (g8 < G && tok0 < end) {
+                            if (tok0 + 2 * t4 + 1 < end) *reinterpret_cast<uint32_t*>(dst) = h0;
+                            else if (tok0 + 2 * t4 < end) dst[0] = __ushort_as_half((unsigned short)(h0 & 0xffffu));
+                            if (tok0 + 8 + 2 * t4 + 1 < end) *reinterpret_cast<uint32_t*>(dst + 8) = h1;
+                            else if (tok0 + 8 + 2 * t4 < end) dst[8] = __ushort_as_half((unsigned short)(h1 & 0xffffu));
+                        }
+                        if (g8 == 0 && (!kCareful || tok0 < end)) {
+                            if (2 * t4 < G) mref_h[(2 * t4) * (C >> 4) + (tok0 >> 4)] = m_run[0];
+                            if (2 * t4 + 1 < G) mref_h[(2 * t4 + 1) * (C >> 4) + (tok0 >> 4)] = m_run[1];
+                        }
                     }
                 }
                 // O^T += V^T P^T: V^T fragments through ldmatrix.trans
 #pragma unroll
                 for (int blk = 0; blk < kBlocks; ++blk) {
-                    const int r0 = w0 + blk * kWarpTokens;
+                    const uint32_t v_row = v_tile + (uint32_t)((w0 + blk * kWarpTokens) * 128) + v_lane;
                     if (kFp8) {
                         // a register of the transposed load = two tokens x two adjacent channels; the permute puts the
                         // even channel's token pair in the low half and the odd channel's in the high half.  Row g of
@@ -923,7 +948,7 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
 #pragma unroll
                         for (int c2 = 0; c2 < D / 32; ++c2) {
                             uint32_t vb[4];      // (tokens 0-7 | 8-15) x (channels 0-15 | 16-31)
-                            ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * c2 + (lm >> 1)), vb);
+                            ldmatrix_x4_trans((v_row ^ (uint32_t)(((2 * c2) & 7) << 4)) + (c2 >> 2) * 8192, vb);
 #pragma unroll
                             for (int h2 = 0; h2 < 2; ++h2) {
                                 const uint32_t lo = __byte_perm(vb[2 * h2], 0u, 0x3120), hi = __byte_perm(vb[2 * h2 + 1], 0u, 0x3120);
@@ -937,11 +962,25 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
 #pragma unroll
                         for (int c = 0; c < D / 16; ++c) {
                             uint32_t vb[4];      // (tokens 0-7 | 8-15) x (channels 0-7 | 8-15) of the group
-                            ldmatrix_x4_trans(v_tile + tile_offset(r0 + (lm & 1) * 8 + li8, 2 * c + (lm >> 1)), vb);
+                            ldmatrix_x4_trans((v_row ^ (uint32_t)(((2 * c) & 7) << 4)) + (c >> 2) * 8192, vb);
                             mma_bf16_full(o[c], vb[0], vb[2], vb[1], vb[3], pb[blk][0], pb[blk][1]);
                         }
                     }
                 }
+            };
+            if (wtok0 < end) {
+                if (kByPosition && pos_evict) {
+                    for (int tok = wtok0 + lane; tok < min(end, wtok0 + kWarpSpan); tok += 32) {
+                        if (tok == hs.f) continue;
+                        const int ps = p.pos[row0 + tok];
+                        if (ps >= p.n_sink && ps <= window_from && ps < old_pos) { old_pos = ps; old_slot = tok; }
+                    }
+                }
+                const bool inside = wtok0 + kWarpSpan <= end;
+                const bool has_hole = hole >= wtok0 && hole < wtok0 + kWarpSpan;
+                const bool has_slot = hs.do_append && hs.f >= wtok0 && hs.f < wtok0 + kWarpSpan;
+                if (inside && !has_hole && !has_slot) stage_body(std::false_type{});
+                else stage_body(std::true_type{});
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_empty[s]));
