@@ -740,7 +740,7 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
         // query fragments (B operand of S^T): head g of the group (zero from G on), per 16-channel step the
         // channels 2 t, 2 t + 1 (q0) and 8 + 2 t, 9 + 2 t (q1); for FP8 slabs the channels 4 t .. 4 t + 3, the order
         // in which the four bytes of a K register arrive (the contraction index may be permuted at will)
-        uint32_t q0[kKSteps], q1[kKSteps];
+        uint32_t qq[2 * kKSteps];                          // (q0, q1) of step ks side by side, as the MMA takes them
         {
             const __nv_bfloat16* q_ptr = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + g8) * D;
 #pragma unroll
@@ -749,11 +749,11 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
                     const uint2 raw = g8 < G ? *reinterpret_cast<const uint2*>(q_ptr + ks * 16 + 4 * t4) : make_uint2(0u, 0u);
                     const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
                     const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-                    q0[ks] = pack_f16(f0.x, f0.y);
-                    q1[ks] = pack_f16(f1.x, f1.y);
+                    qq[2 * ks] = pack_f16(f0.x, f0.y);
+                    qq[2 * ks + 1] = pack_f16(f1.x, f1.y);
                 } else {
-                    q0[ks] = g8 < G ? *reinterpret_cast<const uint32_t*>(q_ptr + ks * 16 + 2 * t4) : 0u;
-                    q1[ks] = g8 < G ? *reinterpret_cast<const uint32_t*>(q_ptr + ks * 16 + 8 + 2 * t4) : 0u;
+                    qq[2 * ks] = g8 < G ? *reinterpret_cast<const uint32_t*>(q_ptr + ks * 16 + 2 * t4) : 0u;
+                    qq[2 * ks + 1] = g8 < G ? *reinterpret_cast<const uint32_t*>(q_ptr + ks * 16 + 8 + 2 * t4) : 0u;
                 }
             }
         }
@@ -763,8 +763,14 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
         // the 128-byte swizzle (16-byte piece c of row r at position c ^ (r % 8)); with the piece index
         // 2 c + b (b = one bit of the matrix index) that is a constant exclusive-or on a per-lane address:
         //   offset(r, 2 c + b) = (c / 4) * 8192 + ((r * 128 + ((b ^ r % 8) << 4)) ^ ((2 c % 8) << 4))
-        const uint32_t k_lane = (uint32_t)(((lm >> 1) * 8 + li8) * 128 + ((li8 ^ (lm & 1)) << 4));   // K: rows (lm / 2) * 8 + .., b = lm % 2
-        const uint32_t v_lane = (uint32_t)(((lm & 1) * 8 + li8) * 128 + ((li8 ^ (lm >> 1)) << 4));   // V: rows (lm % 2) * 8 + .., b = lm / 2
+        // The four matrices of a load come out in the order of the MMA's A registers (a0 .. a3), so that no register
+        // has to be moved in between: for K (rows = tokens) matrix 1 is the second token half and matrix 2 the
+        // second channel half (bf16; for FP8 bytes the order of the conversions is free anyway), for the transposed
+        // V load (rows of the MMA = channels) it is the other way round.
+        const uint32_t k_lane = kFp8 ? (uint32_t)(((lm >> 1) * 8 + li8) * 128 + ((li8 ^ (lm & 1)) << 4))    // rows (lm / 2) * 8 + .., b = lm % 2
+                                     : (uint32_t)(((lm & 1) * 8 + li8) * 128 + ((li8 ^ (lm >> 1)) << 4));   // rows (lm % 2) * 8 + .., b = lm / 2
+        const uint32_t v_lane = kFp8 ? (uint32_t)(((lm & 1) * 8 + li8) * 128 + ((li8 ^ (lm >> 1)) << 4))
+                                     : (uint32_t)(((lm >> 1) * 8 + li8) * 128 + ((li8 ^ (lm & 1)) << 4));
         // where this lane leaves the probabilities of head g8 (tokens 2 t4, 2 t4 + 1 of a block) for the score pass
         __half* const prob_lane = prob_h + (int64_t)g8 * C + 2 * t4;
         bool alive = true;
@@ -849,15 +855,15 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
                                 uint32_t a0, a2, a1, a3;
                                 fp8::f16x4_from_e4m3x4(kb[c], a0, a2);
                                 fp8::f16x4_from_e4m3x4(kb[2 + c], a1, a3);
-                                mma_f16_full(st[blk], a0, a1, a2, a3, q0[2 * kk + c], q1[2 * kk + c]);
+                                mma_f16_full(st[blk], a0, a1, a2, a3, qq[2 * (2 * kk + c)], qq[2 * (2 * kk + c) + 1]);
                             }
                         }
                     } else {
 #pragma unroll
                         for (int ks = 0; ks < kKSteps; ++ks) {
-                            uint32_t kb[4];      // (tokens 0-7 | 8-15) x (channels 0-7 | 8-15) of the step
+                            uint32_t kb[4];      // channels 0-7 of the step: tokens 0-7, 8-15; channels 8-15: tokens 0-7, 8-15
                             ldmatrix_x4((k_row ^ (uint32_t)(((2 * ks) & 7) << 4)) + (ks >> 2) * 8192, kb);
-                            mma_bf16_full(st[blk], kb[0], kb[2], kb[1], kb[3], q0[ks], q1[ks]);
+                            mma_bf16_full(st[blk], kb[0], kb[1], kb[2], kb[3], qq[2 * ks], qq[2 * ks + 1]);
                         }
                     }
                 }
@@ -961,9 +967,9 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
                     } else {
 #pragma unroll
                         for (int c = 0; c < D / 16; ++c) {
-                            uint32_t vb[4];      // (tokens 0-7 | 8-15) x (channels 0-7 | 8-15) of the group
+                            uint32_t vb[4];      // tokens 0-7: channels 0-7, 8-15 of the group; tokens 8-15: channels 0-7, 8-15
                             ldmatrix_x4_trans((v_row ^ (uint32_t)(((2 * c) & 7) << 4)) + (c >> 2) * 8192, vb);
-                            mma_bf16_full(o[c], vb[0], vb[2], vb[1], vb[3], pb[blk][0], pb[blk][1]);
+                            mma_bf16_full(o[c], vb[0], vb[1], vb[2], vb[3], pb[blk][0], pb[blk][1]);
                         }
                     }
                 }
