@@ -454,7 +454,7 @@ def main():
         sess.prefill_synthetic()
     if args.per_layer != "off":
         # layer by layer, as a model calls attention; positions live on the device and advance there
-        sess.per_layer_plans(args.chunk)
+        sess.per_layer_plans(args.chunk, overlap=not args.no_overlap)
         t_dev = torch.full((w.B,), w.T, dtype=torch.int32, device=dev)
         sq, sk, sv = (torch.empty_like(t) for t in wl.decode_inputs(w, 0, sess.scales, dev))
 
@@ -584,7 +584,13 @@ def main():
             "data": "synthetic",
             "config": {"workload": w.name, "layers": w.L, "batch": w.B, "context": w.T, "budget": w.budget,
                        "kv_bytes_per_step": bytes_per_step, "l2": "inputs larger than L2 (no flush)",
-                       "launch": "one baklava_decode_attn%s call per step covering all layers" % (
+                       "launch": ("one baklava_decode_attn_varlen call per layer (%s), %s" % (
+                                      "CUDA graph replay" if args.per_layer == "graph" else "issued one by one",
+                                      "each waiting for the one before it" if args.no_overlap else
+                                      "layers after the first flagged BAKLAVA_FLAG_OVERLAP_PREV: every layer's inputs are "
+                                      "ready before the first call, so a layer streams beside the tails of those before it"))
+                       if args.per_layer != "off" else
+                       "one baklava_decode_attn%s call per step covering all layers" % (
                            "_varlen" if args.mixed_lengths else ""), "policy": args.policy,
                        "replicas": world},
             "tokens_per_s": whole_job_rate(world, w.B, args.steps, elapsed_ms),

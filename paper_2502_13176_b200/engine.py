@@ -70,8 +70,13 @@ class DecodeSession:
                                       self.plan, self.ws)
         return self.out
 
-    def per_layer_plans(self, chunk_tokens=0):
-        """One plan and workspace per layer, for callers that run attention layer by layer (as a model does)."""
+    def per_layer_plans(self, chunk_tokens=0, overlap=True):
+        """One plan and workspace per layer, for callers that run attention layer by layer (as a model does).
+        With `overlap` (the calls after the first will carry BAKLAVA_FLAG_OVERLAP_PREV) and no chunk length given,
+        chunks of 1024 tokens: consecutive layers' kernels then share the GPU, and what counts is the fixed cost
+        per chunk, not that one layer's chunks fill one wave."""
+        if overlap and chunk_tokens == 0:
+            chunk_tokens = 1024
         n_sm = torch.cuda.get_device_properties(self.device).multi_processor_count
         self.layer_plans = []
         for l in range(self.lb, self.le):
