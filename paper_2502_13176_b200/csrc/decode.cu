@@ -1094,18 +1094,22 @@ __global__ void __launch_bounds__(kThreads) sweep_kernel(const DecodeParams p) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.G;
     launch_dependents();                                  // what follows waits for this grid by itself
-    grid_dependency_wait();                               // the attention kernel: statistics, scratch, appended rows
+    // The piece and the head's state are read while the attention kernel is still running: that kernel (never an
+    // overlapping call here) released this one only after its own dependency wait, so the previous step's
+    // bookkeeping is complete, and it leaves len / free_slot alone when this kernel follows.
     const int4 item = p.items[p.n_items + blockIdx.x];
     const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
     const Unit u = decode_unit(p, unit);
     const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
-    const HeadState hs = head_state(p, u);                // unchanged so far: this kernel does the bookkeeping
-    if (hs.bad || t_pos < 0) return;                      // reported by the attention kernel / idle sequence
+    const HeadState hs = head_state(p, u);
     const int C = hs.C, n = hs.n, n_hi = hs.n_att;
     const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
-    if (piece >= active) return;
     const int end = min(begin + chunk_len, n_hi);
     const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    if (tid == 0 || !(hs.bad || t_pos < 0 || piece >= active))
+        grid_dependency_wait();                           // the attention kernel: statistics, scratch, partials, appended rows
+    if (hs.bad || t_pos < 0) return;                      // reported by the attention kernel / idle sequence
+    if (piece >= active) return;
     const float* stats = p.stats + (int64_t)unit * kStatsStride;
     if (tid < G) {
         sm_M[tid] = stats[tid];

@@ -60,6 +60,17 @@ def test_one_call_per_layer_overlapping_the_previous_layers_tail(chunk):
     s = Session(w, chunk_tokens=chunk, per_layer=True)
     for i in range(w.steps):
         s.step(i)
+    w = wl.scaled(wl.LLAMA3_8B_32K, L=3, T=1800, steps=4)             # FP8 slabs through the same layer loop
+    s = Session(w, chunk_tokens=chunk, per_layer=True, kv_dtype=bk.KV_FP8_E4M3)
+    for i in range(w.steps):
+        s.step(i)
+
+
+def test_window_policy_one_call_per_layer():
+    w = wl.scaled(wl.LLAMA3_8B_32K, L=3, T=900, steps=12, recent_num=1, recent_den=1)
+    s = Session(w, chunk_tokens=128, per_layer=True)
+    for i in range(w.steps):
+        s.step(i, flags=bk.FLAG_NO_SCORE)
 
 
 def test_one_call_per_layer_leaves_the_same_cache_as_one_call_for_all_layers():

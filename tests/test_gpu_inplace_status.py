@@ -201,11 +201,14 @@ def test_capacity_too_small_for_sinks_and_window_is_reported():
     assert int(s.cache.status.item()) == bk.STATUS_OVERFLOW
 
 
+@pytest.mark.parametrize("one_kernel", [False, True], ids=["two-kernels", "one-kernel"])
 @pytest.mark.parametrize("kv", [bk.KV_BF16, bk.KV_FP8_E4M3], ids=["bf16", "fp8"])
-def test_wait_that_runs_out_sets_timeout_and_leaves_everything_usable(kv):
+def test_wait_that_runs_out_sets_timeout_and_leaves_everything_usable(kv, one_kernel):
     """The first chunk of every head is fed one tile only (test flag), so the consumers' bounded wait for the
     second tile runs out after a short limit: TIMEOUT is set, no head changes, and the next step on the same
-    workspace is an ordinary, correct step."""
+    workspace is an ordinary, correct step.  A launch this short ends in a second kernel for the score update;
+    with BAKLAVA_FLAG_OVERLAP_PREV (nothing is in flight here, so the flag is lawful) the CTA that finishes a head
+    does it, and that path must drop the head's step just as cleanly."""
     w = wl.scaled(wl.LLAMA3_8B_32K, L=2, T=3000, steps=4)
     s = Session(w, chunk_tokens=256, kv_dtype=kv)
     assert int(s.cap.min()) > 2 * 128
@@ -215,7 +218,8 @@ def test_wait_that_runs_out_sets_timeout_and_leaves_everything_usable(kv):
     bk.baklava_set_wait_limit(2_000_000)                             # about a millisecond
     try:
         s.out.fill_(7.0)
-        bk.baklava_decode_attn(s.shape, s.cache, q, kn, vn, s.t, s.out, s.lse, bk.FLAG_TEST_STALL, s.plan, s.ws)
+        flags = bk.FLAG_TEST_STALL | (bk.FLAG_OVERLAP_PREV if one_kernel else 0)
+        bk.baklava_decode_attn(s.shape, s.cache, q, kn, vn, s.t, s.out, s.lse, flags, s.plan, s.ws)
         torch.cuda.synchronize()
     finally:
         bk.baklava_set_wait_limit(100_000_000)
