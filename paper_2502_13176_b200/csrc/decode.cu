@@ -250,7 +250,7 @@ struct SweepGroup {
     int4 p0, p1;
 };
 
-template <int G>
+template <int G, int NT = kThreads>
 __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, const int32_t* pos, int n_sink, int C,
                                            int j_begin, int n_hi, int hole, bool evict, int newest_candidate,
                                            const float* sm_M, const float* sm_invL, unsigned long long* sm_key,
@@ -311,7 +311,7 @@ __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, c
         }
     };
 
-    constexpr int kStride = 8 * kThreads;
+    constexpr int kStride = 8 * NT;
     const int n_full = n_hi & ~7;                          // rows covered by full groups
     int j0 = j_begin + 8 * tid;
     if (G <= 4) {
@@ -338,7 +338,7 @@ __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, c
         finish(g0, j0);
     }
     // the ragged end of the head: fewer than eight rows, one thread
-    if (tid == (((n_full - j_begin) >> 3) % kThreads) && n_full < n_hi) {
+    if (tid == (((n_full - j_begin) >> 3) % NT) && n_full < n_hi) {
         float f[G];
 #pragma unroll
         for (int a = 0; a < G; ++a) {
@@ -393,7 +393,7 @@ struct TailArgs {
     bool keep_logits, do_append, may_evict, pos_evict, overlap, split;
 };
 
-template <int D, bool kByPosition>
+template <int D, bool kByPosition, int NT = kThreads>
 __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch, int unit, int piece, int active) {
     // everything about the head is derived again from the parameters, so that the call passes five values
     const DecodeParams& p = *pp;
@@ -427,8 +427,8 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
     __shared__ float sm_M[kG];
     __shared__ float sm_invL[kG];
     __shared__ int sm_gave_up;
-    __shared__ unsigned long long sm_key[kThreads / 32];   // each warp's eviction candidate
-    __shared__ int sm_slot[kThreads / 32];
+    __shared__ unsigned long long sm_key[NT / 32];   // each warp's eviction candidate
+    __shared__ int sm_slot[NT / 32];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = t.G;
     const int psz = partial_floats(G, D);
@@ -440,7 +440,7 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
     const int n_ml = active * G;
     if (tid == 0) sm_gave_up = 0;
     __syncthreads();
-    for (int i = tid; i < n_ml; i += kThreads) {
+    for (int i = tid; i < n_ml; i += NT) {
         const int c = i / G, a = i - c * G;
         const float* pc = part0 + (int64_t)c * psz + G * D;
         const float mc = __ldcg(pc + a);
@@ -458,7 +458,7 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
         }
         return;
     }
-    for (int a = warp; a < G; a += kThreads / 32) {         // one warp per query head, lanes over the chunks
+    for (int a = warp; a < G; a += NT / 32) {         // one warp per query head, lanes over the chunks
         float mm = -INFINITY;
         for (int c = lane; c < active; c += 32) mm = fmaxf(mm, sm_mc[c * G + a]);
 #pragma unroll
@@ -488,13 +488,13 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
         }
         return;
     }
-    for (int i = tid; i < n_ml; i += kThreads) {            // each chunk's weight in the merged output
+    for (int i = tid; i < n_ml; i += NT) {            // each chunk's weight in the merged output
         const int a = i % G;
         const float mc = sm_mc[i];
         sm_lc[i] = (mc == -INFINITY) ? 0.0f : exp2f(mc - sm_M[a]);
     }
     __syncthreads();
-    for (int grp = tid; grp < G * D / 4; grp += kThreads) { // four output elements per thread, chunks in order
+    for (int grp = tid; grp < G * D / 4; grp += NT) { // four output elements per thread, chunks in order
         const int a = (grp * 4) / D;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         int c = 0;
@@ -541,14 +541,14 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
     const bool evict = !kByPosition && t.keep_logits && t.may_evict;
     if (!kByPosition && t.keep_logits) {
         switch (G) {
-            case 1: sweep_head<1>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 2: sweep_head<2>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 3: sweep_head<3>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 4: sweep_head<4>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 5: sweep_head<5>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 6: sweep_head<6>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            case 7: sweep_head<7>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
-            default: sweep_head<8>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 1: sweep_head<1, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 2: sweep_head<2, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 3: sweep_head<3, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 4: sweep_head<4, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 5: sweep_head<5, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 6: sweep_head<6, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            case 7: sweep_head<7, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
+            default: sweep_head<8, NT>(t.logit_h, t.score, t.pos, t.n_sink, t.C, 0, t.n_hi, t.hole, evict, t.newest_candidate, sm_M, sm_invL, sm_key, sm_slot); break;
         }
     }
     __syncthreads();                                        // output, scores and the warps' candidates are written
@@ -568,7 +568,7 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
             } else if (evict) {
                 wanted = true;
                 unsigned long long bk = ~0ull;
-                for (int w = 0; w < kThreads / 32; ++w)
+                for (int w = 0; w < NT / 32; ++w)
                     if (sm_key[w] < bk) { bk = sm_key[w]; victim = sm_slot[w]; }
             }
             if (wanted && victim < 0) atomicOr(t.status, BAKLAVA_STATUS_BAD_STATE);   // nothing outside sinks + window
@@ -1078,6 +1078,403 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
     finish_head<D, kByPosition>(&p, reinterpret_cast<float*>(ring_ptr), unit, piece, active);   // the ring is idle now
 }
 
+// ---------------------------------------------------------------- FP8 slabs on the 5th-generation tensor cores
+// With one-byte rows the bytes per token halve but the consumer warps' work per token does not, and converting
+// the codes in registers for mma.sync is most of that work.  Here both contractions of a 128-token stage run on
+// tcgen05 with E4M3 operands taken straight from the swizzled tiles TMA delivers, accumulators in tensor memory:
+//   S^T [128 tokens x 16] = K_tile (A, K-major) x (Q_hi | Q_lo)^T   (B: 16 rows x 128 channels in shared memory)
+//   O^T [128 channels x 16] += V_tile^T (A, MN-major) x (P_hi | P_lo)^T   (B: 16 rows x 128 tokens)
+// The query rows and the probabilities enter as sums of two E4M3 terms (eight significant bits, the precision of
+// their bf16 originals), the two halves of the 16 columns are added when they are read.  Warp 0 streams tiles
+// (TMA), warp 1 patches a landed tile where needed (append, rows that are no tokens) and issues the MMAs, warps
+// 2-5 do the softmax: thread = token for S^T (one tcgen05.ld of 16 columns per stage), thread = channel for O^T.
+constexpr int kTcThreads = 192;
+constexpr int kTcCtasPerSm = 3;
+constexpr int kTcTokens = 128;                          // tokens per stage
+constexpr uint32_t kTcTmemColumns = 64;                 // S^T twice (16 columns each) and O^T (16)
+constexpr uint32_t kTcOColumn = 32;
+constexpr int kTcSmem = 2 * 2 * kTcTokens * 128 + 2048 + 2 * 2048 + 1024;   // ring, query operand, two probability operands
+
+__device__ __forceinline__ float warp_max_f32(float x) {  // maximum over the warp through the integer reduction
+    int k = __float_as_int(x);
+    k = k >= 0 ? k : k ^ 0x7fffffff;                      // order-preserving map to signed integers
+    k = __reduce_max_sync(0xffffffffu, k);
+    return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel(const __grid_constant__ DecodeParams p,
+                                                                              const __grid_constant__ CUtensorMap k_map,
+                                                                              const __grid_constant__ CUtensorMap v_map) {
+    static_assert(D == 128, "one 128-byte swizzle span per row");
+    constexpr int kTT = kTcTokens;
+    constexpr int kTileBytes = kTT * D;                // one K (or V) tile: 16 KB
+    constexpr int kStageBytes = 2 * kTileBytes;
+    constexpr int kNS = 2;
+    constexpr int kG = BAKLAVA_MAX_GROUP;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[kNS], bar_pv[kNS], bar_s[2], bar_p[2], bar_done;
+    __shared__ uint32_t tmem_slot;
+    __shared__ float sm_wmax[2][4][kG];
+    __shared__ float sm_qdown[kG];
+    __shared__ float sm_l[4][kG];
+    __shared__ int sm_last;
+    __shared__ int sm_abort;
+    __shared__ int sm_issued;
+    __shared__ int sm_cabort;                           // set by the softmax warps only, read after their barrier
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = p.G;
+    const bool overlap = (p.flags & BAKLAVA_FLAG_OVERLAP_PREV) != 0;
+    if (tid == 0) {
+        for (int s = 0; s < kNS; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_pv[s]), 1);
+            mbar_init(smem_u32(&bar_s[s]), 1);
+            mbar_init(smem_u32(&bar_p[s]), 4);
+        }
+        mbar_init(smem_u32(&bar_done), 1);
+        sm_abort = 0;
+        sm_cabort = 0;
+        sm_issued = 0;
+        ptx::fence_mbar_init();
+        prefetch_tensormap(&k_map);
+        prefetch_tensormap(&v_map);
+    }
+    if (!overlap) grid_dependency_wait();
+    else launch_dependents();
+    const int4 item = p.items[blockIdx.x];
+    const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
+    const Unit u = decode_unit(p, unit);
+    if (!overlap) launch_dependents();
+    const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
+    const HeadState hs = head_state(p, u);
+    const int C = hs.C, hole = hs.hole, n_hi = hs.n_att;
+    const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
+    if (t_pos < 0 || hs.bad || piece >= active) {
+        if (t_pos >= 0 && hs.bad && tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
+        if (overlap && tid == 0) grid_dependency_wait();
+        return;
+    }
+    if (hs.overflow && tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_OVERFLOW);
+    const int end = min(begin + chunk_len, n_hi);
+    const int n_tiles = end > begin ? (end - begin + kTT - 1) / kTT : 0;
+    const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
+    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
+    __half* prob_h = reinterpret_cast<__half*>(p.logit + row0 * G);
+    float* mref_h = reinterpret_cast<float*>(prob_h + (int64_t)G * C);
+
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
+    const uint32_t q_op = ring + kNS * kStageBytes;         // (Q_hi | Q_lo): 16 rows x 128 bytes, swizzled like a tile
+    uint8_t* q_ptr8 = ring_ptr + kNS * kStageBytes;
+    const uint32_t p_op = q_op + 2048;                      // two (P_hi | P_lo) operands of 16 rows x 128 tokens
+    uint8_t* p_ptr8 = q_ptr8 + 2048;
+
+    // the first tiles are requested before anything else is set up
+    const uint64_t stream_policy = l2_evict_first_policy();
+    auto request = [&](int it) {
+        const int s = it % kNS;
+        const uint32_t full = smem_u32(&bar_full[s]);
+        const uint32_t dst = ring + s * kStageBytes;
+        const int y = (int)(row0 + begin + it * kTT);
+        mbar_arrive_expect_tx(full, kStageBytes);
+        tma_load_2d(dst, &k_map, 0, y, full, stream_policy);
+        tma_load_2d(dst + kTileBytes, &v_map, 0, y, full, stream_policy);
+    };
+    int first_requests = 0;
+    if (tid == 0) {
+        for (; first_requests < n_tiles && first_requests < kNS; ++first_requests) {
+            if ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0 && first_requests == 1) break;
+            request(first_requests);
+        }
+        sm_issued = first_requests;
+    }
+    if (keep_logits) {
+        for (int r = begin + 32 * tid; r < end; r += 32 * kTcThreads) {
+            prefetch_l2(p.score + row0 + r);
+            prefetch_l2(p.pos + row0 + r);
+        }
+    }
+    if (warp == 1) {
+        tc::tmem_alloc(smem_u32(&tmem_slot), kTcTmemColumns);
+        tc::tmem_relinquish();
+    }
+    if (warp >= 2) {
+        // the query operand: consumer warp cw brings the rows of heads 2 cw and 2 cw + 1 to two E4M3 terms after a
+        // power-of-two scaling of the row (its largest magnitude to [128, 256)), four channels per lane
+        const int cw = warp - 2;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int h = 2 * cw + e;
+            const __nv_bfloat16* src = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + h) * D + 4 * lane;
+            const uint2 raw = h < G ? *reinterpret_cast<const uint2*>(src) : make_uint2(0u, 0u);
+            const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+            const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+            float amax = fmaxf(fmaxf(fabsf(f0.x), fabsf(f0.y)), fmaxf(fabsf(f1.x), fabsf(f1.y)));
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+            const int e2 = (amax > 0.0f && amax < INFINITY) ? max(-60, min(60, 7 - ilogbf(amax))) : 0;
+            const float up = exp2f((float)e2);
+            uint32_t hi0, lo0, hi1, lo1;
+            fp8::split_e4m3x2(pack_f16(f0.x * up, f0.y * up), hi0, lo0);
+            fp8::split_e4m3x2(pack_f16(f1.x * up, f1.y * up), hi1, lo1);
+            const uint32_t off_in_row = (uint32_t)((((lane >> 2) ^ (h & 7)) << 4) + ((lane & 3) << 2));
+            *reinterpret_cast<uint32_t*>(q_ptr8 + h * 128 + off_in_row) = hi0 | (hi1 << 16);
+            *reinterpret_cast<uint32_t*>(q_ptr8 + (8 + h) * 128 + off_in_row) = lo0 | (lo1 << 16);
+            if (lane == 0) sm_qdown[h] = exp2f((float)-e2);
+        }
+        tc::fence_proxy_async_smem();
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    tc::fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- producer
+        if (lane == 0) {
+            int it = first_requests;
+            for (; it < n_tiles; ++it) {
+                if ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0 && it == 1) break;
+                if (it >= kNS &&
+                    !mbar_wait(smem_u32(&bar_pv[it % kNS]), ((it / kNS) - 1) & 1, p.wait_cycles)) {   // the stage's tile is consumed
+                    atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
+                    sm_abort = 1;
+                    break;
+                }
+                request(it);
+            }
+            sm_issued = it;
+        }
+    } else if (warp == 1) {
+        // ---------------- tile patches (whole warp) and MMA issue (lane 0)
+        constexpr uint32_t idesc_s = tc::idesc_e4m3_f32(kTT, 16, false);
+        constexpr uint32_t idesc_o = tc::idesc_e4m3_f32(D, 16, true);
+        bool ok = true;
+        auto prepare = [&](int it) -> bool {                 // tile `it` has landed and holds what the MMAs must see
+            const int s = it % kNS;
+            int landed = mbar_wait(smem_u32(&bar_full[s]), (it / kNS) & 1, p.wait_cycles) ? 1 : 0;
+            landed = __shfl_sync(0xffffffffu, landed, 0);
+            if (!landed) return false;
+            const int tok0 = begin + it * kTT;
+            const int valid = min(kTT, end - tok0);
+            bool touched = false;
+            uint8_t* k_ptr = ring_ptr + s * kStageBytes;
+            if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
+                // step 1 (Eq. 4): the new token's row, quantised, replaces whatever the tile holds at the free slot,
+                // in shared memory for this pass and in the slab for the steps to come: lane = 8 elements of K or V
+                const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
+                const int64_t row = row0 + hs.f;
+                const bool is_v = lane >= 16;
+                const int c = lane & 15;
+                const uint4 raw = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
+                const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + (is_v ? 3 : 1)]);
+                *reinterpret_cast<uint2*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(hs.f - tok0, c >> 1) + (c & 1) * 8) = val;
+                uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
+                *(reinterpret_cast<uint2*>(slab + row * D) + c) = val;
+                if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
+                touched = true;
+            }
+            // rows past the end of the head (or the freed slot) may hold anything: keep them out of V^T P^T
+            if (valid < kTT || (hole >= tok0 && hole < tok0 + kTT)) {
+                uint8_t* v_ptr = k_ptr + kTileBytes;
+                const int first_bad = (hole >= tok0 && hole < tok0 + valid) ? hole - tok0 : valid;
+                for (int i = first_bad * 8 + lane; i < kTT * 8; i += 32) {
+                    const int r = i >> 3, c = i & 7;
+                    if (r >= valid || tok0 + r == hole)
+                        *reinterpret_cast<uint4*>(v_ptr + tile_offset(r, c)) = make_uint4(0, 0, 0, 0);
+                }
+                touched = true;
+            }
+            if (touched) tc::fence_proxy_async_smem();
+            __syncwarp();
+            return true;
+        };
+        auto issue_s = [&](int it) {                          // S^T of tile `it` into buffer it % 2
+            if (lane == 0) {
+                tc::fence_after_sync();
+                const uint64_t dk = tc::desc_k_major_sw128(ring + (it % kNS) * kStageBytes);
+                const uint64_t dq = tc::desc_k_major_sw128(q_op);
+#pragma unroll
+                for (int ks = 0; ks < D / 32; ++ks)           // 32 channels = 32 bytes per step
+                    tc::umma_e4m3(tmem_base + (it & 1) * 16, dk + ks * 2, dq + ks * 2, idesc_s, ks > 0);
+                tc::umma_commit(smem_u32(&bar_s[it & 1]));
+            }
+        };
+        if (n_tiles > 0) {
+            ok = prepare(0);
+            if (ok) issue_s(0);
+        }
+        for (int it = 0; it < n_tiles && ok; ++it) {
+            if (it + 1 < n_tiles) {
+                ok = prepare(it + 1);
+                if (!ok) break;
+                issue_s(it + 1);                              // its buffer held S^T of tile it - 1, long read
+            }
+            int ready = mbar_wait(smem_u32(&bar_p[it & 1]), (it >> 1) & 1, p.wait_cycles) ? 1 : 0;   // P^T of tile `it` is written
+            ready = __shfl_sync(0xffffffffu, ready, 0);
+            if (!ready) { ok = false; break; }
+            if (lane == 0) {
+                tc::fence_after_sync();
+                const uint64_t dv = tc::desc_mn_major_sw128(ring + (it % kNS) * kStageBytes + kTileBytes, 16);   // one 128-channel group: the leading offset is not used
+                const uint64_t dp = tc::desc_k_major_sw128(p_op + (it & 1) * 2048);
+#pragma unroll
+                for (int ks = 0; ks < kTT / 32; ++ks)         // 32 tokens per step: four 8-row groups of V, 32 bytes of P^T
+                    tc::umma_e4m3(tmem_base + kTcOColumn, dv + ((ks * 4096) >> 4), dp + ks * 2, idesc_o, (it > 0) || (ks > 0));
+                tc::umma_commit(smem_u32(&bar_pv[it % kNS]));  // the stage, the P^T buffer and (for a rescale) O^T are free
+            }
+        }
+        if (!ok) {
+            if (lane == 0) { atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT); sm_abort = 1; }
+        }
+        // nothing of this CTA's may still be running on the tensor cores when tensor memory is given back
+        if (lane == 0) {
+            tc::umma_commit(smem_u32(&bar_done));
+            mbar_wait(smem_u32(&bar_done), 0, p.wait_cycles);
+        }
+        __syncwarp();
+    } else {
+        // ---------------- softmax warps
+        const int cw = warp - 2;                              // slot in the exchange arrays
+        const int quarter = warp & 3;                         // the quarter of tensor memory this warp may touch
+        const int j = 32 * quarter + lane;                    // token of a stage (S^T) and channel (O^T)
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * quarter) << 16);
+        const float scale_k = p.scale_log2 * p.kv_scale[u.head * 4 + 0];
+        float scale_h[kG], m_run[kG], l_part[kG];
+#pragma unroll
+        for (int h = 0; h < kG; ++h) { scale_h[h] = scale_k * sm_qdown[h]; m_run[h] = -INFINITY; l_part[h] = 0.0f; }
+        for (int it = 0; it < n_tiles; ++it) {
+            const int b = it & 1;
+            if (!mbar_wait(smem_u32(&bar_s[b]), (it >> 1) & 1, p.wait_cycles)) sm_cabort = 1;
+            tc::fence_after_sync();
+            uint32_t c[16];
+            tc::tmem_ld_32x32_x16(lane_addr + b * 16, c);
+            tc::tmem_ld_wait();
+            const int tok = begin + it * kTT + j;
+            const bool valid = tok < end && tok != hole;
+            float sv[kG];
+#pragma unroll
+            for (int h = 0; h < kG; ++h) {
+                sv[h] = valid ? (__uint_as_float(c[h]) + __uint_as_float(c[8 + h])) * scale_h[h] : -INFINITY;
+                const float wm = warp_max_f32(sv[h]);
+                if (lane == h) sm_wmax[b][cw][h] = wm;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (sm_cabort) break;                             // the same for all four warps: written before the barrier
+            float corr[kG];
+            bool rescale = false;
+#pragma unroll
+            for (int h = 0; h < kG; ++h) {
+                const float ms = fmaxf(fmaxf(sm_wmax[b][0][h], sm_wmax[b][1][h]), fmaxf(sm_wmax[b][2][h], sm_wmax[b][3][h]));
+                const float m_new = fmaxf(m_run[h], ms);
+                corr[h] = (m_new == -INFINITY) ? 1.0f : fast_exp2(m_run[h] - m_new);
+                rescale |= corr[h] != 1.0f;
+                m_run[h] = m_new;
+            }
+            if (it >= 2 && !mbar_wait(smem_u32(&bar_pv[b]), ((it - 2) >> 1) & 1, p.wait_cycles)) sm_cabort = 1;   // P^T buffer b is free
+            if (rescale && it > 0) {
+                // the maximum of a head moved: O^T so far is brought to the new one (thread = channel)
+                if (!mbar_wait(smem_u32(&bar_pv[(it - 1) & 1]), ((it - 1) >> 1) & 1, p.wait_cycles)) sm_cabort = 1;
+                tc::fence_after_sync();
+                uint32_t o[16];
+                tc::tmem_ld_32x32_x16(lane_addr + kTcOColumn, o);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int h = 0; h < kG; ++h) {
+                    o[h] = __float_as_uint(__uint_as_float(o[h]) * corr[h]);
+                    o[8 + h] = __float_as_uint(__uint_as_float(o[8 + h]) * corr[h]);
+                }
+                tc::tmem_st_32x32_x16(lane_addr + kTcOColumn, o);
+                tc::tmem_st_wait();
+            }
+            float pv[kG];
+#pragma unroll
+            for (int h = 0; h < kG; ++h) {
+                pv[h] = valid ? fast_exp2(sv[h] - m_run[h]) : 0.0f;
+                l_part[h] = l_part[h] * corr[h] + pv[h];
+            }
+            // 256 p as two E4M3 terms into the P^T operand: row h the first, row 8 + h the second term, column = token
+#pragma unroll
+            for (int h2 = 0; h2 < kG / 2; ++h2) {
+                uint32_t hi, lo;
+                fp8::split_e4m3x2(pack_f16(pv[2 * h2] * 256.0f, pv[2 * h2 + 1] * 256.0f), hi, lo);
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int h = 2 * h2 + e;
+                    const uint32_t at = (uint32_t)(h * 128 + ((((j >> 4) ^ h) & 7) << 4) + (j & 15));   // (h and 8 + h share h % 8)
+                    p_ptr8[b * 2048 + at] = (uint8_t)(hi >> (8 * e));
+                    p_ptr8[b * 2048 + 1024 + at] = (uint8_t)(lo >> (8 * e));
+                }
+            }
+            if (keep_logits && tok < end) {
+                // the unnormalised probabilities, in fp16, and the maximum they were taken under, for the score pass
+#pragma unroll
+                for (int h = 0; h < kG; ++h)
+                    if (h < G) prob_h[(int64_t)h * C + tok] = __float2half_rn(pv[h]);
+                if ((tok & 15) == 0) {
+#pragma unroll
+                    for (int h = 0; h < kG; ++h)
+                        if (h < G) mref_h[h * (C >> 4) + (tok >> 4)] = m_run[h];
+                }
+            }
+            tc::fence_proxy_async_smem();
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_p[b]));
+        }
+        // ---- the chunk's partial: O^T (thread = channel), the maxima and the sums
+        const int psz_ = partial_floats(G, D);
+        float* part_ = p.partial + (int64_t)blockIdx.x * psz_;
+        uint32_t o[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) o[i] = 0u;
+        if (n_tiles > 0 && !sm_cabort) {
+            if (!mbar_wait(smem_u32(&bar_pv[(n_tiles - 1) & 1]), ((n_tiles - 1) >> 1) & 1, p.wait_cycles)) sm_cabort = 1;
+            tc::fence_after_sync();
+            tc::tmem_ld_32x32_x16(lane_addr + kTcOColumn, o);
+            tc::tmem_ld_wait();
+        }
+        const float sv_ = p.kv_scale[u.head * 4 + 2] * (1.0f / 256.0f);   // the probabilities went in as 256 p
+#pragma unroll
+        for (int h = 0; h < kG; ++h) {
+            if (h < G) part_[h * D + j] = (__uint_as_float(o[h]) + __uint_as_float(o[8 + h])) * sv_;
+            float ls = l_part[h];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, off);
+            if (lane == 0) sm_l[cw][h] = ls;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (sm_cabort) sm_abort = 1;
+        if (cw == 0 && lane < G) {
+            part_[G * D + lane] = m_run[lane];   // (every thread holds the same maxima)
+            part_[G * D + G + lane] = (sm_l[0][lane] + sm_l[1][lane]) + (sm_l[2][lane] + sm_l[3][lane]);
+        }
+    }
+    tc::fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc::fence_after_sync();
+        tc::tmem_dealloc(tmem_base, kTcTmemColumns);
+    }
+    const int psz = partial_floats(G, D);
+    float* part = p.partial + (int64_t)blockIdx.x * psz;
+    if (sm_abort) {
+        // lost step (see decode_chunk_kernel): no copy may be left in flight, the chunk still arrives, with a mark
+        if (tid == 0) {
+            atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
+            for (int t = max(0, sm_issued - kNS); t < sm_issued; ++t)
+                mbar_wait(smem_u32(&bar_full[t % kNS]), (t / kNS) & 1, p.wait_cycles);
+        }
+        if (tid < G) part[G * D + tid] = __int_as_float(0x7fc00000);
+    }
+    __syncthreads();
+    if (tid == 0) sm_last = (arrive_acq_rel(p.arrive + unit) == active - 1);
+    __syncthreads();
+    if (!sm_last) return;
+    finish_head<D, false, kTcThreads>(&p, reinterpret_cast<float*>(ring_ptr), unit, piece, active);   // the ring is idle now
+}
+
 // ---------------------------------------------------------------- steps 3-4 as a kernel of their own
 // A short launch (one layer of one sequence) ends with a few long heads, and one CTA sweeping a long head would
 // be most of the call's time.  There the attention kernel stops after the heads' final statistics and this
@@ -1276,6 +1673,22 @@ bool make_slab_map_fp8(CUtensorMap* map, void* base, int64_t rows, int D) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+cudaError_t launch_fp8_tc(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
+    cudaError_t e = cudaFuncSetAttribute(decode_fp8_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.n_items);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kTcSmem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_fp8_tc_kernel<128>, p, km, vm);
+}
+
 template <int D, bool kByPosition, bool kFp8 = false>
 cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
     constexpr int kSmem = (kFp8 ? kFp8Stages * 2 * kFp8StageTokens * D : kStages * 2 * kTileTokens * D * 2) + 1024;
@@ -1389,7 +1802,7 @@ int decode_attn_impl(
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
-    if (quantised) err = p.window_evict ? launch_chunks<128, true, true>(p, k_map, v_map, s) : launch_chunks<128, false, true>(p, k_map, v_map, s);
+    if (quantised) err = p.window_evict ? launch_chunks<128, true, true>(p, k_map, v_map, s) : launch_fp8_tc(p, k_map, v_map, s);
     else if (p.window_evict) err = shape->D == 128 ? launch_chunks<128, true>(p, k_map, v_map, s) : launch_chunks<64, true>(p, k_map, v_map, s);
     else err = shape->D == 128 ? launch_chunks<128, false>(p, k_map, v_map, s) : launch_chunks<64, false>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;
