@@ -1090,10 +1090,11 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
 // 2-5 do the softmax: thread = token for S^T (one tcgen05.ld of 16 columns per stage), thread = channel for O^T.
 constexpr int kTcThreads = 192;
 constexpr int kTcCtasPerSm = 3;
+constexpr int kTcStages = 2;
 constexpr int kTcTokens = 128;                          // tokens per stage
 constexpr uint32_t kTcTmemColumns = 64;                 // S^T twice (16 columns each) and O^T (16)
 constexpr uint32_t kTcOColumn = 32;
-constexpr int kTcSmem = 2 * 2 * kTcTokens * 128 + 2048 + 2 * 2048 + 1024;   // ring, query operand, two probability operands
+constexpr int kTcSmem = kTcStages * 2 * kTcTokens * 128 + 2048 + 2 * 2048 + 1024;   // ring, query operand, two probability operands
 
 __device__ __forceinline__ float warp_max_f32(float x) {  // maximum over the warp through the integer reduction
     int k = __float_as_int(x);
@@ -1110,17 +1111,20 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
     constexpr int kTT = kTcTokens;
     constexpr int kTileBytes = kTT * D;                // one K (or V) tile: 16 KB
     constexpr int kStageBytes = 2 * kTileBytes;
-    constexpr int kNS = 2;
+    constexpr int kNS = kTcStages;
     constexpr int kG = BAKLAVA_MAX_GROUP;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_full[kNS], bar_pv[kNS], bar_s[2], bar_p[2], bar_done;
+    // K and V tiles have rings of their own: a K tile is free as soon as its S^T is computed (early), a V tile only
+    // after its V^T P^T, and it is K that the next S^T waits for
+    __shared__ __align__(8) uint64_t bar_fullk[kNS], bar_fullv[kNS], bar_pv[kNS], bar_s[2], bar_p[2], bar_done;
+    static_assert(kNS == 2, "bar_s doubles as the K ring's release");
     __shared__ uint32_t tmem_slot;
     __shared__ float sm_wmax[2][4][kG];
     __shared__ float sm_qdown[kG];
     __shared__ float sm_l[4][kG];
     __shared__ int sm_last;
     __shared__ int sm_abort;
-    __shared__ int sm_issued;
+    __shared__ int sm_issued;                           // K tiles requested (low 16 bits) and V tiles (high)
     __shared__ int sm_cabort;                           // set by the softmax warps only, read after their barrier
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1128,8 +1132,11 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
     const bool overlap = (p.flags & BAKLAVA_FLAG_OVERLAP_PREV) != 0;
     if (tid == 0) {
         for (int s = 0; s < kNS; ++s) {
-            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_fullk[s]), 1);
+            mbar_init(smem_u32(&bar_fullv[s]), 1);
             mbar_init(smem_u32(&bar_pv[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&bar_s[s]), 1);
             mbar_init(smem_u32(&bar_p[s]), 4);
         }
@@ -1173,22 +1180,25 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
 
     // the first tiles are requested before anything else is set up
     const uint64_t stream_policy = l2_evict_first_policy();
-    auto request = [&](int it) {
-        const int s = it % kNS;
-        const uint32_t full = smem_u32(&bar_full[s]);
-        const uint32_t dst = ring + s * kStageBytes;
-        const int y = (int)(row0 + begin + it * kTT);
-        mbar_arrive_expect_tx(full, kStageBytes);
-        tma_load_2d(dst, &k_map, 0, y, full, stream_policy);
-        tma_load_2d(dst + kTileBytes, &v_map, 0, y, full, stream_policy);
+    auto request_k = [&](int it) {
+        const uint32_t full = smem_u32(&bar_fullk[it % kNS]);
+        mbar_arrive_expect_tx(full, kTileBytes);
+        tma_load_2d(ring + (it % kNS) * kStageBytes, &k_map, 0, (int)(row0 + begin + it * kTT), full, stream_policy);
     };
+    auto request_v = [&](int it) {
+        const uint32_t full = smem_u32(&bar_fullv[it % kNS]);
+        mbar_arrive_expect_tx(full, kTileBytes);
+        tma_load_2d(ring + (it % kNS) * kStageBytes + kTileBytes, &v_map, 0, (int)(row0 + begin + it * kTT), full, stream_policy);
+    };
+    // test aid (BAKLAVA_FLAG_TEST_STALL): the first chunk of a head gets its first tile only
+    const int n_feed = ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0) ? min(n_tiles, 1) : n_tiles;
     int first_requests = 0;
     if (tid == 0) {
-        for (; first_requests < n_tiles && first_requests < kNS; ++first_requests) {
-            if ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0 && first_requests == 1) break;
-            request(first_requests);
+        for (; first_requests < n_feed && first_requests < kNS; ++first_requests) {
+            request_k(first_requests);
+            request_v(first_requests);
         }
-        sm_issued = first_requests;
+        sm_issued = first_requests | (first_requests << 16);
     }
     if (keep_logits) {
         for (int r = begin + 32 * tid; r < end; r += 32 * kTcThreads) {
@@ -1232,53 +1242,74 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
     const uint32_t tmem_base = tmem_slot;
 
     if (warp == 0) {
-        // ---------------- producer
+        // ---------------- producer: two streams, each waiting for its own ring
         if (lane == 0) {
-            int it = first_requests;
-            for (; it < n_tiles; ++it) {
-                if ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0 && it == 1) break;
-                if (it >= kNS &&
-                    !mbar_wait(smem_u32(&bar_pv[it % kNS]), ((it / kNS) - 1) & 1, p.wait_cycles)) {   // the stage's tile is consumed
+            int k_next = first_requests, v_next = first_requests;
+            long long since = clock64();
+            while (k_next < n_feed || v_next < n_feed) {
+                bool progressed = false;
+                if (k_next < n_feed && ptx::mbar_try(smem_u32(&bar_s[k_next & 1]), ((k_next >> 1) - 1) & 1)) {   // S^T of tile k_next - 2 is done
+                    request_k(k_next++);
+                    progressed = true;
+                }
+                if (v_next < n_feed && ptx::mbar_try(smem_u32(&bar_pv[v_next % kNS]), ((v_next / kNS) - 1) & 1)) {   // its V^T P^T too
+                    request_v(v_next++);
+                    progressed = true;
+                }
+                if (progressed) {
+                    since = clock64();
+                } else if (clock64() - since > p.wait_cycles) {
                     atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
                     sm_abort = 1;
                     break;
                 }
-                request(it);
             }
-            sm_issued = it;
+            sm_issued = k_next | (v_next << 16);
         }
     } else if (warp == 1) {
         // ---------------- tile patches (whole warp) and MMA issue (lane 0)
         constexpr uint32_t idesc_s = tc::idesc_e4m3_f32(kTT, 16, false);
         constexpr uint32_t idesc_o = tc::idesc_e4m3_f32(D, 16, true);
         bool ok = true;
-        auto prepare = [&](int it) -> bool {                 // tile `it` has landed and holds what the MMAs must see
+        auto prepare_k = [&](int it) {                       // the landed K tile holds what S^T must see
             const int s = it % kNS;
-            int landed = mbar_wait(smem_u32(&bar_full[s]), (it / kNS) & 1, p.wait_cycles) ? 1 : 0;
-            landed = __shfl_sync(0xffffffffu, landed, 0);
-            if (!landed) return false;
+            const int tok0 = begin + it * kTT;
+            const int valid = min(kTT, end - tok0);
+            if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
+                // step 1 (Eq. 4): the new token's row, quantised, replaces whatever the tiles hold at the free slot, in
+                // shared memory for this pass and in the slab for the steps to come: lane = 8 elements of K (or of V)
+                const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
+                const int64_t row = row0 + hs.f;
+                if (lane < 16) {
+                    const uint4 raw = *(reinterpret_cast<const uint4*>(p.k_new + src) + lane);
+                    const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + 1]);
+                    *reinterpret_cast<uint2*>(ring_ptr + s * kStageBytes + tile_offset(hs.f - tok0, lane >> 1) + (lane & 1) * 8) = val;
+                    *(reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.k_slab) + row * D) + lane) = val;
+                }
+                if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
+                tc::fence_proxy_async_smem();
+            }
+            __syncwarp();
+        };
+        auto prepare_v = [&](int it) {                       // and the V tile what V^T P^T must see
+            const int s = it % kNS;
             const int tok0 = begin + it * kTT;
             const int valid = min(kTT, end - tok0);
             bool touched = false;
-            uint8_t* k_ptr = ring_ptr + s * kStageBytes;
+            uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
             if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
-                // step 1 (Eq. 4): the new token's row, quantised, replaces whatever the tile holds at the free slot,
-                // in shared memory for this pass and in the slab for the steps to come: lane = 8 elements of K or V
                 const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
                 const int64_t row = row0 + hs.f;
-                const bool is_v = lane >= 16;
-                const int c = lane & 15;
-                const uint4 raw = *(reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src) + c);
-                const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + (is_v ? 3 : 1)]);
-                *reinterpret_cast<uint2*>(k_ptr + (is_v ? kTileBytes : 0) + tile_offset(hs.f - tok0, c >> 1) + (c & 1) * 8) = val;
-                uint8_t* slab = reinterpret_cast<uint8_t*>(is_v ? p.v_slab : p.k_slab);
-                *(reinterpret_cast<uint2*>(slab + row * D) + c) = val;
-                if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
+                if (lane < 16) {
+                    const uint4 raw = *(reinterpret_cast<const uint4*>(p.v_new + src) + lane);
+                    const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + 3]);
+                    *reinterpret_cast<uint2*>(v_ptr + tile_offset(hs.f - tok0, lane >> 1) + (lane & 1) * 8) = val;
+                    *(reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.v_slab) + row * D) + lane) = val;
+                }
                 touched = true;
             }
             // rows past the end of the head (or the freed slot) may hold anything: keep them out of V^T P^T
             if (valid < kTT || (hole >= tok0 && hole < tok0 + kTT)) {
-                uint8_t* v_ptr = k_ptr + kTileBytes;
                 const int first_bad = (hole >= tok0 && hole < tok0 + valid) ? hole - tok0 : valid;
                 for (int i = first_bad * 8 + lane; i < kTT * 8; i += 32) {
                     const int r = i >> 3, c = i & 7;
@@ -1289,7 +1320,6 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
             }
             if (touched) tc::fence_proxy_async_smem();
             __syncwarp();
-            return true;
         };
         auto issue_s = [&](int it) {                          // S^T of tile `it` into buffer it % 2
             if (lane == 0) {
@@ -1302,27 +1332,49 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
                 tc::umma_commit(smem_u32(&bar_s[it & 1]));
             }
         };
-        if (n_tiles > 0) {
-            ok = prepare(0);
-            if (ok) issue_s(0);
-        }
-        for (int it = 0; it < n_tiles && ok; ++it) {
-            if (it + 1 < n_tiles) {
-                ok = prepare(it + 1);
-                if (!ok) break;
-                issue_s(it + 1);                              // its buffer held S^T of tile it - 1, long read
+        // Two things can become ready, in either order: the next tile (then its S^T is issued, as long as its
+        // buffer's previous contents are read: at most one tile ahead of the P^T V products) and the probabilities
+        // of the oldest tile without its product (then O^T += V^T P^T is issued).  The thread looks at both.
+        int s_next = 0, pv_next = 0;
+        long long since = clock64();
+        while (pv_next < n_tiles && ok) {
+            int progressed = 0;
+            if (s_next < n_tiles && s_next <= pv_next + 1) {
+                int landed = ptx::mbar_try(smem_u32(&bar_fullk[s_next % kNS]), (s_next / kNS) & 1) ? 1 : 0;
+                landed = __shfl_sync(0xffffffffu, landed, 0);
+                if (landed) {
+                    prepare_k(s_next);
+                    issue_s(s_next);
+                    ++s_next;
+                    progressed = 1;
+                }
             }
-            int ready = mbar_wait(smem_u32(&bar_p[it & 1]), (it >> 1) & 1, p.wait_cycles) ? 1 : 0;   // P^T of tile `it` is written
-            ready = __shfl_sync(0xffffffffu, ready, 0);
-            if (!ready) { ok = false; break; }
-            if (lane == 0) {
-                tc::fence_after_sync();
-                const uint64_t dv = tc::desc_mn_major_sw128(ring + (it % kNS) * kStageBytes + kTileBytes, 16);   // one 128-channel group: the leading offset is not used
-                const uint64_t dp = tc::desc_k_major_sw128(p_op + (it & 1) * 2048);
+            if (pv_next < s_next) {
+                int ready = (ptx::mbar_try(smem_u32(&bar_p[pv_next & 1]), (pv_next >> 1) & 1) &&           // P^T of the tile is written
+                             ptx::mbar_try(smem_u32(&bar_fullv[pv_next % kNS]), (pv_next / kNS) & 1)) ? 1 : 0;   // and its V tile is there
+                ready = __shfl_sync(0xffffffffu, ready, 0);
+                if (ready) {
+                    const int it = pv_next;
+                    prepare_v(it);
+                    if (lane == 0) {
+                        tc::fence_after_sync();
+                        const uint64_t dv = tc::desc_mn_major_sw128(ring + (it % kNS) * kStageBytes + kTileBytes, 16);   // one 128-channel group: the leading offset is not used
+                        const uint64_t dp = tc::desc_k_major_sw128(p_op + (it & 1) * 2048);
 #pragma unroll
-                for (int ks = 0; ks < kTT / 32; ++ks)         // 32 tokens per step: four 8-row groups of V, 32 bytes of P^T
-                    tc::umma_e4m3(tmem_base + kTcOColumn, dv + ((ks * 4096) >> 4), dp + ks * 2, idesc_o, (it > 0) || (ks > 0));
-                tc::umma_commit(smem_u32(&bar_pv[it % kNS]));  // the stage, the P^T buffer and (for a rescale) O^T are free
+                        for (int ks = 0; ks < kTT / 32; ++ks)     // 32 tokens per step: four 8-row groups of V, 32 bytes of P^T
+                            tc::umma_e4m3(tmem_base + kTcOColumn, dv + ((ks * 4096) >> 4), dp + ks * 2, idesc_o, (it > 0) || (ks > 0));
+                        tc::umma_commit(smem_u32(&bar_pv[it % kNS]));   // the stage, the P^T buffer and (for a rescale) O^T are free
+                    }
+                    ++pv_next;
+                    progressed = 1;
+                }
+            }
+            if (progressed) {
+                since = clock64();
+            } else {
+                int late = (clock64() - since > p.wait_cycles) ? 1 : 0;
+                late = __shfl_sync(0xffffffffu, late, 0);
+                if (late) ok = false;
             }
         }
         if (!ok) {
@@ -1362,20 +1414,23 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (sm_cabort) break;                             // the same for all four warps: written before the barrier
+            // The reference of a head's probabilities only follows its maximum when that has moved by more than 1
+            // (a factor of two): probabilities then stay below 2, which 128 p in E4M3 holds, and O^T is rarely rescaled.
             float corr[kG];
             bool rescale = false;
 #pragma unroll
             for (int h = 0; h < kG; ++h) {
                 const float ms = fmaxf(fmaxf(sm_wmax[b][0][h], sm_wmax[b][1][h]), fmaxf(sm_wmax[b][2][h], sm_wmax[b][3][h]));
-                const float m_new = fmaxf(m_run[h], ms);
-                corr[h] = (m_new == -INFINITY) ? 1.0f : fast_exp2(m_run[h] - m_new);
+                const bool move = ms > m_run[h] + 1.0f;       // (also the first tokens of a head: -inf + 1 = -inf)
+                const float m_new = move ? ms : m_run[h];
+                corr[h] = (move && m_run[h] != -INFINITY) ? fast_exp2(m_run[h] - m_new) : 1.0f;
                 rescale |= corr[h] != 1.0f;
                 m_run[h] = m_new;
             }
-            if (it >= 2 && !mbar_wait(smem_u32(&bar_pv[b]), ((it - 2) >> 1) & 1, p.wait_cycles)) sm_cabort = 1;   // P^T buffer b is free
+            if (it >= 2 && !mbar_wait(smem_u32(&bar_pv[(it - 2) % kNS]), ((it - 2) / kNS) & 1, p.wait_cycles)) sm_cabort = 1;   // P^T buffer b is free
             if (rescale && it > 0) {
                 // the maximum of a head moved: O^T so far is brought to the new one (thread = channel)
-                if (!mbar_wait(smem_u32(&bar_pv[(it - 1) & 1]), ((it - 1) >> 1) & 1, p.wait_cycles)) sm_cabort = 1;
+                if (!mbar_wait(smem_u32(&bar_pv[(it - 1) % kNS]), ((it - 1) / kNS) & 1, p.wait_cycles)) sm_cabort = 1;
                 tc::fence_after_sync();
                 uint32_t o[16];
                 tc::tmem_ld_32x32_x16(lane_addr + kTcOColumn, o);
@@ -1394,11 +1449,11 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
                 pv[h] = valid ? fast_exp2(sv[h] - m_run[h]) : 0.0f;
                 l_part[h] = l_part[h] * corr[h] + pv[h];
             }
-            // 256 p as two E4M3 terms into the P^T operand: row h the first, row 8 + h the second term, column = token
+            // 128 p as two E4M3 terms into the P^T operand: row h the first, row 8 + h the second term, column = token
 #pragma unroll
             for (int h2 = 0; h2 < kG / 2; ++h2) {
                 uint32_t hi, lo;
-                fp8::split_e4m3x2(pack_f16(pv[2 * h2] * 256.0f, pv[2 * h2 + 1] * 256.0f), hi, lo);
+                fp8::split_e4m3x2(pack_f16(pv[2 * h2] * 128.0f, pv[2 * h2 + 1] * 128.0f), hi, lo);
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int h = 2 * h2 + e;
@@ -1407,6 +1462,11 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
                     p_ptr8[b * 2048 + 1024 + at] = (uint8_t)(lo >> (8 * e));
                 }
             }
+            tc::fence_proxy_async_smem();
+            tc::fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_p[b]));
+            // (after the hand-over: these stores are nobody's business but the score pass's)
             if (keep_logits && tok < end) {
                 // the unnormalised probabilities, in fp16, and the maximum they were taken under, for the score pass
 #pragma unroll
@@ -1418,10 +1478,6 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
                         if (h < G) mref_h[h * (C >> 4) + (tok >> 4)] = m_run[h];
                 }
             }
-            tc::fence_proxy_async_smem();
-            tc::fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_p[b]));
         }
         // ---- the chunk's partial: O^T (thread = channel), the maxima and the sums
         const int psz_ = partial_floats(G, D);
@@ -1430,12 +1486,12 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
 #pragma unroll
         for (int i = 0; i < 16; ++i) o[i] = 0u;
         if (n_tiles > 0 && !sm_cabort) {
-            if (!mbar_wait(smem_u32(&bar_pv[(n_tiles - 1) & 1]), ((n_tiles - 1) >> 1) & 1, p.wait_cycles)) sm_cabort = 1;
+            if (!mbar_wait(smem_u32(&bar_pv[(n_tiles - 1) % kNS]), ((n_tiles - 1) / kNS) & 1, p.wait_cycles)) sm_cabort = 1;
             tc::fence_after_sync();
             tc::tmem_ld_32x32_x16(lane_addr + kTcOColumn, o);
             tc::tmem_ld_wait();
         }
-        const float sv_ = p.kv_scale[u.head * 4 + 2] * (1.0f / 256.0f);   // the probabilities went in as 256 p
+        const float sv_ = p.kv_scale[u.head * 4 + 2] * (1.0f / 128.0f);   // the probabilities went in as 128 p
 #pragma unroll
         for (int h = 0; h < kG; ++h) {
             if (h < G) part_[h * D + j] = (__uint_as_float(o[h]) + __uint_as_float(o[8 + h])) * sv_;
@@ -1463,8 +1519,9 @@ __global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel
         // lost step (see decode_chunk_kernel): no copy may be left in flight, the chunk still arrives, with a mark
         if (tid == 0) {
             atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
-            for (int t = max(0, sm_issued - kNS); t < sm_issued; ++t)
-                mbar_wait(smem_u32(&bar_full[t % kNS]), (t / kNS) & 1, p.wait_cycles);
+            const int nk = sm_issued & 0xffff, nv = sm_issued >> 16;
+            for (int t = max(0, nk - kNS); t < nk; ++t) mbar_wait(smem_u32(&bar_fullk[t % kNS]), (t / kNS) & 1, p.wait_cycles);
+            for (int t = max(0, nv - kNS); t < nv; ++t) mbar_wait(smem_u32(&bar_fullv[t % kNS]), (t / kNS) & 1, p.wait_cycles);
         }
         if (tid < G) part[G * D + tid] = __int_as_float(0x7fc00000);
     }
