@@ -210,13 +210,15 @@ int baklava_allocate(const baklava_shape* shape, const double* kv_importance,
  *   cap           host int32 [L, Hkv]
  *   chunk_tokens  target chunk length, 0 = choose from the total work and n_sm
  *   n_sm          streaming multiprocessors of the device (used when chunk_tokens = 0)
+ *   kv_dtype      BAKLAVA_KV_* of the cache the plan is for: with one-byte rows a chunk of the same
+ *                 length is half the bytes, so the automatic choice makes chunks twice as long
  *   items_out     host int32 [4 * items_capacity] or NULL to only fill `info`
  * The caller copies items_out ((info->n_items + info->n_score_items) * 16 bytes) to the device and hands it
  * to baklava_decode_attn together with `info`. */
 int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t B,
                         int32_t layer_begin, int32_t layer_end, int32_t chunk_tokens, int32_t n_sm,
-                        int64_t seq_stride_tokens, int32_t* items_out, int64_t items_capacity,
-                        baklava_plan_info* info);
+                        int32_t kv_dtype, int64_t seq_stride_tokens, int32_t* items_out,
+                        int64_t items_capacity, baklava_plan_info* info);
 
 /* One decode step for layers [layer_begin, layer_end) of every sequence, in this order
  * per (sequence, layer, KV head):

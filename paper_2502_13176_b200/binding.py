@@ -70,7 +70,7 @@ def lib():
         L.baklava_allocate.argtypes = [POINTER(Shape), POINTER(c_double), POINTER(AllocParams), c_int64,
                                        POINTER(c_int32), POINTER(c_int64), POINTER(c_int64)]
         L.baklava_decode_plan.argtypes = [POINTER(Shape), POINTER(c_int32), c_int32, c_int32, c_int32, c_int32,
-                                          c_int32, c_int64, POINTER(c_int32), c_int64, POINTER(PlanInfo)]
+                                          c_int32, c_int32, c_int64, POINTER(c_int32), c_int64, POINTER(PlanInfo)]
         L.baklava_decode_attn.argtypes = [POINTER(Shape), POINTER(CacheStruct), c_void_p, c_void_p, c_void_p, c_int32,
                                           c_void_p, c_void_p, c_uint32, c_void_p, POINTER(PlanInfo),
                                           c_void_p, c_size_t, c_void_p]
@@ -164,15 +164,15 @@ class Plan:
         return self
 
 
-def baklava_decode_plan(shape, cap, B, layer_begin, layer_end, seq_stride_tokens, chunk_tokens=0, n_sm=148):
+def baklava_decode_plan(shape, cap, B, layer_begin, layer_end, seq_stride_tokens, chunk_tokens=0, n_sm=148, kv_dtype=0):
     cap = np.ascontiguousarray(cap, dtype=np.int32).reshape(shape.L, shape.Hkv)
     info = PlanInfo()
     capp = cap.ctypes.data_as(POINTER(c_int32))
-    _check(lib().baklava_decode_plan(ctypes.byref(shape), capp, B, layer_begin, layer_end, chunk_tokens, n_sm,
+    _check(lib().baklava_decode_plan(ctypes.byref(shape), capp, B, layer_begin, layer_end, chunk_tokens, n_sm, kv_dtype,
                                      int(seq_stride_tokens), None, 0, ctypes.byref(info)), "baklava_decode_plan")
     total = info.n_items + info.n_score_items
     items = np.empty((total, 4), dtype=np.int32)
-    _check(lib().baklava_decode_plan(ctypes.byref(shape), capp, B, layer_begin, layer_end, chunk_tokens, n_sm,
+    _check(lib().baklava_decode_plan(ctypes.byref(shape), capp, B, layer_begin, layer_end, chunk_tokens, n_sm, kv_dtype,
                                      int(seq_stride_tokens), items.ctypes.data_as(POINTER(c_int32)), total,
                                      ctypes.byref(info)), "baklava_decode_plan")
     return Plan(items, info)

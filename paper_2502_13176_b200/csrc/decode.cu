@@ -1078,460 +1078,6 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
     finish_head<D, kByPosition>(&p, reinterpret_cast<float*>(ring_ptr), unit, piece, active);   // the ring is idle now
 }
 
-// ---------------------------------------------------------------- FP8 slabs on the 5th-generation tensor cores
-// With one-byte rows the bytes per token halve but the consumer warps' work per token does not, and converting
-// the codes in registers for mma.sync is most of that work.  Here both contractions of a 128-token stage run on
-// tcgen05 with E4M3 operands taken straight from the swizzled tiles TMA delivers, accumulators in tensor memory:
-//   S^T [128 tokens x 16] = K_tile (A, K-major) x (Q_hi | Q_lo)^T   (B: 16 rows x 128 channels in shared memory)
-//   O^T [128 channels x 16] += V_tile^T (A, MN-major) x (P_hi | P_lo)^T   (B: 16 rows x 128 tokens)
-// The query rows and the probabilities enter as sums of two E4M3 terms (eight significant bits, the precision of
-// their bf16 originals), the two halves of the 16 columns are added when they are read.  Warp 0 streams tiles
-// (TMA), warp 1 patches a landed tile where needed (append, rows that are no tokens) and issues the MMAs, warps
-// 2-5 do the softmax: thread = token for S^T (one tcgen05.ld of 16 columns per stage), thread = channel for O^T.
-constexpr int kTcThreads = 192;
-constexpr int kTcCtasPerSm = 3;
-constexpr int kTcStages = 2;
-constexpr int kTcTokens = 128;                          // tokens per stage
-constexpr uint32_t kTcTmemColumns = 64;                 // S^T twice (16 columns each) and O^T (16)
-constexpr uint32_t kTcOColumn = 32;
-constexpr int kTcSmem = kTcStages * 2 * kTcTokens * 128 + 2048 + 2 * 2048 + 1024;   // ring, query operand, two probability operands
-
-__device__ __forceinline__ float warp_max_f32(float x) {  // maximum over the warp through the integer reduction
-    int k = __float_as_int(x);
-    k = k >= 0 ? k : k ^ 0x7fffffff;                      // order-preserving map to signed integers
-    k = __reduce_max_sync(0xffffffffu, k);
-    return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff);
-}
-
-template <int D>
-__global__ void __launch_bounds__(kTcThreads, kTcCtasPerSm) decode_fp8_tc_kernel(const __grid_constant__ DecodeParams p,
-                                                                              const __grid_constant__ CUtensorMap k_map,
-                                                                              const __grid_constant__ CUtensorMap v_map) {
-    static_assert(D == 128, "one 128-byte swizzle span per row");
-    constexpr int kTT = kTcTokens;
-    constexpr int kTileBytes = kTT * D;                // one K (or V) tile: 16 KB
-    constexpr int kStageBytes = 2 * kTileBytes;
-    constexpr int kNS = kTcStages;
-    constexpr int kG = BAKLAVA_MAX_GROUP;
-    extern __shared__ uint8_t smem_raw[];
-    // K and V tiles have rings of their own: a K tile is free as soon as its S^T is computed (early), a V tile only
-    // after its V^T P^T, and it is K that the next S^T waits for
-    __shared__ __align__(8) uint64_t bar_fullk[kNS], bar_fullv[kNS], bar_pv[kNS], bar_s[2], bar_p[2], bar_done;
-    static_assert(kNS == 2, "bar_s doubles as the K ring's release");
-    __shared__ uint32_t tmem_slot;
-    __shared__ float sm_wmax[2][4][kG];
-    __shared__ float sm_qdown[kG];
-    __shared__ float sm_l[4][kG];
-    __shared__ int sm_last;
-    __shared__ int sm_abort;
-    __shared__ int sm_issued;                           // K tiles requested (low 16 bits) and V tiles (high)
-    __shared__ int sm_cabort;                           // set by the softmax warps only, read after their barrier
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = p.G;
-    const bool overlap = (p.flags & BAKLAVA_FLAG_OVERLAP_PREV) != 0;
-    if (tid == 0) {
-        for (int s = 0; s < kNS; ++s) {
-            mbar_init(smem_u32(&bar_fullk[s]), 1);
-            mbar_init(smem_u32(&bar_fullv[s]), 1);
-            mbar_init(smem_u32(&bar_pv[s]), 1);
-        }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&bar_s[s]), 1);
-            mbar_init(smem_u32(&bar_p[s]), 4);
-        }
-        mbar_init(smem_u32(&bar_done), 1);
-        sm_abort = 0;
-        sm_cabort = 0;
-        sm_issued = 0;
-        ptx::fence_mbar_init();
-        prefetch_tensormap(&k_map);
-        prefetch_tensormap(&v_map);
-    }
-    if (!overlap) grid_dependency_wait();
-    else launch_dependents();
-    const int4 item = p.items[blockIdx.x];
-    const int unit = item.x, begin = item.y, chunk_len = item.z, piece = item.w & 0xffff;
-    const Unit u = decode_unit(p, unit);
-    if (!overlap) launch_dependents();
-    const int t_pos = p.t_pos_seq ? p.t_pos_seq[u.b] : p.t_pos;
-    const HeadState hs = head_state(p, u);
-    const int C = hs.C, hole = hs.hole, n_hi = hs.n_att;
-    const int active = n_hi > 0 ? (n_hi + chunk_len - 1) / chunk_len : 1;
-    if (t_pos < 0 || hs.bad || piece >= active) {
-        if (t_pos >= 0 && hs.bad && tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_BAD_STATE);
-        if (overlap && tid == 0) grid_dependency_wait();
-        return;
-    }
-    if (hs.overflow && tid == 0 && piece == 0) atomicOr(p.status, BAKLAVA_STATUS_OVERFLOW);
-    const int end = min(begin + chunk_len, n_hi);
-    const int n_tiles = end > begin ? (end - begin + kTT - 1) / kTT : 0;
-    const bool keep_logits = (p.flags & BAKLAVA_FLAG_NO_SCORE) == 0;
-    const int64_t row0 = (int64_t)u.b * p.seq_stride + p.slab_off[u.head];
-    __half* prob_h = reinterpret_cast<__half*>(p.logit + row0 * G);
-    float* mref_h = reinterpret_cast<float*>(prob_h + (int64_t)G * C);
-
-    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
-    const uint32_t q_op = ring + kNS * kStageBytes;         // (Q_hi | Q_lo): 16 rows x 128 bytes, swizzled like a tile
-    uint8_t* q_ptr8 = ring_ptr + kNS * kStageBytes;
-    const uint32_t p_op = q_op + 2048;                      // two (P_hi | P_lo) operands of 16 rows x 128 tokens
-    uint8_t* p_ptr8 = q_ptr8 + 2048;
-
-    // the first tiles are requested before anything else is set up
-    const uint64_t stream_policy = l2_evict_first_policy();
-    auto request_k = [&](int it) {
-        const uint32_t full = smem_u32(&bar_fullk[it % kNS]);
-        mbar_arrive_expect_tx(full, kTileBytes);
-        tma_load_2d(ring + (it % kNS) * kStageBytes, &k_map, 0, (int)(row0 + begin + it * kTT), full, stream_policy);
-    };
-    auto request_v = [&](int it) {
-        const uint32_t full = smem_u32(&bar_fullv[it % kNS]);
-        mbar_arrive_expect_tx(full, kTileBytes);
-        tma_load_2d(ring + (it % kNS) * kStageBytes + kTileBytes, &v_map, 0, (int)(row0 + begin + it * kTT), full, stream_policy);
-    };
-    // test aid (BAKLAVA_FLAG_TEST_STALL): the first chunk of a head gets its first tile only
-    const int n_feed = ((p.flags & BAKLAVA_FLAG_TEST_STALL) && piece == 0) ? min(n_tiles, 1) : n_tiles;
-    int first_requests = 0;
-    if (tid == 0) {
-        for (; first_requests < n_feed && first_requests < kNS; ++first_requests) {
-            request_k(first_requests);
-            request_v(first_requests);
-        }
-        sm_issued = first_requests | (first_requests << 16);
-    }
-    if (keep_logits) {
-        for (int r = begin + 32 * tid; r < end; r += 32 * kTcThreads) {
-            prefetch_l2(p.score + row0 + r);
-            prefetch_l2(p.pos + row0 + r);
-        }
-    }
-    if (warp == 1) {
-        tc::tmem_alloc(smem_u32(&tmem_slot), kTcTmemColumns);
-        tc::tmem_relinquish();
-    }
-    if (warp >= 2) {
-        // the query operand: consumer warp cw brings the rows of heads 2 cw and 2 cw + 1 to two E4M3 terms after a
-        // power-of-two scaling of the row (its largest magnitude to [128, 256)), four channels per lane
-        const int cw = warp - 2;
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int h = 2 * cw + e;
-            const __nv_bfloat16* src = p.q + ((int64_t)(u.li * p.B + u.b) * p.Hq + u.h * G + h) * D + 4 * lane;
-            const uint2 raw = h < G ? *reinterpret_cast<const uint2*>(src) : make_uint2(0u, 0u);
-            const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-            const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-            float amax = fmaxf(fmaxf(fabsf(f0.x), fabsf(f0.y)), fmaxf(fabsf(f1.x), fabsf(f1.y)));
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
-            const int e2 = (amax > 0.0f && amax < INFINITY) ? max(-60, min(60, 7 - ilogbf(amax))) : 0;
-            const float up = exp2f((float)e2);
-            uint32_t hi0, lo0, hi1, lo1;
-            fp8::split_e4m3x2(pack_f16(f0.x * up, f0.y * up), hi0, lo0);
-            fp8::split_e4m3x2(pack_f16(f1.x * up, f1.y * up), hi1, lo1);
-            const uint32_t off_in_row = (uint32_t)((((lane >> 2) ^ (h & 7)) << 4) + ((lane & 3) << 2));
-            *reinterpret_cast<uint32_t*>(q_ptr8 + h * 128 + off_in_row) = hi0 | (hi1 << 16);
-            *reinterpret_cast<uint32_t*>(q_ptr8 + (8 + h) * 128 + off_in_row) = lo0 | (lo1 << 16);
-            if (lane == 0) sm_qdown[h] = exp2f((float)-e2);
-        }
-        tc::fence_proxy_async_smem();
-    }
-    tc::fence_before_sync();
-    __syncthreads();
-    tc::fence_after_sync();
-    const uint32_t tmem_base = tmem_slot;
-
-    if (warp == 0) {
-        // ---------------- producer: two streams, each waiting for its own ring
-        if (lane == 0) {
-            int k_next = first_requests, v_next = first_requests;
-            long long since = clock64();
-            while (k_next < n_feed || v_next < n_feed) {
-                bool progressed = false;
-                if (k_next < n_feed && ptx::mbar_try(smem_u32(&bar_s[k_next & 1]), ((k_next >> 1) - 1) & 1)) {   // S^T of tile k_next - 2 is done
-                    request_k(k_next++);
-                    progressed = true;
-                }
-                if (v_next < n_feed && ptx::mbar_try(smem_u32(&bar_pv[v_next % kNS]), ((v_next / kNS) - 1) & 1)) {   // its V^T P^T too
-                    request_v(v_next++);
-                    progressed = true;
-                }
-                if (progressed) {
-                    since = clock64();
-                } else if (clock64() - since > p.wait_cycles) {
-                    atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
-                    sm_abort = 1;
-                    break;
-                }
-            }
-            sm_issued = k_next | (v_next << 16);
-        }
-    } else if (warp == 1) {
-        // ---------------- tile patches (whole warp) and MMA issue (lane 0)
-        constexpr uint32_t idesc_s = tc::idesc_e4m3_f32(kTT, 16, false);
-        constexpr uint32_t idesc_o = tc::idesc_e4m3_f32(D, 16, true);
-        bool ok = true;
-        auto prepare_k = [&](int it) {                       // the landed K tile holds what S^T must see
-            const int s = it % kNS;
-            const int tok0 = begin + it * kTT;
-            const int valid = min(kTT, end - tok0);
-            if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
-                // step 1 (Eq. 4): the new token's row, quantised, replaces whatever the tiles hold at the free slot, in
-                // shared memory for this pass and in the slab for the steps to come: lane = 8 elements of K (or of V)
-                const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
-                const int64_t row = row0 + hs.f;
-                if (lane < 16) {
-                    const uint4 raw = *(reinterpret_cast<const uint4*>(p.k_new + src) + lane);
-                    const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + 1]);
-                    *reinterpret_cast<uint2*>(ring_ptr + s * kStageBytes + tile_offset(hs.f - tok0, lane >> 1) + (lane & 1) * 8) = val;
-                    *(reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.k_slab) + row * D) + lane) = val;
-                }
-                if (lane == 0) { p.pos[row] = t_pos; p.score[row] = 0.0f; }
-                tc::fence_proxy_async_smem();
-            }
-            __syncwarp();
-        };
-        auto prepare_v = [&](int it) {                       // and the V tile what V^T P^T must see
-            const int s = it % kNS;
-            const int tok0 = begin + it * kTT;
-            const int valid = min(kTT, end - tok0);
-            bool touched = false;
-            uint8_t* v_ptr = ring_ptr + s * kStageBytes + kTileBytes;
-            if (hs.do_append && hs.f >= tok0 && hs.f < tok0 + valid) {
-                const int64_t src = ((int64_t)(u.li * p.B + u.b) * p.Hkv + u.h) * D;
-                const int64_t row = row0 + hs.f;
-                if (lane < 16) {
-                    const uint4 raw = *(reinterpret_cast<const uint4*>(p.v_new + src) + lane);
-                    const uint2 val = fp8::quantise8(raw, p.kv_scale[u.head * 4 + 3]);
-                    *reinterpret_cast<uint2*>(v_ptr + tile_offset(hs.f - tok0, lane >> 1) + (lane & 1) * 8) = val;
-                    *(reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.v_slab) + row * D) + lane) = val;
-                }
-                touched = true;
-            }
-            // rows past the end of the head (or the freed slot) may hold anything: keep them out of V^T P^T
-            if (valid < kTT || (hole >= tok0 && hole < tok0 + kTT)) {
-                const int first_bad = (hole >= tok0 && hole < tok0 + valid) ? hole - tok0 : valid;
-                for (int i = first_bad * 8 + lane; i < kTT * 8; i += 32) {
-                    const int r = i >> 3, c = i & 7;
-                    if (r >= valid || tok0 + r == hole)
-                        *reinterpret_cast<uint4*>(v_ptr + tile_offset(r, c)) = make_uint4(0, 0, 0, 0);
-                }
-                touched = true;
-            }
-            if (touched) tc::fence_proxy_async_smem();
-            __syncwarp();
-        };
-        auto issue_s = [&](int it) {                          // S^T of tile `it` into buffer it % 2
-            if (lane == 0) {
-                tc::fence_after_sync();
-                const uint64_t dk = tc::desc_k_major_sw128(ring + (it % kNS) * kStageBytes);
-                const uint64_t dq = tc::desc_k_major_sw128(q_op);
-#pragma unroll
-                for (int ks = 0; ks < D / 32; ++ks)           // 32 channels = 32 bytes per step
-                    tc::umma_e4m3(tmem_base + (it & 1) * 16, dk + ks * 2, dq + ks * 2, idesc_s, ks > 0);
-                tc::umma_commit(smem_u32(&bar_s[it & 1]));
-            }
-        };
-        // Two things can become ready, in either order: the next tile (then its S^T is issued, as long as its
-        // buffer's previous contents are read: at most one tile ahead of the P^T V products) and the probabilities
-        // of the oldest tile without its product (then O^T += V^T P^T is issued).  The thread looks at both.
-        int s_next = 0, pv_next = 0;
-        long long since = clock64();
-        while (pv_next < n_tiles && ok) {
-            int progressed = 0;
-            if (s_next < n_tiles && s_next <= pv_next + 1) {
-                int landed = ptx::mbar_try(smem_u32(&bar_fullk[s_next % kNS]), (s_next / kNS) & 1) ? 1 : 0;
-                landed = __shfl_sync(0xffffffffu, landed, 0);
-                if (landed) {
-                    prepare_k(s_next);
-                    issue_s(s_next);
-                    ++s_next;
-                    progressed = 1;
-                }
-            }
-            if (pv_next < s_next) {
-                int ready = (ptx::mbar_try(smem_u32(&bar_p[pv_next & 1]), (pv_next >> 1) & 1) &&           // P^T of the tile is written
-                             ptx::mbar_try(smem_u32(&bar_fullv[pv_next % kNS]), (pv_next / kNS) & 1)) ? 1 : 0;   // and its V tile is there
-                ready = __shfl_sync(0xffffffffu, ready, 0);
-                if (ready) {
-                    const int it = pv_next;
-                    prepare_v(it);
-                    if (lane == 0) {
-                        tc::fence_after_sync();
-                        const uint64_t dv = tc::desc_mn_major_sw128(ring + (it % kNS) * kStageBytes + kTileBytes, 16);   // one 128-channel group: the leading offset is not used
-                        const uint64_t dp = tc::desc_k_major_sw128(p_op + (it & 1) * 2048);
-#pragma unroll
-                        for (int ks = 0; ks < kTT / 32; ++ks)     // 32 tokens per step: four 8-row groups of V, 32 bytes of P^T
-                            tc::umma_e4m3(tmem_base + kTcOColumn, dv + ((ks * 4096) >> 4), dp + ks * 2, idesc_o, (it > 0) || (ks > 0));
-                        tc::umma_commit(smem_u32(&bar_pv[it % kNS]));   // the stage, the P^T buffer and (for a rescale) O^T are free
-                    }
-                    ++pv_next;
-                    progressed = 1;
-                }
-            }
-            if (progressed) {
-                since = clock64();
-            } else {
-                int late = (clock64() - since > p.wait_cycles) ? 1 : 0;
-                late = __shfl_sync(0xffffffffu, late, 0);
-                if (late) ok = false;
-            }
-        }
-        if (!ok) {
-            if (lane == 0) { atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT); sm_abort = 1; }
-        }
-        // nothing of this CTA's may still be running on the tensor cores when tensor memory is given back
-        if (lane == 0) {
-            tc::umma_commit(smem_u32(&bar_done));
-            mbar_wait(smem_u32(&bar_done), 0, p.wait_cycles);
-        }
-        __syncwarp();
-    } else {
-        // ---------------- softmax warps
-        const int cw = warp - 2;                              // slot in the exchange arrays
-        const int quarter = warp & 3;                         // the quarter of tensor memory this warp may touch
-        const int j = 32 * quarter + lane;                    // token of a stage (S^T) and channel (O^T)
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * quarter) << 16);
-        const float scale_k = p.scale_log2 * p.kv_scale[u.head * 4 + 0];
-        float scale_h[kG], m_run[kG], l_part[kG];
-#pragma unroll
-        for (int h = 0; h < kG; ++h) { scale_h[h] = scale_k * sm_qdown[h]; m_run[h] = -INFINITY; l_part[h] = 0.0f; }
-        for (int it = 0; it < n_tiles; ++it) {
-            const int b = it & 1;
-            if (!mbar_wait(smem_u32(&bar_s[b]), (it >> 1) & 1, p.wait_cycles)) sm_cabort = 1;
-            tc::fence_after_sync();
-            uint32_t c[16];
-            tc::tmem_ld_32x32_x16(lane_addr + b * 16, c);
-            tc::tmem_ld_wait();
-            const int tok = begin + it * kTT + j;
-            const bool valid = tok < end && tok != hole;
-            float sv[kG];
-#pragma unroll
-            for (int h = 0; h < kG; ++h) {
-                sv[h] = valid ? (__uint_as_float(c[h]) + __uint_as_float(c[8 + h])) * scale_h[h] : -INFINITY;
-                const float wm = warp_max_f32(sv[h]);
-                if (lane == h) sm_wmax[b][cw][h] = wm;
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (sm_cabort) break;                             // the same for all four warps: written before the barrier
-            // The reference of a head's probabilities only follows its maximum when that has moved by more than 1
-            // (a factor of two): probabilities then stay below 2, which 128 p in E4M3 holds, and O^T is rarely rescaled.
-            float corr[kG];
-            bool rescale = false;
-#pragma unroll
-            for (int h = 0; h < kG; ++h) {
-                const float ms = fmaxf(fmaxf(sm_wmax[b][0][h], sm_wmax[b][1][h]), fmaxf(sm_wmax[b][2][h], sm_wmax[b][3][h]));
-                const bool move = ms > m_run[h] + 1.0f;       // (also the first tokens of a head: -inf + 1 = -inf)
-                const float m_new = move ? ms : m_run[h];
-                corr[h] = (move && m_run[h] != -INFINITY) ? fast_exp2(m_run[h] - m_new) : 1.0f;
-                rescale |= corr[h] != 1.0f;
-                m_run[h] = m_new;
-            }
-            if (it >= 2 && !mbar_wait(smem_u32(&bar_pv[(it - 2) % kNS]), ((it - 2) / kNS) & 1, p.wait_cycles)) sm_cabort = 1;   // P^T buffer b is free
-            if (rescale && it > 0) {
-                // the maximum of a head moved: O^T so far is brought to the new one (thread = channel)
-                if (!mbar_wait(smem_u32(&bar_pv[(it - 1) % kNS]), ((it - 1) / kNS) & 1, p.wait_cycles)) sm_cabort = 1;
-                tc::fence_after_sync();
-                uint32_t o[16];
-                tc::tmem_ld_32x32_x16(lane_addr + kTcOColumn, o);
-                tc::tmem_ld_wait();
-#pragma unroll
-                for (int h = 0; h < kG; ++h) {
-                    o[h] = __float_as_uint(__uint_as_float(o[h]) * corr[h]);
-                    o[8 + h] = __float_as_uint(__uint_as_float(o[8 + h]) * corr[h]);
-                }
-                tc::tmem_st_32x32_x16(lane_addr + kTcOColumn, o);
-                tc::tmem_st_wait();
-            }
-            float pv[kG];
-#pragma unroll
-            for (int h = 0; h < kG; ++h) {
-                pv[h] = valid ? fast_exp2(sv[h] - m_run[h]) : 0.0f;
-                l_part[h] = l_part[h] * corr[h] + pv[h];
-            }
-            // 128 p as two E4M3 terms into the P^T operand: row h the first, row 8 + h the second term, column = token
-#pragma unroll
-            for (int h2 = 0; h2 < kG / 2; ++h2) {
-                uint32_t hi, lo;
-                fp8::split_e4m3x2(pack_f16(pv[2 * h2] * 128.0f, pv[2 * h2 + 1] * 128.0f), hi, lo);
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int h = 2 * h2 + e;
-                    const uint32_t at = (uint32_t)(h * 128 + ((((j >> 4) ^ h) & 7) << 4) + (j & 15));   // (h and 8 + h share h % 8)
-                    p_ptr8[b * 2048 + at] = (uint8_t)(hi >> (8 * e));
-                    p_ptr8[b * 2048 + 1024 + at] = (uint8_t)(lo >> (8 * e));
-                }
-            }
-            tc::fence_proxy_async_smem();
-            tc::fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_p[b]));
-            // (after the hand-over: these stores are nobody's business but the score pass's)
-            if (keep_logits && tok < end) {
-                // the unnormalised probabilities, in fp16, and the maximum they were taken under, for the score pass
-#pragma unroll
-                for (int h = 0; h < kG; ++h)
-                    if (h < G) prob_h[(int64_t)h * C + tok] = __float2half_rn(pv[h]);
-                if ((tok & 15) == 0) {
-#pragma unroll
-                    for (int h = 0; h < kG; ++h)
-                        if (h < G) mref_h[h * (C >> 4) + (tok >> 4)] = m_run[h];
-                }
-            }
-        }
-        // ---- the chunk's partial: O^T (thread = channel), the maxima and the sums
-        const int psz_ = partial_floats(G, D);
-        float* part_ = p.partial + (int64_t)blockIdx.x * psz_;
-        uint32_t o[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) o[i] = 0u;
-        if (n_tiles > 0 && !sm_cabort) {
-            if (!mbar_wait(smem_u32(&bar_pv[(n_tiles - 1) % kNS]), ((n_tiles - 1) / kNS) & 1, p.wait_cycles)) sm_cabort = 1;
-            tc::fence_after_sync();
-            tc::tmem_ld_32x32_x16(lane_addr + kTcOColumn, o);
-            tc::tmem_ld_wait();
-        }
-        const float sv_ = p.kv_scale[u.head * 4 + 2] * (1.0f / 128.0f);   // the probabilities went in as 128 p
-#pragma unroll
-        for (int h = 0; h < kG; ++h) {
-            if (h < G) part_[h * D + j] = (__uint_as_float(o[h]) + __uint_as_float(o[8 + h])) * sv_;
-            float ls = l_part[h];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, off);
-            if (lane == 0) sm_l[cw][h] = ls;
-        }
-        asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (sm_cabort) sm_abort = 1;
-        if (cw == 0 && lane < G) {
-            part_[G * D + lane] = m_run[lane];   // (every thread holds the same maxima)
-            part_[G * D + G + lane] = (sm_l[0][lane] + sm_l[1][lane]) + (sm_l[2][lane] + sm_l[3][lane]);
-        }
-    }
-    tc::fence_before_sync();
-    __syncthreads();
-    if (warp == 1) {
-        tc::fence_after_sync();
-        tc::tmem_dealloc(tmem_base, kTcTmemColumns);
-    }
-    const int psz = partial_floats(G, D);
-    float* part = p.partial + (int64_t)blockIdx.x * psz;
-    if (sm_abort) {
-        // lost step (see decode_chunk_kernel): no copy may be left in flight, the chunk still arrives, with a mark
-        if (tid == 0) {
-            atomicOr(p.status, BAKLAVA_STATUS_TIMEOUT);
-            const int nk = sm_issued & 0xffff, nv = sm_issued >> 16;
-            for (int t = max(0, nk - kNS); t < nk; ++t) mbar_wait(smem_u32(&bar_fullk[t % kNS]), (t / kNS) & 1, p.wait_cycles);
-            for (int t = max(0, nv - kNS); t < nv; ++t) mbar_wait(smem_u32(&bar_fullv[t % kNS]), (t / kNS) & 1, p.wait_cycles);
-        }
-        if (tid < G) part[G * D + tid] = __int_as_float(0x7fc00000);
-    }
-    __syncthreads();
-    if (tid == 0) sm_last = (arrive_acq_rel(p.arrive + unit) == active - 1);
-    __syncthreads();
-    if (!sm_last) return;
-    finish_head<D, false, kTcThreads>(&p, reinterpret_cast<float*>(ring_ptr), unit, piece, active);   // the ring is idle now
-}
-
 // ---------------------------------------------------------------- steps 3-4 as a kernel of their own
 // A short launch (one layer of one sequence) ends with a few long heads, and one CTA sweeping a long head would
 // be most of the call's time.  There the attention kernel stops after the heads' final statistics and this
@@ -1730,22 +1276,6 @@ bool make_slab_map_fp8(CUtensorMap* map, void* base, int64_t rows, int D) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-cudaError_t launch_fp8_tc(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
-    cudaError_t e = cudaFuncSetAttribute(decode_fp8_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
-    if (e != cudaSuccess) return e;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)p.n_items);
-    cfg.blockDim = dim3(kTcThreads);
-    cfg.dynamicSmemBytes = kTcSmem;
-    cfg.stream = s;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_fp8_tc_kernel<128>, p, km, vm);
-}
-
 template <int D, bool kByPosition, bool kFp8 = false>
 cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
     constexpr int kSmem = (kFp8 ? kFp8Stages * 2 * kFp8StageTokens * D : kStages * 2 * kTileTokens * D * 2) + 1024;
@@ -1859,7 +1389,7 @@ int decode_attn_impl(
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t err = cudaSuccess;
-    if (quantised) err = p.window_evict ? launch_chunks<128, true, true>(p, k_map, v_map, s) : launch_fp8_tc(p, k_map, v_map, s);
+    if (quantised) err = p.window_evict ? launch_chunks<128, true, true>(p, k_map, v_map, s) : launch_chunks<128, false, true>(p, k_map, v_map, s);
     else if (p.window_evict) err = shape->D == 128 ? launch_chunks<128, true>(p, k_map, v_map, s) : launch_chunks<64, true>(p, k_map, v_map, s);
     else err = shape->D == 128 ? launch_chunks<128, false>(p, k_map, v_map, s) : launch_chunks<64, false>(p, k_map, v_map, s);
     if (err != cudaSuccess) return BAKLAVA_ERR_CUDA;

@@ -1,7 +1,6 @@
 // FP8 E4M3 conversions for quantised K/V slabs (device side): the hardware's own converters.
 #pragma once
 #include <cuda_bf16.h>
-#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -29,22 +28,6 @@ __device__ __forceinline__ void f16x4_from_e4m3x4(uint32_t four, uint32_t& lo, u
         "cvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
         : "=r"(lo), "=r"(hi) : "r"(four));
 }
-// two fp16 values -> two E4M3 codes (round to nearest even, saturating); the low half lands in the low byte
-__device__ __forceinline__ uint32_t e4m3x2_from_f16x2(uint32_t pair) {
-    uint16_t d;
-    asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(d) : "r"(pair));
-    return d;
-}
-// A value x as the sum of two E4M3 numbers, hi = E4M3(x) and lo = E4M3(x - hi): eight significant bits instead of
-// four (the residual of the first rounding is at most 2^-4 of x and is itself kept to 2^-4).  Two values at a time,
-// given as an fp16 pair; returns the codes as (hi0, hi1) and (lo0, lo1), each in the low 16 bits.
-__device__ __forceinline__ void split_e4m3x2(uint32_t x_f16x2, uint32_t& hi, uint32_t& lo) {
-    hi = e4m3x2_from_f16x2(x_f16x2);
-    const uint32_t back = f16x2_from_e4m3x2(hi);
-    const __half2 res = __hsub2(*reinterpret_cast<const __half2*>(&x_f16x2), *reinterpret_cast<const __half2*>(&back));
-    lo = e4m3x2_from_f16x2(*reinterpret_cast<const uint32_t*>(&res));
-}
-
 // eight bf16 values (16 bytes) times `inv_scale` -> eight codes (8 bytes)
 __device__ __forceinline__ uint2 quantise8(uint4 raw, float inv_scale) {
     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};

@@ -179,13 +179,14 @@ size_t baklava_decode_ws_bytes(const baklava_shape* s, int64_t n_items, int64_t 
 
 extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const baklava_shape* shape, const int32_t* cap, int32_t B,
                                    int32_t layer_begin, int32_t layer_end, int32_t chunk_tokens, int32_t n_sm,
-                                   int64_t seq_stride_tokens, int32_t* items_out, int64_t items_capacity,
+                                   int32_t kv_dtype, int64_t seq_stride_tokens, int32_t* items_out, int64_t items_capacity,
                                    baklava_plan_info* info) {
     int rc = baklava_check_shape(shape);
     if (rc) return rc;
     if (!cap || !info || B <= 0 || seq_stride_tokens <= 0) return BAKLAVA_ERR_INVALID_ARG;
     if (layer_begin < 0 || layer_end > shape->L || layer_begin >= layer_end) return BAKLAVA_ERR_INVALID_ARG;
     if (chunk_tokens < 0 || (chunk_tokens == 0 && n_sm <= 0)) return BAKLAVA_ERR_INVALID_ARG;
+    if (kv_dtype != BAKLAVA_KV_BF16 && kv_dtype != BAKLAVA_KV_FP8_E4M3) return BAKLAVA_ERR_INVALID_ARG;
     const int Hkv = shape->Hkv, layers = layer_end - layer_begin;
 
     std::vector<int> heads((size_t)layers * Hkv);       // index (li * Hkv + h) inside the range
@@ -205,11 +206,15 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
     // dispatched in item order, so the list starts with long chunks (about half of a CTA slot's share of
     // the tokens: little per-chunk overhead) and ends with short ones (a short tail).
     bool guided = chunk_tokens == 0;
-    int64_t target = chunk_tokens;
+    int64_t target = chunk_tokens, min_chunk = kMinChunk;
     if (guided) {
         const int64_t slots = (int64_t)n_sm * kCtasPerSm;
-        target = (tokens / (2 * slots) + kTile - 1) / kTile * kTile;
-        target = std::max<int64_t>(kMinChunk, std::min<int64_t>(target, 4096));
+        // what a chunk costs besides its rows (start-up, partial, arrival) is paid per chunk, not per byte: with
+        // one-byte rows the same balance between that and the tail of the launch is struck at twice the length
+        const int64_t wide = kv_dtype == BAKLAVA_KV_FP8_E4M3 ? 2 : 1;
+        min_chunk = wide * kMinChunk;
+        target = (wide * tokens / (2 * slots) + kTile - 1) / kTile * kTile;
+        target = std::max<int64_t>(kMinChunk, std::min<int64_t>(target, wide * 4096));
         if (target == kMinChunk) {
             // A short launch (one layer of a model): nothing balances a second, partly filled wave, so all chunks
             // get the same length, the shortest (from the minimum up) with which every chunk is resident at once.
@@ -240,7 +245,7 @@ extern "C" __attribute__((visibility("default"))) int baklava_decode_plan(const 
                 if (done * 20 >= tokens * 19) want = base / 8;          // last 5 % of the tokens
                 else if (done * 5 >= tokens * 4) want = base / 4;       // 80 % .. 95 %
                 else if (done * 2 >= tokens) want = base / 2;           // 50 % .. 80 %
-                want = std::max<int64_t>(kMinChunk, want);
+                want = std::max<int64_t>(min_chunk, want);
             }
             done += c * B;
             int64_t pieces = (c + want - 1) / want;

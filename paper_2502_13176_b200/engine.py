@@ -33,7 +33,7 @@ class DecodeSession:
         self.lb, self.le = (0, w.L) if layers is None else layers
         n_sm = torch.cuda.get_device_properties(self.device).multi_processor_count
         self.plan = bk.baklava_decode_plan(self.shape, self.cap, w.B, self.lb, self.le, self.stride,
-                                           chunk_tokens=chunk_tokens, n_sm=n_sm).to(self.device)
+                                           chunk_tokens=chunk_tokens, n_sm=n_sm, kv_dtype=kv_dtype).to(self.device)
         self.ws = bk.decode_workspace(self.plan, self.device)
         nl = self.le - self.lb
         self.out = torch.zeros((nl, w.B, w.Hq, w.D), dtype=torch.bfloat16, device=self.device)
@@ -81,7 +81,7 @@ class DecodeSession:
         self.layer_plans = []
         for l in range(self.lb, self.le):
             plan = bk.baklava_decode_plan(self.shape, self.cap, self.w.B, l, l + 1, self.stride, chunk_tokens=chunk_tokens,
-                                          n_sm=n_sm).to(self.device)
+                                          n_sm=n_sm, kv_dtype=self.kv_dtype).to(self.device)
             self.layer_plans.append((plan, bk.decode_workspace(plan, self.device)))
 
     def step_layers(self, q, k_new, v_new, t_pos, flags=0, overlap=True):

@@ -67,14 +67,14 @@ class Session:
         self.lb, self.le = (0, w.L) if layers is None else layers
         self.plan = bk.baklava_decode_plan(self.shape, self.cap, w.B, self.lb, self.le, self.stride,
                                            chunk_tokens=chunk_tokens,
-                                           n_sm=torch.cuda.get_device_properties(0).multi_processor_count).to(device)
+                                           n_sm=torch.cuda.get_device_properties(0).multi_processor_count, kv_dtype=kv_dtype).to(device)
         self.ws = bk.decode_workspace(self.plan, device)
         self.layer_plans = None
         if per_layer:
             self.layer_plans = []
             for l in range(self.lb, self.le):
                 plan = bk.baklava_decode_plan(self.shape, self.cap, w.B, l, l + 1, self.stride, chunk_tokens=chunk_tokens,
-                                              n_sm=torch.cuda.get_device_properties(0).multi_processor_count).to(device)
+                                              n_sm=torch.cuda.get_device_properties(0).multi_processor_count, kv_dtype=kv_dtype).to(device)
                 self.layer_plans.append((plan, bk.decode_workspace(plan, device)))
         nl = self.le - self.lb
         self.out = torch.zeros((nl, w.B, w.Hq, w.D), dtype=torch.bfloat16, device=device)
