@@ -1279,8 +1279,16 @@ bool make_slab_map_fp8(CUtensorMap* map, void* base, int64_t rows, int D) {
 template <int D, bool kByPosition, bool kFp8 = false>
 cudaError_t launch_chunks(const DecodeParams& p, const CUtensorMap& km, const CUtensorMap& vm, cudaStream_t s) {
     constexpr int kSmem = (kFp8 ? kFp8Stages * 2 * kFp8StageTokens * D : kStages * 2 * kTileTokens * D * 2) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(decode_chunk_kernel<D, kByPosition, kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    // the attribute belongs to the function on the current device: set once per device and instantiation
+    static std::atomic<uint64_t> configured{0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    if (dev >= 64 || !(configured.load(std::memory_order_acquire) >> dev & 1)) {
+        e = cudaFuncSetAttribute(decode_chunk_kernel<D, kByPosition, kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+        if (e != cudaSuccess) return e;
+        if (dev < 64) configured.fetch_or(1ull << dev, std::memory_order_release);
+    }
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
