@@ -56,8 +56,15 @@ class VarlenSession(Session):
         self.out.fill_(7.0)                    # idle sequences must leave their rows alone
         self.lse.fill_(7.0)
         before = {b: (self.cache.len[b].clone(), self.cache.free_slot[b].clone()) for b in idle}
-        bk.baklava_decode_attn_varlen(self.shape, self.cache, q, kn, vn, t_dev, self.out, self.lse, flags,
-                                      self.plan, self.ws)
+        if self.layer_plans is None:
+            bk.baklava_decode_attn_varlen(self.shape, self.cache, q, kn, vn, t_dev, self.out, self.lse, flags,
+                                          self.plan, self.ws)
+        else:                                  # the layer loop of a model, every call after the first overlapping
+            torch.cuda.synchronize()
+            for i, (plan, ws) in enumerate(self.layer_plans):
+                bk.baklava_decode_attn_varlen(self.shape, self.cache, q[i:i + 1], kn[i:i + 1], vn[i:i + 1], t_dev,
+                                              self.out[i:i + 1], self.lse[i:i + 1],
+                                              flags | (bk.FLAG_OVERLAP_PREV if i > 0 else 0), plan, ws)
         torch.cuda.synchronize()
         qh, knh, vnh = f64(q), f64(kn), f64(vn)
         out, lse = f64(self.out), f64(self.lse)
@@ -115,6 +122,19 @@ def test_idle_sequences_are_left_untouched():
     s.step_varlen(4, idle=(0, 1, 2, 3))                 # a step with nobody in it
     st = s.head_state(3, 0, 0)
     assert st["len"] == 2
+
+
+def test_idle_sequences_in_overlapping_per_layer_calls():
+    """Per-layer calls with the overlap flag on a batch where sequences sit steps out: the CTAs of an idle
+    sequence have nothing to do but still take part in keeping the stream's order."""
+    w = wl.scaled(wl.TINY, B=4, L=4)
+    s = VarlenSession(w, [512, 128, 37, 0], per_layer=True)
+    s.step_varlen(0, idle=(3,))
+    s.step_varlen(1, idle=(1, 3))
+    s.step_varlen(2, idle=(0, 1, 2))
+    s.step_varlen(3)
+    s.step_varlen(4, idle=(0, 1, 2, 3))
+    s.step_varlen(5)
 
 
 def test_short_sequence_grows_into_its_budget_and_starts_evicting():
