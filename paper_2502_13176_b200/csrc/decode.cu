@@ -147,8 +147,31 @@ __device__ __forceinline__ int arrive_acq_rel(int32_t* ptr) {
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
-__device__ __forceinline__ void prefetch_l2(const void* ptr) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+__device__ __forceinline__ void prefetch_l2_keep(const void* ptr) {
+    asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(ptr));
+}
+// Scores and positions are read and rewritten once per step while a thousand times their size streams past: they
+// are accessed with the keep-longest priority, so that they are still in L2 a step later where they fit.
+__device__ __forceinline__ uint64_t l2_evict_last_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ float4 ld_keep(const float4* ptr, uint64_t policy) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr), "l"(policy));
+    return v;
+}
+__device__ __forceinline__ int4 ld_keep(const int4* ptr, uint64_t policy) {
+    int4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.s32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr), "l"(policy));
+    return v;
+}
+__device__ __forceinline__ void st_keep(float4* ptr, const float4 v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                 ::"l"(ptr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy) : "memory");
 }
 __device__ __forceinline__ int ld_acquire(const int32_t* ptr) {
     int v;
@@ -157,6 +180,17 @@ __device__ __forceinline__ int ld_acquire(const int32_t* ptr) {
 }
 __device__ __forceinline__ void st_release(int32_t* ptr, int v) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ptr), "r"(v) : "memory");
+}
+
+// Scratch that has been read for the last time: its lines are dropped from L2 where they stand, so that they are
+// never written back to device memory (what they hold afterwards is undefined; it is rewritten before it is read).
+// Only lines that lie wholly inside [lo, hi) are touched.
+template <int NT>
+__device__ __forceinline__ void drop_lines(const void* lo, const void* hi) {
+    const uintptr_t first = (reinterpret_cast<uintptr_t>(lo) + 127u) & ~(uintptr_t)127u;
+    const uintptr_t last = reinterpret_cast<uintptr_t>(hi) & ~(uintptr_t)127u;
+    for (uintptr_t x = first + 128u * threadIdx.x; x < last; x += 128u * NT)
+        asm volatile("discard.global.L2 [%0], 128;" ::"l"(x) : "memory");
 }
 
 // K and V are read once per step and never fit in L2: ask L2 to drop them first, so that the
@@ -263,6 +297,7 @@ __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, c
     for (int a = 0; a < G; ++a) { Mq[a] = sm_M[a]; iL[a] = sm_invL[a]; }
     unsigned long long best = ~0ull;
     int best_slot = -1;
+    const uint64_t keep = l2_evict_last_policy();
 
     auto load = [&](SweepGroup<G>& g, int j0) {              // a full group: rows j0 .. j0 + 7 all inside the head
 #pragma unroll
@@ -270,11 +305,11 @@ __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, c
             g.fac[a] = __ldcg(mref_h + a * (C >> 4) + (j0 >> 4));
             g.pr[a] = __ldcg(reinterpret_cast<const uint4*>(prob_h + (int64_t)a * C + j0));
         }
-        g.s0 = *reinterpret_cast<const float4*>(score + j0);
-        g.s1 = *reinterpret_cast<const float4*>(score + j0 + 4);
+        g.s0 = ld_keep(reinterpret_cast<const float4*>(score + j0), keep);
+        g.s1 = ld_keep(reinterpret_cast<const float4*>(score + j0 + 4), keep);
         if (evict) {
-            g.p0 = *reinterpret_cast<const int4*>(pos + j0);
-            g.p1 = *reinterpret_cast<const int4*>(pos + j0 + 4);
+            g.p0 = ld_keep(reinterpret_cast<const int4*>(pos + j0), keep);
+            g.p1 = ld_keep(reinterpret_cast<const int4*>(pos + j0 + 4), keep);
         }
     };
     auto finish = [&](SweepGroup<G>& g, int j0) {
@@ -296,8 +331,8 @@ __device__ __forceinline__ void sweep_head(const float* logit_h, float* score, c
         float sc[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) sc[e] = (j0 + e == hole) ? old[e] : old[e] + inc[e];   // the freed slot is not a row
-        *reinterpret_cast<float4*>(score + j0) = make_float4(sc[0], sc[1], sc[2], sc[3]);
-        *reinterpret_cast<float4*>(score + j0 + 4) = make_float4(sc[4], sc[5], sc[6], sc[7]);
+        st_keep(reinterpret_cast<float4*>(score + j0), make_float4(sc[0], sc[1], sc[2], sc[3]), keep);
+        st_keep(reinterpret_cast<float4*>(score + j0 + 4), make_float4(sc[4], sc[5], sc[6], sc[7]), keep);
         if (evict) {
             const int ps[8] = {g.p0.x, g.p0.y, g.p0.z, g.p0.w, g.p1.x, g.p1.y, g.p1.z, g.p1.w};
 #pragma unroll
@@ -552,6 +587,12 @@ __device__ __noinline__ void finish_head(const DecodeParams* pp, float* scratch,
         }
     }
     __syncthreads();                                        // output, scores and the warps' candidates are written
+    if (!kByPosition && t.keep_logits) {                    // the head's probabilities and reference maxima are spent
+        const char* h0 = reinterpret_cast<const char*>(t.logit_h);
+        drop_lines<NT>(h0, h0 + (size_t)G * t.C * 2 + (size_t)G * (t.C >> 4) * 4);
+    }
+    // and so are the chunks' partials (the sinks + window policy still reads its candidates from them below)
+    if (!kByPosition) drop_lines<NT>(part0, part0 + (int64_t)active * psz);
     if (tid == 0) {
         *t.arrive = 0;
         if (t.do_append) {
@@ -684,8 +725,8 @@ __global__ void __launch_bounds__(kThreads, kFp8 ? kFp8CtasPerSm : kCtasPerSm) d
     // touched a whole step ago.  Each chunk asks for its own share now, so that the tail finds them in L2.
     if (!kByPosition && keep_logits) {
         for (int r = begin + 32 * tid; r < end; r += 32 * kThreads) {
-            prefetch_l2(p.score + row0 + r);
-            prefetch_l2(p.pos + row0 + r);
+            prefetch_l2_keep(p.score + row0 + r);
+            prefetch_l2_keep(p.pos + row0 + r);
         }
     }
     __syncthreads();                                      // the barriers are initialised
@@ -1190,6 +1231,11 @@ __global__ void __launch_bounds__(kThreads) sweep_kernel(const DecodeParams p) {
         }
     }
     __syncthreads();
+    if (!lost && begin < end) {                             // this piece's probabilities are spent
+        const char* h0 = reinterpret_cast<const char*>(p.logit + row0 * G);
+        for (int a = 0; a < G; ++a)
+            drop_lines<kThreads>(h0 + ((size_t)a * C + begin) * 2, h0 + ((size_t)a * C + end) * 2);
+    }
     if (tid == 0) {
         unsigned long long bk = ~0ull;
         int bs = -1;
