@@ -54,7 +54,7 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
     constexpr int kBoxBytes = kTileRows * 128;              // one TMA box: 128 rows x 64 elements
     constexpr int kTileBytes = kTileRows * D * 2;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_res, bar_full[2], bar_empty[2], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ __align__(8) uint64_t bar_res, bar_full[2], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ float sm_lse[2][kTileRows];
     __shared__ int sm_abort;
@@ -94,7 +94,6 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
         mbar_init(smem_u32(&bar_res), 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), 1);
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
             mbar_init(smem_u32(&bar_acc_empty[s]), kEpilogueThreads / 32);
         }
@@ -125,7 +124,8 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
                 tma_load_3d(res_tile + bx * kBoxBytes, res_map, bx * 64, blk * kTileRows, head_res, smem_u32(&bar_res));
             for (int it = 0; it < n_it; ++it) {
                 const int s = it & 1;
-                if (it >= 2 && !mbar_wait(smem_u32(&bar_empty[s]), ((it >> 1) - 1) & 1)) { sm_abort = 1; break; }
+                // the stage is free once the MMAs of the tile two back have completed: their commit says so
+                if (it >= 2 && !mbar_wait(smem_u32(&bar_acc_full[s]), ((it >> 1) - 1) & 1)) { sm_abort = 1; break; }
                 const uint32_t bar = smem_u32(&bar_full[s]);
                 mbar_arrive_expect_tx(bar, kTileBytes);
 #pragma unroll
@@ -154,7 +154,7 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
                     tc::umma_bf16(tmem_base + s * kTileRows, da + off, db + off, idesc, ks > 0);
                 }
                 // one commit per tile (a commit costs the tensor pipe about as much as a third of this tile's
-                // MMAs): the epilogue, which sees the accumulator complete, releases the stage for the producer
+                // MMAs): it tells the epilogue that the accumulator is complete and the producer that the stage is free
                 tc::umma_commit(smem_u32(&bar_acc_full[s]));
             }
             if (!ok) sm_abort = 1;
@@ -184,7 +184,6 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
             float next_lse = 0.0f;
             if (PASS == kPassColumnSums && e < kTileRows && it + 1 < n_it) next_lse = fetch_lse(it + 1);
             if (!mbar_wait(smem_u32(&bar_acc_full[s]), (it >> 1) & 1)) { ok = false; break; }
-            if (tid == 64) tc::mbar_arrive(smem_u32(&bar_empty[s]));       // the MMAs have read the streamed tile
             tc::fence_after_sync();
             const bool diagonal = stream_blk(it) == blk;
             const uint32_t acc = lane_addr + s * kTileRows;
@@ -294,7 +293,6 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
         mbar_inval(smem_u32(&bar_res));
         for (int s = 0; s < 2; ++s) {
             mbar_inval(smem_u32(&bar_full[s]));
-            mbar_inval(smem_u32(&bar_empty[s]));
             mbar_inval(smem_u32(&bar_acc_full[s]));
             mbar_inval(smem_u32(&bar_acc_empty[s]));
         }
