@@ -6,10 +6,11 @@
 // 5th-generation tensor cores.  A CTA keeps one
 // 128-row operand tile resident in shared memory and streams the other operand's tiles through a
 // two-stage TMA ring; one thread issues tcgen05.mma into a double-buffered 128 x 128 fp32 accumulator in
-// tensor memory; eight epilogue warps read it back with tcgen05.ld, one accumulator row per pair of threads.
+// tensor memory; two groups of four epilogue warps, one per accumulator, read it back with tcgen05.ld, a thread
+// owning an accumulator row of every other tile.
 //   pass 1 (rows = queries): every query row's log-sum-exp, a running max / sum kept by its thread;
 //   pass 2 (rows = keys):    exp2(logit - lse[query]) summed along each key's row, again by its thread.
-// The only reduction across threads joins the two halves of a row in a fixed order, so the result is
+// The only reduction across threads joins the two groups' shares of a row in a fixed order, so the result is
 // reproducible bit for bit.
 #include <cmath>
 #include <cstdint>
@@ -24,7 +25,7 @@ using namespace ptx;
 
 constexpr int kTileRows = 128;       // rows of an operand tile = accumulator rows = accumulator columns
 constexpr int kThreads = 320;        // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, warps 2-9: epilogue
-constexpr int kEpilogueThreads = 256; // two threads per accumulator row, 64 columns each
+constexpr int kEpilogueThreads = 256; // two groups of 128, one per accumulator; a thread owns an accumulator row
 constexpr uint32_t kTmemColumns = 256;   // two 128-column accumulators
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kPassLse = 0, kPassColumnSums = 1, kPassRowMax = 2;   // row passes: kPassLse and kPassRowMax
@@ -56,7 +57,7 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_res, bar_full[2], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
-    __shared__ float sm_lse[2][kTileRows];
+    __shared__ float sm_lse[2][2][kTileRows];              // [group][tile parity inside the group][streamed row]
     __shared__ int sm_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -95,7 +96,7 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_acc_full[s]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[s]), kEpilogueThreads / 32);
+            mbar_init(smem_u32(&bar_acc_empty[s]), kEpilogueThreads / 64);   // the four warps of accumulator s
         }
         sm_abort = 0;
         fence_mbar_init();
@@ -160,44 +161,46 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
             if (!ok) sm_abort = 1;
         }
     } else {
-        // ---------------- epilogue: a warp reads its quarter of the TMEM lanes (thread = accumulator row);
-        // warps 2-5 take columns 0..63 of every tile, warps 6-9 columns 64..127
-        const int e = tid - 64;
-        const int row = 32 * (warp & 3) + lane;
-        const int half = (warp - 2) >> 2;
-        const int col_base = half * (kTileRows / 2);
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + col_base;
+        // ---------------- epilogue: a warp reads its quarter of the TMEM lanes (thread = accumulator row).
+        // Warps 2-5 take the tiles of accumulator 0 (the even ones), warps 6-9 those of accumulator 1: the two groups
+        // never wait for each other, so one of them has exponentials to do while the other waits for its next tile.
+        const int grp = (warp - 2) >> 2;
+        const int row = 32 * (warp & 3) + lane;              // = this thread's index inside its group
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + grp * kTileRows;
         float m_run = -INFINITY, l_run = 0.0f, colsum = 0.0f;
-        auto fetch_lse = [&](int it) -> float {              // the log-sum-exp of streamed query row e of tile it
-            const int t = stream_blk(it) * kTileRows + e;
+        auto fetch_lse = [&](int it) -> float {              // the log-sum-exp of streamed query row `row` of tile it
+            const int t = stream_blk(it) * kTileRows + row;
             if (p.lse_nat)                                   // the caller's own (natural logarithm; rows past the prompt: none)
                 return t < len ? p.lse_nat[(int64_t)stream_head(it) * p.T + t] * kLog2e : INFINITY;
             return t < p.T ? p.lse2[(int64_t)stream_head(it) * p.T + t] : INFINITY;
         };
+        auto group_barrier = [&]() {
+            if (grp == 0) asm volatile("bar.sync 1, 128;" ::: "memory");
+            else asm volatile("bar.sync 2, 128;" ::: "memory");
+        };
         if (PASS == kPassColumnSums) {
-            if (e < kTileRows) sm_lse[0][e] = fetch_lse(0);
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (grp < n_it) sm_lse[grp][0][row] = fetch_lse(grp);
+            group_barrier();
         }
         bool ok = true;
-        for (int it = 0; it < n_it; ++it) {
-            const int s = it & 1;
+        for (int it = grp; it < n_it; it += 2) {
+            const int par = (it >> 1) & 1;
             float next_lse = 0.0f;
-            if (PASS == kPassColumnSums && e < kTileRows && it + 1 < n_it) next_lse = fetch_lse(it + 1);
-            if (!mbar_wait(smem_u32(&bar_acc_full[s]), (it >> 1) & 1)) { ok = false; break; }
+            if (PASS == kPassColumnSums && it + 2 < n_it) next_lse = fetch_lse(it + 2);
+            if (!mbar_wait(smem_u32(&bar_acc_full[grp]), par)) { ok = false; break; }
             tc::fence_after_sync();
             const bool diagonal = stream_blk(it) == blk;
-            const uint32_t acc = lane_addr + s * kTileRows;
             if (PASS == kPassRowMax) {
                 // row = query, columns = keys: only the largest logit of the row is wanted (no exponentials)
 #pragma unroll
-                for (int c0 = 0; c0 < kTileRows / 2; c0 += 32) {
+                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
                     uint32_t v[32];
-                    tc::tmem_ld_32x32(acc + c0, v);
+                    tc::tmem_ld_32x32(lane_addr + c0, v);
                     tc::tmem_ld_wait();
                     if (diagonal) {
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (col_base + c0 + c > row) v[c] = 0xff800000u;    // -inf
+                            if (c0 + c > row) v[c] = 0xff800000u;    // -inf
                     }
                     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -208,14 +211,14 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
                 // row = query, columns = keys: keys above the query are masked on the diagonal tile.
                 // Online softmax statistics, 32 columns at a time.
 #pragma unroll
-                for (int c0 = 0; c0 < kTileRows / 2; c0 += 32) {
+                for (int c0 = 0; c0 < kTileRows; c0 += 32) {
                     uint32_t v[32];
-                    tc::tmem_ld_32x32(acc + c0, v);
+                    tc::tmem_ld_32x32(lane_addr + c0, v);
                     tc::tmem_ld_wait();
                     if (diagonal) {                            // keys above the query do not exist for it
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (col_base + c0 + c > row) v[c] = 0xff800000u;    // -inf
+                            if (c0 + c > row) v[c] = 0xff800000u;    // -inf
                     }
                     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -233,52 +236,55 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
             } else {
                 // row = key, columns = queries: queries before the key are masked on the diagonal tile;
                 // queries past the prompt carry lse = +inf and contribute exp2(-inf) = 0
-                const float* lse = sm_lse[s] + col_base;
-                uint32_t v0[32], v1[32];                     // this thread's 64 columns of the tile
-                tc::tmem_ld_32x32(acc, v0);
-                tc::tmem_ld_32x32(acc + 32, v1);
-                tc::tmem_ld_wait();
-                if (diagonal) {                                // queries before the key do not see it
+                const float* lse = sm_lse[grp][par];
+#pragma unroll
+                for (int c0 = 0; c0 < kTileRows; c0 += 64) {
+                    uint32_t v0[32], v1[32];                 // 64 columns of the tile at a time
+                    tc::tmem_ld_32x32(lane_addr + c0, v0);
+                    tc::tmem_ld_32x32(lane_addr + c0 + 32, v1);
+                    tc::tmem_ld_wait();
+                    if (diagonal) {                            // queries before the key do not see it
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            if (row > c0 + c) v0[c] = 0xff800000u;               // -inf
+                            if (row > c0 + 32 + c) v1[c] = 0xff800000u;
+                        }
+                    }
+                    float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
-                        if (row > col_base + c) v0[c] = 0xff800000u;             // -inf
-                        if (row > col_base + 32 + c) v1[c] = 0xff800000u;
+                        sum[c & 3] += fast_exp2(fmaf(__uint_as_float(v0[c]), p.scale_log2, -lse[c0 + c]));
+                        sum[(c + 2) & 3] += fast_exp2(fmaf(__uint_as_float(v1[c]), p.scale_log2, -lse[c0 + 32 + c]));
                     }
+                    colsum += (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 }
-                float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    sum[c & 3] += fast_exp2(fmaf(__uint_as_float(v0[c]), p.scale_log2, -lse[c]));
-                    sum[(c + 2) & 3] += fast_exp2(fmaf(__uint_as_float(v1[c]), p.scale_log2, -lse[32 + c]));
-                }
-                colsum += (sum[0] + sum[1]) + (sum[2] + sum[3]);
             }
             tc::fence_before_sync();
             __syncwarp();
-            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_acc_empty[s]));
+            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_acc_empty[grp]));
             if (PASS == kPassColumnSums) {
-                if (e < kTileRows) sm_lse[s ^ 1][e] = next_lse;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                sm_lse[grp][par ^ 1][row] = next_lse;         // (the buffer of this group's tile before this one)
+                group_barrier();
             }
         }
-        // join the two halves of every row: the upper half hands its state over through shared memory
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (half == 1) { sm_lse[0][row] = PASS != kPassColumnSums ? m_run : colsum; sm_lse[1][row] = l_run; }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // join the two groups' shares of every row: the second group hands its state over through shared memory
+        asm volatile("bar.sync 3, 256;" ::: "memory");
+        if (grp == 1) { sm_lse[0][0][row] = PASS != kPassColumnSums ? m_run : colsum; sm_lse[0][1][row] = l_run; }
+        asm volatile("bar.sync 3, 256;" ::: "memory");
         if (!ok) {
             sm_abort = 1;
-        } else if (half == 0) {
+        } else if (grp == 0) {
             const int t = blk * kTileRows + row;
             if (PASS == kPassRowMax) {
                 // scaled to the log2 domain like the log-sum-exp it stands in for
-                if (t < p.T) p.lse2[(int64_t)head_res * p.T + t] = t < len ? fmaxf(m_run, sm_lse[0][row]) * p.scale_log2 : INFINITY;
+                if (t < p.T) p.lse2[(int64_t)head_res * p.T + t] = t < len ? fmaxf(m_run, sm_lse[0][0][row]) * p.scale_log2 : INFINITY;
             } else if (PASS == kPassLse) {
-                const float m_hi = sm_lse[0][row], l_hi = sm_lse[1][row];
-                const float m_all = fmaxf(m_run, m_hi);      // m_run is finite: column 0 belongs to the lower half
+                const float m_hi = sm_lse[0][0][row], l_hi = sm_lse[0][1][row];
+                const float m_all = fmaxf(m_run, m_hi);      // m_run is finite: tile 0, with key 0, belongs to the first group
                 const float l_all = l_run * exp2f(m_run - m_all) + (m_hi == -INFINITY ? 0.0f : l_hi * exp2f(m_hi - m_all));
                 if (t < p.T) p.lse2[(int64_t)head_res * p.T + t] = t < len ? m_all + log2f(l_all) : INFINITY;
             } else {
-                if (t < p.T) p.score[(int64_t)head_res * p.T + t] = colsum + sm_lse[0][row];
+                if (t < p.T) p.score[(int64_t)head_res * p.T + t] = colsum + sm_lse[0][0][row];
             }
         }
     }
