@@ -9,8 +9,10 @@
 //
 // Inside a chunk: a producer warp streams 64-token K and V tiles with TMA (128-byte swizzle)
 // into a ring of shared-memory stages guarded by full/empty mbarriers; four consumer warps take
-// 16 tokens of each tile, contract the padded query group against K and the probabilities
-// against V with bf16 mma.sync (fp32 accumulate), and keep an online-softmax state each.
+// 16 tokens of each tile (the tokens are the M side of both contractions: S^T = K Q^T and
+// O^T += V^T P^T, bf16 mma.sync with fp32 accumulation) and keep an online-softmax state each.
+// What the step writes besides the cache (probabilities, partials) is dropped from L2 once it has
+// been read, and the scores and positions are kept in L2 from one step to the next where they fit.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
