@@ -7,13 +7,15 @@
 // among its first eight keys serves: p = exp2(s - reference), no running maximum, no sum, no rescaling of O, no
 // division.  (Rows whose later logits leave the fp32 range that way are detected in the epilogue and redone
 // by a second instantiation that takes the true row maxima from a row pass; see profile_pv_block.)
-// A CTA owns 128 query rows: the Q tile stays in shared memory, K and V tiles of 128 keys stream through
-// three-stage TMA rings; one thread issues S = Q K^T into tensor memory (double-buffered), sixteen softmax
-// warps read S back, form the probabilities in bf16 and write them back to tensor memory, from where the next
-// MMA takes them as its A operand, and the same thread issues O += P V with V as an MN-major B operand; O
-// accumulates in tensor memory over all key tiles and is never written.  The last key tile is the
-// diagonal one, whose V rows are exactly the rows the cosine needs, so the final epilogue reads them from
-// shared memory.
+// A CTA owns 128 query rows and half an SM: the Q tile, one K tile and one V tile of 128 keys in shared memory
+// (96 KB), 256 columns of tensor memory (S, with the probabilities written over it, and O), ten warps.  Per key
+// tile one thread issues O += P V for the tile before and S = Q K^T for this one (one commit), eight softmax warps
+// read S back, form the probabilities in bf16 and write them over the logits they came from, from where the next
+// MMA takes them as its A operand; V is an MN-major B operand; O accumulates in tensor memory over all key
+// tiles and is never written.  Inside one CTA these steps follow one another, each waiting for the one before it
+// and for the next tiles to land; the SM's second CTA, at another point of its own chain (or in its start-up or
+// its epilogue), uses the tensor pipe and the special-function unit meanwhile.  The last key tile is the diagonal
+// one, whose V rows are exactly the rows the cosine needs, so the final epilogue reads them from shared memory.
 // Per-CTA cosine sums go to the workspace and a small kernel adds them in a fixed order.
 #include <cmath>
 #include <cstdint>
@@ -27,11 +29,10 @@ namespace {
 using namespace ptx;
 
 constexpr int kTileRows = 128;        // query rows per CTA = keys per streamed tile
-constexpr int kSoftmaxWarps = 16;     // four threads per query row, 32 keys of a tile each
+constexpr int kSoftmaxWarps = 8;      // two threads per query row, 64 keys of a tile each
 constexpr int kThreads = (2 + kSoftmaxWarps) * 32;   // warp 0: TMA producer, warp 1: MMA issuer + TMEM owner, then softmax
 constexpr int kGroupRing = 4;         // mbarriers that track the MMA groups in flight
-constexpr int kKvStages = 3;          // K and V tiles in flight: the streamed operands come from L2 at a bounded rate
-constexpr uint32_t kTmemColumns = 512;    // S: 2 x 128 columns, O: D columns (at most 128), P: 2 x 64 columns
+constexpr uint32_t kTmemColumns = 256;    // S / P: 128 columns, O: D columns (at most 128)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kCosEps = 1e-12f;
 
@@ -73,12 +74,13 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
     constexpr int kPvSteps = kTileRows / 16;                 // MMA steps over the keys (O += P V)
     constexpr int kBoxBytes = kTileRows * 128;               // one TMA box: 128 rows x 64 elements
     constexpr int kTileBytes = kTileRows * D * 2;            // a Q, K or V tile
-    constexpr int kStageBytes = 2 * kTileBytes;              // K then V
-    constexpr uint32_t kOColumn = 2 * kTileRows;             // O sits after the two S buffers in tensor memory
-    constexpr uint32_t kPColumn = 3 * kTileRows;             // then two probability tiles: 128 keys in bf16 = 64 columns
-    constexpr uint32_t kPColumns = kTileRows / 2;
+    constexpr uint32_t kOColumn = kTileRows;                 // O sits after S in tensor memory
+    // A thread turns its 64 logits (64 columns) into 64 probabilities in bf16 (32 columns) and writes them into the
+    // upper half of its own 64 columns once it has read all of them: nobody else reads or writes those, and the
+    // tile's first columns, which every thread of a row reads for the reference, stay as they are.
+    constexpr uint32_t kPOffset = 32;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q, bar_k01[2], bar_in[kGroupRing], bar_group[kGroupRing];
+    __shared__ __align__(8) uint64_t bar_q, bar_k0, bar_in[kGroupRing], bar_group[kGroupRing];
     __shared__ uint32_t tmem_slot;
     __shared__ float sm_warp_sum[kSoftmaxWarps];
     __shared__ int sm_abort;
@@ -95,14 +97,13 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
     const int n_it = qb + 1;                                 // key tiles 0 .. qb
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
-    const uint32_t q_tile = base;
-    const uint32_t stage0 = base + kTileBytes;
+    const uint32_t q_tile = base, k_tile = base + kTileBytes, v_tile = base + 2 * kTileBytes;
 
     if (tid == 0) {
         mbar_init(smem_u32(&bar_q), 1);
-        for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&bar_k01[s]), 1);
+        mbar_init(smem_u32(&bar_k0), 1);
         for (int s = 0; s < kGroupRing; ++s) {
-            mbar_init(smem_u32(&bar_in[s]), kSoftmaxWarps + 2);   // P(it) written, V(it) landed, K(it + 2) landed
+            mbar_init(smem_u32(&bar_in[s]), kSoftmaxWarps + 2);   // P(it) written, V(it) landed, K(it + 1) landed
             mbar_init(smem_u32(&bar_group[s]), 1);
         }
         sm_abort = 0;
@@ -124,31 +125,27 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            mbar_arrive_expect_tx(smem_u32(&bar_q), kTileBytes);
-#pragma unroll
-            for (int bx = 0; bx < D / 64; ++bx)
-                tma_load_3d(q_tile + bx * kBoxBytes, &q_map, bx * 64, qb * kTileRows, pr * p.Hq + h, smem_u32(&bar_q));
-            // The single MMA thread pays well over a hundred cycles for every mbarrier it looks at, so
-            // everything group it + 2 = { P(it) V(it), S(it + 2) } needs arrives on ONE barrier, bar_in[it % 4]:
-            // the sixteen softmax warps (P(it) written) and the two loads V(it) and K(it + 2).
-            // K(j) reuses the stage of K(j - 3), consumed by S(j - 3) = MMA group j - 3; V(j) the stage of
-            // V(j - 3), consumed by P V of tile j - 3 = MMA group j - 1: both loads of bar_in[j % 4] wait for
-            // group j - 1.
-            auto load = [&](const CUtensorMap* map, uint32_t bar, uint32_t dst, int it) {
+            auto load = [&](const CUtensorMap* map, uint32_t bar, uint32_t dst, int row0, int head) {
                 mbar_arrive_expect_tx(bar, kTileBytes);
 #pragma unroll
-                for (int bx = 0; bx < D / 64; ++bx)
-                    tma_load_3d(dst + (it % kKvStages) * kStageBytes + bx * kBoxBytes, map, bx * 64, it * kTileRows,
-                                pr * p.Hkv + kvh, bar);
+                for (int bx = 0; bx < D / 64; ++bx) tma_load_3d(dst + bx * kBoxBytes, map, bx * 64, row0, head, bar);
             };
-            for (int j = 0; j < 2 && j < n_it; ++j) load(&k_map, smem_u32(&bar_k01[j]), stage0, j);
+            load(&q_map, smem_u32(&bar_q), q_tile, qb * kTileRows, pr * p.Hq + h);
+            load(&k_map, smem_u32(&bar_k0), k_tile, 0, pr * p.Hkv + kvh);
+            // The MMA thread pays well over a hundred cycles for every mbarrier it looks at, so everything group
+            // it + 1 = { P(it) V(it), S(it + 1) } needs arrives on ONE barrier, bar_in[it % 4]: the eight softmax warps
+            // (P(it) written) and the two loads V(it) and K(it + 1).  There is one K and one V tile: K(j + 1) takes
+            // the place of K(j) once S(j) is complete and V(j) that of V(j - 1) once P V of tile j - 1 is, and both
+            // are in MMA group j.
             bool ok = true;
             for (int j = 0; j < n_it && ok; ++j) {
-                if (j >= 1) ok = group_wait(j - 1);           // (K(3) and K(4) already reuse a stage)
-                if (!ok) break;
                 const uint32_t bar = smem_u32(&bar_in[j % kGroupRing]);
-                load(&v_map, bar, stage0 + kTileBytes, j);
-                if (j + 2 < n_it) load(&k_map, bar, stage0, j + 2);
+                if (j >= 1) ok = group_wait(j);
+                if (!ok) break;
+                load(&v_map, bar, v_tile, j * kTileRows, pr * p.Hkv + kvh);
+                if (j == 0) ok = group_wait(0);
+                if (!ok) break;
+                if (j + 1 < n_it) load(&k_map, bar, k_tile, (j + 1) * kTileRows, pr * p.Hkv + kvh);
                 else tc::mbar_arrive(bar);
             }
             if (!ok) sm_abort = 1;
@@ -159,54 +156,49 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
             constexpr uint32_t idesc_s = tc::idesc_bf16_f32(kTileRows, kTileRows);      // S[128 q x 128 keys]
             constexpr uint32_t idesc_o = tc::idesc_bf16_f32_b_mn(kTileRows, D);         // O[128 q x D]
             // A tcgen05.commit occupies the tensor pipe for about as long as a quarter of a 128 x 128 x 128
-            // MMA, so the work is issued in groups with ONE commit each: group 0 = S(0), group 1 = S(1),
-            // group it + 2 = { O += P(it) V(it), S(it + 2) }.  Completion of group g therefore tells the
-            // softmax warps that S(g) is ready and that the probability buffer of tile g - 2 is free, and
-            // the producer that K(g) and V(g - 2) are consumed.
-            bool ok = mbar_wait(smem_u32(&bar_q), 0);
-            auto issue_s = [&](int it) {                     // S_it = Q K_it^T into S buffer it & 1
-                const int s = it & 1, kv = it % kKvStages;
-                const uint32_t k_tile = stage0 + kv * kStageBytes;
-                // a descriptor's address field is (address >> 4), so stepping through a tile is an addition: the
-                // issuing thread's instruction count per MMA is what bounds this kernel
-                const uint64_t dq = tc::desc_k_major_sw128(q_tile), dk = tc::desc_k_major_sw128(k_tile);
+            // MMA, so the work is issued in groups with ONE commit each: group 0 = S(0),
+            // group it + 1 = { O += P(it) V(it), S(it + 1) }.  S(it + 1) overwrites the logits and probabilities of
+            // tile it, which P V has just read (the tensor pipe runs its work in order).  Completion of group g
+            // tells the softmax warps that S(g) is ready and the producer that K(g) and V(g - 1) are consumed.
+            // A descriptor's address field is (address >> 4), so stepping through a tile is an addition: the
+            // issuing thread's instruction count per MMA matters.
+            const uint64_t dq = tc::desc_k_major_sw128(q_tile), dk = tc::desc_k_major_sw128(k_tile);
+            const uint64_t dv = tc::desc_mn_major_sw128(v_tile, kBoxBytes);
+            auto issue_s = [&]() {
 #pragma unroll
                 for (int ks = 0; ks < kKSteps; ++ks) {
                     const uint32_t off = ((ks >> 2) * kBoxBytes + (ks & 3) * 32) >> 4;
-                    tc::umma_bf16(tmem_base + s * kTileRows, dq + off, dk + off, idesc_s, ks > 0);
+                    tc::umma_bf16(tmem_base, dq + off, dk + off, idesc_s, ks > 0);
                 }
             };
-            for (int g = 0; g < 2 && g < n_it && ok; ++g) {
-                ok = mbar_wait(smem_u32(&bar_k01[g]), 0);
-                if (!ok) break;
+            bool ok = mbar_wait(smem_u32(&bar_q), 0);
+            if (ok) ok = mbar_wait(smem_u32(&bar_k0), 0);
+            if (ok) {
                 tc::fence_after_sync();
-                issue_s(g);
-                tc::umma_commit(smem_u32(&bar_group[g % kGroupRing]));
+                issue_s();
+                tc::umma_commit(smem_u32(&bar_group[0]));
             }
             for (int it = 0; it < n_it && ok; ++it) {
-                const int s = it & 1, kv = it % kKvStages;
-                // P(it) is written (so S(it) has been read), V(it) and K(it + 2) have landed
+                // P(it) is written (so S(it) has been read), V(it) and K(it + 1) have landed
                 ok = mbar_wait(smem_u32(&bar_in[it % kGroupRing]), (it / kGroupRing) & 1);
                 if (!ok) break;
                 tc::fence_after_sync();
-                const uint32_t v_tile = stage0 + kv * kStageBytes + kTileBytes;
-                const uint64_t dv = tc::desc_mn_major_sw128(v_tile, kBoxBytes);
 #pragma unroll
-                for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step = 8 columns of the probability tile
-                    tc::umma_bf16_ts(tmem_base + kOColumn, tmem_base + kPColumn + s * kPColumns + ks * 8,
+                for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step = 8 columns of probabilities
+                    tc::umma_bf16_ts(tmem_base + kOColumn, tmem_base + (ks >> 2) * 64 + kPOffset + (ks & 3) * 8,
                                      dv + (ks * 2048 >> 4), idesc_o, (it > 0) || (ks > 0));
                 }
-                if (it + 2 < n_it) issue_s(it + 2);          // into the S buffer tile `it` has just left
-                tc::umma_commit(smem_u32(&bar_group[(it + 2) % kGroupRing]));
+                if (it + 1 < n_it) issue_s();
+                tc::umma_commit(smem_u32(&bar_group[(it + 1) % kGroupRing]));
             }
             if (!ok) sm_abort = 1;
         }
     } else {
         // ---------------- softmax warps: a warp reads its quarter of the TMEM lanes (thread = query row);
-        // warps 2-5 take keys 0..31 of every tile, warps 6-9 keys 32..63, and so on
+        // the first four of them take keys 0..63 of every tile, the others keys 64..127
         const int row = 32 * (warp & 3) + lane;
-        const int part = (warp - 2) >> 2;                     // 0 .. 3
-        const int col_base = part * 32;
+        const int part = (warp - 2) >> 2;                     // 0 .. 1
+        const int col_base = part * 64;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
         const int t = qb * kTileRows + row;
         // the softmax's reference logit of this row, log2 domain (exact mode: the row's maximum; +inf past the prompt)
@@ -214,13 +206,11 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
         if (kExact) lse = t < p.T ? p.lse2[((int64_t)pr * p.Hq + h) * p.T + t] : INFINITY;
         bool ok = true;
         for (int it = 0; it < n_it; ++it) {
-            const int s = it & 1;
-            if (!group_wait(it)) { ok = false; break; }        // S(it) is ready and P V of tile it - 2 has read its P
+            if (!group_wait(it)) { ok = false; break; }        // S(it) is ready
             tc::fence_after_sync();
-            uint32_t v[32];
             if (!kExact && it == 0) {
                 // reference = the row's largest logit among the first eight keys (those of them it may see):
-                // every thread of the row reads the same eight columns, so the four agree without talking
+                // every thread of the row reads the same eight columns, so the two agree without talking
                 uint32_t first[8];
                 tc::tmem_ld_32x32_x8(lane_addr, first);
                 tc::tmem_ld_wait();
@@ -230,68 +220,79 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
                     if (qb > 0 || c <= row) mx = fmaxf(mx, __uint_as_float(first[c]));
                 lse = mx * p.scale_log2;
             }
-            tc::tmem_ld_32x32(lane_addr + s * kTileRows + col_base, v);
-            tc::tmem_ld_wait();
-            if (it == qb) {                                   // diagonal tile: keys above the query do not exist
+            // probabilities of this thread's 64 keys -> bf16, two per 32-bit column of the A operand
+            uint32_t w[32];
 #pragma unroll
-                for (int c = 0; c < 32; ++c)
-                    if (col_base + c > row) v[c] = 0xff800000u;
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t v[32];
+                tc::tmem_ld_32x32(lane_addr + col_base + hh * 32, v);
+                tc::tmem_ld_wait();
+                if (it == qb) {                               // diagonal tile: keys above the query do not exist
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (col_base + hh * 32 + c > row) v[c] = 0xff800000u;
+                }
+#pragma unroll
+                for (int c = 0; c < 16; ++c)
+                    w[hh * 16 + c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(v[2 * c]), p.scale_log2, -lse)),
+                                               fast_exp2(fmaf(__uint_as_float(v[2 * c + 1]), p.scale_log2, -lse)));
             }
-            // probabilities of this thread's 32 keys -> bf16, two per 32-bit column of the A operand
-            uint32_t w[16];
+            // (all 64 logits are in registers by now: the stores go over the second half of them)
+            {
+                uint32_t w0[16], w1[16];
 #pragma unroll
-            for (int c = 0; c < 16; ++c)
-                w[c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(v[2 * c]), p.scale_log2, -lse)),
-                                 fast_exp2(fmaf(__uint_as_float(v[2 * c + 1]), p.scale_log2, -lse)));
-            tc::tmem_st_32x32_x16(lane_addr + kPColumn + s * kPColumns + part * 16, w);
+                for (int c = 0; c < 16; ++c) { w0[c] = w[c]; w1[c] = w[16 + c]; }
+                tc::tmem_st_32x32_x16(lane_addr + col_base + kPOffset, w0);
+                tc::tmem_st_32x32_x16(lane_addr + col_base + kPOffset + 16, w1);
+            }
             tc::tmem_st_wait();
             tc::fence_before_sync();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(smem_u32(&bar_in[it % kGroupRing]));
         }
-        // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile.
-        // Four threads per row take 32 columns of the head dimension each (two of them when D = 64).
-        if (ok) ok = group_wait(n_it + 1);                    // the last group: O is complete
+        // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile,
+        // the last one loaded.  Two threads per row take half of the head dimension each.
+        if (ok) ok = group_wait(n_it);                        // the last group: O is complete
         float dot = 0.0f, vv = 0.0f, oo = 0.0f;
-        if (ok && part * 32 < D) {
+        if (ok) {
             tc::fence_after_sync();
-            const uint8_t* v_row = base_ptr + (stage0 - base) + (qb % kKvStages) * kStageBytes + kTileBytes + row * 128;
-            uint32_t o[32];
-            tc::tmem_ld_32x32(lane_addr + kOColumn + part * 32, o);
-            tc::tmem_ld_wait();
+            const uint8_t* v_row = base_ptr + 2 * kTileBytes + row * 128;
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {                  // 16-byte pieces of 8 elements
-                const int piece = part * 4 + cc;              // within the row: 0 .. D/8 - 1
-                const uint4 raw = *reinterpret_cast<const uint4*>(v_row + (piece >> 3) * kBoxBytes +
-                                                                  (((piece & 7) ^ (row & 7)) << 4));
-                const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+            for (int ch = 0; ch < D / 64; ++ch) {             // 32 columns of the head dimension at a time
+                const int col0 = part * (D / 2) + ch * 32;
+                uint32_t o[32];
+                tc::tmem_ld_32x32(lane_addr + kOColumn + col0, o);
+                tc::tmem_ld_wait();
 #pragma unroll
-                for (int k2 = 0; k2 < 4; ++k2) {
-                    const float2 vx = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[k2]));
-                    const float o0 = __uint_as_float(o[cc * 8 + k2 * 2]), o1 = __uint_as_float(o[cc * 8 + k2 * 2 + 1]);
-                    dot = fmaf(vx.x, o0, fmaf(vx.y, o1, dot));
-                    vv = fmaf(vx.x, vx.x, fmaf(vx.y, vx.y, vv));
-                    oo = fmaf(o0, o0, fmaf(o1, o1, oo));
+                for (int cc = 0; cc < 4; ++cc) {              // 16-byte pieces of 8 elements
+                    const int piece = col0 / 8 + cc;          // within the row: 0 .. D/8 - 1
+                    const uint4 raw = *reinterpret_cast<const uint4*>(v_row + (piece >> 3) * kBoxBytes +
+                                                                      (((piece & 7) ^ (row & 7)) << 4));
+                    const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int k2 = 0; k2 < 4; ++k2) {
+                        const float2 vx = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[k2]));
+                        const float o0 = __uint_as_float(o[cc * 8 + k2 * 2]), o1 = __uint_as_float(o[cc * 8 + k2 * 2 + 1]);
+                        dot = fmaf(vx.x, o0, fmaf(vx.y, o1, dot));
+                        vv = fmaf(vx.x, vx.x, fmaf(vx.y, vx.y, vv));
+                        oo = fmaf(o0, o0, fmaf(o1, o1, oo));
+                    }
                 }
             }
         }
-        // join the four parts of every row through shared memory (the stage without the diagonal tile is idle)
-        float* sm_part = reinterpret_cast<float*>(base_ptr + (stage0 - base) + ((qb + 1) % kKvStages) * kStageBytes);   // [3][4][128]
-        sm_part[(0 * 4 + part) * kTileRows + row] = dot;
-        sm_part[(1 * 4 + part) * kTileRows + row] = vv;
-        sm_part[(2 * 4 + part) * kTileRows + row] = oo;
-        asm volatile("bar.sync 1, 512;" ::: "memory");
+        // join the two halves of every row through shared memory (the K tile is idle by now)
+        float* sm_part = reinterpret_cast<float*>(base_ptr + kTileBytes);   // [3][2][128]
+        sm_part[(0 * 2 + part) * kTileRows + row] = dot;
+        sm_part[(1 * 2 + part) * kTileRows + row] = vv;
+        sm_part[(2 * 2 + part) * kTileRows + row] = oo;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         float c = 0.0f;
         if (part == 0 && ok && t < len) {
-            float d4 = 0.0f, v4 = 0.0f, o4 = 0.0f;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                d4 += sm_part[(0 * 4 + k) * kTileRows + row];
-                v4 += sm_part[(1 * 4 + k) * kTileRows + row];
-                o4 += sm_part[(2 * 4 + k) * kTileRows + row];
-            }
-            c = d4 / fmaxf(sqrtf(v4) * sqrtf(o4), kCosEps);
-            if (!kExact && !(fabsf(d4) <= 3.0e38f && o4 <= 3.0e38f)) {   // left the fp32 range (or NaN): redo this block
+            const float d2 = sm_part[(0 * 2 + 0) * kTileRows + row] + sm_part[(0 * 2 + 1) * kTileRows + row];
+            const float v2 = sm_part[(1 * 2 + 0) * kTileRows + row] + sm_part[(1 * 2 + 1) * kTileRows + row];
+            const float o2 = sm_part[(2 * 2 + 0) * kTileRows + row] + sm_part[(2 * 2 + 1) * kTileRows + row];
+            c = d2 / fmaxf(sqrtf(v2) * sqrtf(o2), kCosEps);
+            if (!kExact && !(fabsf(d2) <= 3.0e38f && o2 <= 3.0e38f)) {   // left the fp32 range (or NaN): redo this block
                 sm_redo = 1;
                 c = 0.0f;
             }
@@ -315,7 +316,7 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
         if (again) p.redo_list[atomicAdd(p.redo_count, 1)] = (pr * p.Hq + h) * p.n_blk + qb;
         // the barriers may be set up again by the next row block of this CTA (exact mode)
         mbar_inval(smem_u32(&bar_q));
-        for (int s = 0; s < 2; ++s) mbar_inval(smem_u32(&bar_k01[s]));
+        mbar_inval(smem_u32(&bar_k0));
         for (int s = 0; s < kGroupRing; ++s) {
             mbar_inval(smem_u32(&bar_in[s]));
             mbar_inval(smem_u32(&bar_group[s]));
@@ -326,7 +327,7 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
 
 // One pass over every row block of the layer: grid (row blocks, query heads, prompts), long blocks first.
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfileParams p,
+__global__ void __launch_bounds__(kThreads, 2) profile_pv_kernel(const ProfileParams p,
                                                                  const __grid_constant__ CUtensorMap q_map,
                                                                  const __grid_constant__ CUtensorMap k_map,
                                                                  const __grid_constant__ CUtensorMap v_map) {
@@ -336,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) profile_pv_kernel(const ProfilePa
 // The exact form over the row blocks the one-pass kernel listed: a small fixed grid whose CTAs take the
 // entries in turn, so that the usual empty list costs nothing.
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1) profile_pv_redo_kernel(const ProfileParams p,
+__global__ void __launch_bounds__(kThreads, 2) profile_pv_redo_kernel(const ProfileParams p,
                                                                       const __grid_constant__ CUtensorMap q_map,
                                                                       const __grid_constant__ CUtensorMap k_map,
                                                                       const __grid_constant__ CUtensorMap v_map) {
@@ -363,8 +364,8 @@ constexpr int kRedoGrid = 148;        // CTAs that share the list of row blocks 
 template <int D, bool kExact>
 cudaError_t launch_profile(const ProfileParams& p, const CUtensorMap& qm, const CUtensorMap& km, const CUtensorMap& vm,
                            cudaStream_t s) {
-    // Q tile and the (K, V) stages
-    constexpr int kSmem = kTileRows * D * 2 * (1 + 2 * kKvStages) + 1024;
+    // the Q, K and V tiles; at least 80 KB, so that never more than two CTAs (2 x 256 TMEM columns) share an SM
+    constexpr int kSmem = (3 * kTileRows * D * 2 + 1024) > 80 * 1024 ? (3 * kTileRows * D * 2 + 1024) : 80 * 1024;
     if (kExact) {
         cudaError_t e = cudaFuncSetAttribute(profile_pv_redo_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
         if (e != cudaSuccess) return e;
