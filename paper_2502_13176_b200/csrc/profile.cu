@@ -75,12 +75,12 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
     constexpr int kBoxBytes = kTileRows * 128;               // one TMA box: 128 rows x 64 elements
     constexpr int kTileBytes = kTileRows * D * 2;            // a Q, K or V tile
     constexpr uint32_t kOColumn = kTileRows;                 // O sits after S in tensor memory
-    // A thread turns its 64 logits (64 columns) into 64 probabilities in bf16 (32 columns) and writes them into the
-    // upper half of its own 64 columns once it has read all of them: nobody else reads or writes those, and the
-    // tile's first columns, which every thread of a row reads for the reference, stay as they are.
-    constexpr uint32_t kPOffset = 32;
+    // A thread turns its 64 logits (64 columns) into 64 probabilities in bf16 in two halves, and writes each half
+    // (16 columns) over the first columns of the 32 logits it came from: nobody else reads or writes those (but for
+    // the tile's first columns, which every thread of a row reads once for the reference, see below).  The MMA
+    // thread is told about each half by itself, so that P V of the first half runs while the second is computed.
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q, bar_k0, bar_in[kGroupRing], bar_group[kGroupRing];
+    __shared__ __align__(8) uint64_t bar_q, bar_k0, bar_pa[kGroupRing], bar_pb[kGroupRing], bar_group[kGroupRing];
     __shared__ uint32_t tmem_slot;
     __shared__ float sm_warp_sum[kSoftmaxWarps];
     __shared__ int sm_abort;
@@ -103,7 +103,8 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
         mbar_init(smem_u32(&bar_q), 1);
         mbar_init(smem_u32(&bar_k0), 1);
         for (int s = 0; s < kGroupRing; ++s) {
-            mbar_init(smem_u32(&bar_in[s]), kSoftmaxWarps + 2);   // P(it) written, V(it) landed, K(it + 1) landed
+            mbar_init(smem_u32(&bar_pa[s]), kSoftmaxWarps + 1);   // first half of P(it) written, V(it) landed
+            mbar_init(smem_u32(&bar_pb[s]), kSoftmaxWarps + 1);   // second half of P(it) written, K(it + 1) landed
             mbar_init(smem_u32(&bar_group[s]), 1);
         }
         sm_abort = 0;
@@ -132,19 +133,19 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
             };
             load(&q_map, smem_u32(&bar_q), q_tile, qb * kTileRows, pr * p.Hq + h);
             load(&k_map, smem_u32(&bar_k0), k_tile, 0, pr * p.Hkv + kvh);
-            // The MMA thread pays well over a hundred cycles for every mbarrier it looks at, so everything group
-            // it + 1 = { P(it) V(it), S(it + 1) } needs arrives on ONE barrier, bar_in[it % 4]: the eight softmax warps
-            // (P(it) written) and the two loads V(it) and K(it + 1).  There is one K and one V tile: K(j + 1) takes
-            // the place of K(j) once S(j) is complete and V(j) that of V(j - 1) once P V of tile j - 1 is, and both
-            // are in MMA group j.
+            // The MMA thread pays well over a hundred cycles for every mbarrier it looks at, so what it needs for
+            // tile `it` arrives on TWO barriers: bar_pa[it % 4] collects the eight softmax warps (first half of P(it)
+            // written) and the load V(it), bar_pb[it % 4] the same warps (second half) and the load K(it + 1).  There
+            // is one K and one V tile: K(j + 1) takes the place of K(j) once S(j) is complete and V(j) that of
+            // V(j - 1) once P V of tile j - 1 is, and both are in MMA group j.
             bool ok = true;
             for (int j = 0; j < n_it && ok; ++j) {
-                const uint32_t bar = smem_u32(&bar_in[j % kGroupRing]);
                 if (j >= 1) ok = group_wait(j);
                 if (!ok) break;
-                load(&v_map, bar, v_tile, j * kTileRows, pr * p.Hkv + kvh);
+                load(&v_map, smem_u32(&bar_pa[j % kGroupRing]), v_tile, j * kTileRows, pr * p.Hkv + kvh);
                 if (j == 0) ok = group_wait(0);
                 if (!ok) break;
+                const uint32_t bar = smem_u32(&bar_pb[j % kGroupRing]);
                 if (j + 1 < n_it) load(&k_map, bar, k_tile, (j + 1) * kTileRows, pr * p.Hkv + kvh);
                 else tc::mbar_arrive(bar);
             }
@@ -179,15 +180,25 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
                 tc::umma_commit(smem_u32(&bar_group[0]));
             }
             for (int it = 0; it < n_it && ok; ++it) {
-                // P(it) is written (so S(it) has been read), V(it) and K(it + 1) have landed
-                ok = mbar_wait(smem_u32(&bar_in[it % kGroupRing]), (it / kGroupRing) & 1);
+                // 16 keys per step = 8 columns of probabilities; a thread's halves are keys 0..31 and 32..63 of its 64
+                auto issue_pv = [&](int hh) {
+#pragma unroll
+                    for (int k4 = 0; k4 < kPvSteps / 2; ++k4) {
+                        const int ks = (k4 >> 1) * 4 + hh * 2 + (k4 & 1);
+                        tc::umma_bf16_ts(tmem_base + kOColumn, tmem_base + (ks >> 2) * 64 + hh * 32 + (ks & 1) * 8,
+                                         dv + (ks * 2048 >> 4), idesc_o, (it > 0) || (hh > 0) || (k4 > 0));
+                    }
+                };
+                // the first half of P(it) is written and V(it) has landed
+                ok = mbar_wait(smem_u32(&bar_pa[it % kGroupRing]), (it / kGroupRing) & 1);
                 if (!ok) break;
                 tc::fence_after_sync();
-#pragma unroll
-                for (int ks = 0; ks < kPvSteps; ++ks) {      // 16 keys per step = 8 columns of probabilities
-                    tc::umma_bf16_ts(tmem_base + kOColumn, tmem_base + (ks >> 2) * 64 + kPOffset + (ks & 3) * 8,
-                                     dv + (ks * 2048 >> 4), idesc_o, (it > 0) || (ks > 0));
-                }
+                issue_pv(0);
+                // the second half is written (so all of S(it) has been read) and K(it + 1) has landed
+                ok = mbar_wait(smem_u32(&bar_pb[it % kGroupRing]), (it / kGroupRing) & 1);
+                if (!ok) break;
+                tc::fence_after_sync();
+                issue_pv(1);
                 if (it + 1 < n_it) issue_s();
                 tc::umma_commit(smem_u32(&bar_group[(it + 1) % kGroupRing]));
             }
@@ -219,9 +230,10 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
                 for (int c = 1; c < 8; ++c)
                     if (qb > 0 || c <= row) mx = fmaxf(mx, __uint_as_float(first[c]));
                 lse = mx * p.scale_log2;
+                // (the first probabilities go over these columns: not before every thread has read them)
+                asm volatile("bar.sync 1, 256;" ::: "memory");
             }
             // probabilities of this thread's 64 keys -> bf16, two per 32-bit column of the A operand
-            uint32_t w[32];
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
                 uint32_t v[32];
@@ -232,23 +244,17 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
                     for (int c = 0; c < 32; ++c)
                         if (col_base + hh * 32 + c > row) v[c] = 0xff800000u;
                 }
+                uint32_t w[16];
 #pragma unroll
                 for (int c = 0; c < 16; ++c)
-                    w[hh * 16 + c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(v[2 * c]), p.scale_log2, -lse)),
-                                               fast_exp2(fmaf(__uint_as_float(v[2 * c + 1]), p.scale_log2, -lse)));
+                    w[c] = pack_bf16(fast_exp2(fmaf(__uint_as_float(v[2 * c]), p.scale_log2, -lse)),
+                                     fast_exp2(fmaf(__uint_as_float(v[2 * c + 1]), p.scale_log2, -lse)));
+                tc::tmem_st_32x32_x16(lane_addr + col_base + hh * 32, w);
+                tc::tmem_st_wait();
+                tc::fence_before_sync();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(smem_u32(hh == 0 ? &bar_pa[it % kGroupRing] : &bar_pb[it % kGroupRing]));
             }
-            // (all 64 logits are in registers by now: the stores go over the second half of them)
-            {
-                uint32_t w0[16], w1[16];
-#pragma unroll
-                for (int c = 0; c < 16; ++c) { w0[c] = w[c]; w1[c] = w[16 + c]; }
-                tc::tmem_st_32x32_x16(lane_addr + col_base + kPOffset, w0);
-                tc::tmem_st_32x32_x16(lane_addr + col_base + kPOffset + 16, w1);
-            }
-            tc::tmem_st_wait();
-            tc::fence_before_sync();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(smem_u32(&bar_in[it % kGroupRing]));
         }
         // ---- O is complete: cosine between V_t and O_t; the V rows of this CTA's tokens are the diagonal tile,
         // the last one loaded.  Two threads per row take half of the head dimension each.
@@ -318,7 +324,8 @@ __device__ __forceinline__ void profile_pv_block(const ProfileParams& p, const C
         mbar_inval(smem_u32(&bar_q));
         mbar_inval(smem_u32(&bar_k0));
         for (int s = 0; s < kGroupRing; ++s) {
-            mbar_inval(smem_u32(&bar_in[s]));
+            mbar_inval(smem_u32(&bar_pa[s]));
+            mbar_inval(smem_u32(&bar_pb[s]));
             mbar_inval(smem_u32(&bar_group[s]));
         }
     }
