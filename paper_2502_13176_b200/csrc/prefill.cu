@@ -57,7 +57,7 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_res, bar_full[2], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
-    __shared__ float sm_lse[2][2][kTileRows];              // [group][tile parity inside the group][streamed row]
+    __shared__ __align__(16) float sm_lse[2][2][kTileRows];   // [group][tile parity inside the group][streamed row]
     __shared__ int sm_abort;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -251,10 +251,16 @@ __device__ __forceinline__ void qk_pass_block(const PrefillParams& p, const CUte
                         }
                     }
                     float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                    const float4* lse4 = reinterpret_cast<const float4*>(lse + c0);
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        sum[c & 3] += fast_exp2(fmaf(__uint_as_float(v0[c]), p.scale_log2, -lse[c0 + c]));
-                        sum[(c + 2) & 3] += fast_exp2(fmaf(__uint_as_float(v1[c]), p.scale_log2, -lse[c0 + 32 + c]));
+                    for (int c4 = 0; c4 < 8; ++c4) {           // four streamed rows' log-sum-exp per shared-memory load
+                        const float4 la = lse4[c4], lb = lse4[8 + c4];
+                        const float l0[4] = {la.x, la.y, la.z, la.w}, l1[4] = {lb.x, lb.y, lb.z, lb.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            sum[k] += fast_exp2(fmaf(__uint_as_float(v0[4 * c4 + k]), p.scale_log2, -l0[k]));
+                            sum[(k + 2) & 3] += fast_exp2(fmaf(__uint_as_float(v1[4 * c4 + k]), p.scale_log2, -l1[k]));
+                        }
                     }
                     colsum += (sum[0] + sum[1]) + (sum[2] + sum[3]);
                 }
